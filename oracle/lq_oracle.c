@@ -1,0 +1,602 @@
+/*
+ * CPU oracle for the per-window 8-bit decode step of Gated DeltaNet (scalar
+ * gate) and Kimi Delta Attention (per-channel gate) recurrent states.
+ *
+ * THIS FILE IS TEST INFRASTRUCTURE.  It is the slow, plain statement of what
+ * the method computes, written from the paper, and is what the GPU library is
+ * checked against.  Only the tests, the smoke check and the benchmark's CPU
+ * baseline leg may build or call it; the product never does.  It shares no
+ * code, header, table or helper with the CUDA path.
+ *
+ * Orientation (Sec. 3.1, Eq. 1): one head has state S in R^{d_k x d_v},
+ * stored row-major S[i*d_v + j] with i the key index and j the value index;
+ * the readout is o = S^T q.
+ *
+ * Arithmetic: IEEE binary32, round to nearest even, compiled with
+ * -ffp-contract=off so that a product is fused with an addition only where
+ * fmaf() is written.  bf16 inputs and fp16 compensators are widened exactly.
+ *
+ * Summation order.  The paper never says in which order a sum is taken, yet
+ * the 8-bit codes and the fp16 compensators are step functions of fp32
+ * values, so the order has to be part of the definition.  Every reduction in
+ * this file goes through csum_dot()/csum_abs(): consecutive blocks of eight
+ * terms are accumulated left to right (first product rounded, the others
+ * folded in with fmaf), and the block results are then added as a balanced
+ * binary tree over the block index (neighbours first).  Building the file
+ * with -DLQO_WIDE replaces this by a plain left-to-right sum in binary64,
+ * rounded once; comparing the two builds measures how much of any
+ * disagreement is attributable to fp32 summation order.
+ *
+ * Parity status of the pieces (what pins each is listed in the tests):
+ *   reference recurrence, windowed decode, reconstruction, quantizer,
+ *   smoothing, rank-r fit as a Frobenius minimiser        : pinned
+ *   the constants n_iter, the all-equal start vector, the 1e-30 zero guard,
+ *   the 1e-6 smoothing floor, the summation tree          : parity unpinned
+ *   (the paper fixes none of them; they are this build's definition).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+enum { LQO_GATE_SCALAR = 0, LQO_GATE_DIAG = 1 };
+
+typedef struct {
+  int batch;     /* sequences                                              */
+  int heads_v;   /* value heads per sequence (one state each)               */
+  int heads_qk;  /* query/key heads per sequence; heads_v % heads_qk == 0   */
+  int d_k, d_v;  /* state is d_k x d_v                                      */
+  int W;         /* window length p                                         */
+  int r;         /* Compensator Tokens per state                            */
+  int n_iter;    /* power-iteration steps per compensator (>= 1)            */
+  int gate;      /* LQO_GATE_SCALAR (GDN) or LQO_GATE_DIAG (KDA)            */
+  int smooth;    /* 1: residual smoothing (Sec. 3.4); 0: c == 1             */
+} lqo_shape;
+
+typedef struct {
+  int8_t *codes;        /* [B,Hv,d_k,d_v]  Z                                */
+  float *col_scale;     /* [B,Hv,d_v]      B, per value channel             */
+  float *row_smooth;    /* [B,Hv,d_k]      c, per key row                   */
+  uint16_t *comp_k;     /* [B,Hv,r,d_k]    fp16 bit patterns                */
+  uint16_t *comp_u;     /* [B,Hv,r,d_v]    fp16 bit patterns                */
+  float *buf_k;         /* [B,Hv,W,d_k]    write keys beta*k                */
+  float *buf_u;         /* [B,Hv,W,d_v]    corrections u                    */
+  float *buf_a;         /* [B,Hv,W] (scalar gate) or [B,Hv,W,d_k] (diag)    */
+  int32_t *win_pos;     /* [B]             records buffered, 0..W-1 at rest */
+  float *S0;            /* [B,Hv,d_k,d_v]  only for the no-quantization mode*/
+} lqo_state;
+
+/* ------------------------------------------------------------------ */
+/* number formats                                                      */
+/* ------------------------------------------------------------------ */
+
+static float bits_f32(uint32_t u) { float f; memcpy(&f, &u, 4); return f; }
+static uint32_t f32_bits(float f) { uint32_t u; memcpy(&u, &f, 4); return u; }
+
+/* bf16 is the upper half of a binary32. */
+static float bf16_to_f32(uint16_t h) { return bits_f32((uint32_t)h << 16); }
+
+/* binary32 -> bfloat16, round to nearest even (used by the bf16-state baseline). */
+uint16_t lqo_f32_to_bf16(float f) {
+  uint32_t x = f32_bits(f);
+  if ((x & 0x7FFFFFFFu) > 0x7F800000u) return (uint16_t)((x >> 16) | 0x0040u);
+  uint32_t keep = x >> 16, rest = x & 0xFFFFu;
+  if (rest > 0x8000u || (rest == 0x8000u && (keep & 1u))) keep++;
+  return (uint16_t)keep;
+}
+
+/* binary16 -> binary32, exact. */
+float lqo_f16_to_f32(uint16_t h) {
+  uint32_t sign = (uint32_t)(h & 0x8000u) << 16;
+  int e = (h >> 10) & 0x1F;
+  uint32_t m = h & 0x3FFu;
+  if (e == 31) return bits_f32(sign | 0x7F800000u | (m << 13));
+  if (e == 0) {
+    /* subnormal: m * 2^-24, exact in binary32 */
+    float mag = (float)m * 5.9604644775390625e-08f;
+    return sign ? -mag : mag;
+  }
+  return bits_f32(sign | ((uint32_t)(e - 15 + 127) << 23) | (m << 13));
+}
+
+/* binary32 -> binary16, round to nearest even; overflow goes to infinity
+ * (callers that must not overflow clamp to +-65504 first). */
+uint16_t lqo_f32_to_f16(float f) {
+  uint32_t x = f32_bits(f);
+  uint16_t sign = (uint16_t)((x >> 16) & 0x8000u);
+  uint32_t mag = x & 0x7FFFFFFFu;
+  if (mag > 0x7F800000u) return (uint16_t)(sign | 0x7E00u);          /* NaN  */
+  if (mag >= 0x477FF000u) return (uint16_t)(sign | 0x7C00u);         /* >= 65520 */
+  if (mag <= 0x33000000u) return sign;                               /* <= 2^-25 */
+  int e = (int)(mag >> 23) - 127;
+  uint32_t m24 = (mag & 0x7FFFFFu) | 0x800000u;  /* 1.m as a 24-bit integer */
+  int drop;            /* low bits of m24 that do not fit                    */
+  uint32_t out;
+  if (e >= -14) {
+    drop = 13;
+    out = ((uint32_t)(e + 15) << 10) + ((m24 >> 13) - 0x400u);
+  } else {
+    drop = 13 + (-14 - e);
+    out = m24 >> drop;
+  }
+  uint32_t rem = m24 & ((1u << drop) - 1u), half = 1u << (drop - 1);
+  if (rem > half || (rem == half && (out & 1u))) out++;  /* a carry moves into the exponent */
+  return (uint16_t)(sign | out);
+}
+
+static float clamp_f16_range(float x) { return fminf(fmaxf(x, -65504.0f), 65504.0f); }
+
+/* ------------------------------------------------------------------ */
+/* the one place where sums are taken                                  */
+/* ------------------------------------------------------------------ */
+
+/* sum_i a[i]*b[i], i = 0..n-1 */
+float lqo_csum_dot(const float *a, const float *b, int n) {
+#ifdef LQO_WIDE
+  double acc = 0.0;
+  for (int i = 0; i < n; i++) acc += (double)a[i] * (double)b[i];
+  return (float)acc;
+#else
+  if (n <= 0) return 0.0f;
+  int nblk = (n + 7) / 8, width = 1;
+  while (width < nblk) width *= 2;
+  float *part = (float *)malloc(sizeof(float) * (size_t)width);
+  for (int c = 0; c < width; c++) {
+    float acc = 0.0f;
+    if (c < nblk) {
+      int lo = 8 * c, hi = lo + 8 < n ? lo + 8 : n;
+      acc = a[lo] * b[lo];
+      for (int i = lo + 1; i < hi; i++) acc = fmaf(a[i], b[i], acc);
+    }
+    part[c] = acc;
+  }
+  for (; width > 1; width /= 2)
+    for (int c = 0; c < width / 2; c++) part[c] = part[2 * c] + part[2 * c + 1];
+  float s = part[0];
+  free(part);
+  return s;
+#endif
+}
+
+/* sum_i |x[i]|, same order */
+float lqo_csum_abs(const float *x, int n) {
+#ifdef LQO_WIDE
+  double acc = 0.0;
+  for (int i = 0; i < n; i++) acc += fabs((double)x[i]);
+  return (float)acc;
+#else
+  if (n <= 0) return 0.0f;
+  int nblk = (n + 7) / 8, width = 1;
+  while (width < nblk) width *= 2;
+  float *part = (float *)malloc(sizeof(float) * (size_t)width);
+  for (int c = 0; c < width; c++) {
+    float acc = 0.0f;
+    if (c < nblk) {
+      int lo = 8 * c, hi = lo + 8 < n ? lo + 8 : n;
+      acc = fabsf(x[lo]);
+      for (int i = lo + 1; i < hi; i++) acc = acc + fabsf(x[i]);
+    }
+    part[c] = acc;
+  }
+  for (; width > 1; width /= 2)
+    for (int c = 0; c < width / 2; c++) part[c] = part[2 * c] + part[2 * c + 1];
+  float s = part[0];
+  free(part);
+  return s;
+#endif
+}
+
+/* column j of a row-major d_k x d_v matrix, gathered so that it can be summed */
+static void column_of(const float *M, int d_k, int d_v, int j, float *out) {
+  for (int i = 0; i < d_k; i++) out[i] = M[(size_t)i * d_v + j];
+}
+
+/* ------------------------------------------------------------------ */
+/* per-head views                                                      */
+/* ------------------------------------------------------------------ */
+
+typedef struct {
+  int8_t *Z; float *B, *c; uint16_t *ck, *cu; float *bk, *bu, *ba; float *S0;
+} head_view;
+
+static head_view view_of(const lqo_shape *sh, const lqo_state *st, int b, int h) {
+  size_t bh = (size_t)b * sh->heads_v + h;
+  size_t K = sh->d_k, V = sh->d_v, W = sh->W, r = sh->r;
+  size_t na = sh->gate == LQO_GATE_DIAG ? K : 1;
+  head_view hv;
+  hv.Z = st->codes ? st->codes + bh * K * V : NULL;
+  hv.B = st->col_scale ? st->col_scale + bh * V : NULL;
+  hv.c = st->row_smooth ? st->row_smooth + bh * K : NULL;
+  hv.ck = st->comp_k ? st->comp_k + bh * r * K : NULL;
+  hv.cu = st->comp_u ? st->comp_u + bh * r * V : NULL;
+  hv.bk = st->buf_k + bh * W * K;
+  hv.bu = st->buf_u + bh * W * V;
+  hv.ba = st->buf_a + bh * W * na;
+  hv.S0 = st->S0 ? st->S0 + bh * K * V : NULL;
+  return hv;
+}
+
+/* decay of record j as a d_k vector (a scalar gate is the same value on every key channel) */
+static void record_decay(const lqo_shape *sh, const head_view *hv, int j, float *out) {
+  for (int i = 0; i < sh->d_k; i++)
+    out[i] = sh->gate == LQO_GATE_DIAG ? hv->ba[(size_t)j * sh->d_k + i] : hv->ba[j];
+}
+
+/* the token's inputs for value head h of sequence b, widened to binary32 */
+typedef struct { float *q, *k, *v, *a; float beta; } token_in;
+
+static token_in token_alloc(const lqo_shape *sh) {
+  token_in t;
+  t.q = (float *)malloc(sizeof(float) * sh->d_k);
+  t.k = (float *)malloc(sizeof(float) * sh->d_k);
+  t.a = (float *)malloc(sizeof(float) * sh->d_k);
+  t.v = (float *)malloc(sizeof(float) * sh->d_v);
+  t.beta = 0.0f;
+  return t;
+}
+static void token_free(token_in *t) { free(t->q); free(t->k); free(t->a); free(t->v); }
+
+static void token_load(const lqo_shape *sh, int b, int h, const uint16_t *q, const uint16_t *k,
+                       const uint16_t *v, const uint16_t *beta, const uint16_t *alpha, token_in *t) {
+  int K = sh->d_k, V = sh->d_v;
+  int group = sh->heads_v / sh->heads_qk;
+  size_t qk_off = ((size_t)b * sh->heads_qk + h / group) * K;  /* value head h reads q/k head h/group */
+  size_t bh = (size_t)b * sh->heads_v + h;
+  for (int i = 0; i < K; i++) {
+    t->q[i] = bf16_to_f32(q[qk_off + i]);
+    t->k[i] = bf16_to_f32(k[qk_off + i]);
+    t->a[i] = sh->gate == LQO_GATE_DIAG ? bf16_to_f32(alpha[bh * K + i]) : bf16_to_f32(alpha[bh]);
+  }
+  for (int j = 0; j < V; j++) t->v[j] = bf16_to_f32(v[bh * V + j]);
+  t->beta = bf16_to_f32(beta[bh]);
+}
+
+/* ------------------------------------------------------------------ */
+/* Eq. 1 with the GDN / KDA coefficients of Table 4 (Appendix A):      */
+/*   write key kt = beta*k, read vector b = alpha (.) k,               */
+/*   u = v - S^T b,  S <- Diag(alpha) S + kt u^T,  o = S^T q           */
+/* ------------------------------------------------------------------ */
+static void head_ref_step(const lqo_shape *sh, float *S, const token_in *t, float *o) {
+  int K = sh->d_k, V = sh->d_v;
+  float *kt = (float *)malloc(sizeof(float) * K), *bv = (float *)malloc(sizeof(float) * K);
+  float *col = (float *)malloc(sizeof(float) * K), *u = (float *)malloc(sizeof(float) * V);
+  for (int i = 0; i < K; i++) { kt[i] = t->beta * t->k[i]; bv[i] = t->a[i] * t->k[i]; }
+  for (int j = 0; j < V; j++) {
+    column_of(S, K, V, j, col);
+    u[j] = t->v[j] - lqo_csum_dot(col, bv, K);
+  }
+  for (int i = 0; i < K; i++)
+    for (int j = 0; j < V; j++) S[(size_t)i * V + j] = fmaf(kt[i], u[j], t->a[i] * S[(size_t)i * V + j]);
+  for (int j = 0; j < V; j++) {
+    column_of(S, K, V, j, col);
+    o[j] = lqo_csum_dot(col, t->q, K);
+  }
+  free(kt); free(bv); free(col); free(u);
+}
+
+/* ------------------------------------------------------------------ */
+/* Reconstruction of the state after the n buffered records, Eq. 7      */
+/* (Eq. 4 when there is no smoothing and no compensator):               */
+/*   S_n = Gamma_{1:n} [ C dequant(Z) + Kc Uc^T ] + sum_j Gamma_{j+1:n} kt_j u_j^T
+ * with dequant(Z) = (Z/127) B (Appendix B.3).  The cumulative decays are
+ * built up record by record from the newest one, as Appendix B.2 describes. */
+/* ------------------------------------------------------------------ */
+static void head_reconstruct(const lqo_shape *sh, const head_view *hv, int n, float *S) {
+  int K = sh->d_k, V = sh->d_v, r = sh->r;
+  float *gam = (float *)malloc(sizeof(float) * K);               /* Gamma_{j+1:n}, ends as Gamma_{1:n} */
+  float *kd = (float *)malloc(sizeof(float) * (size_t)(n > 0 ? n : 1) * K); /* Gamma_{j+1:n} kt_j       */
+  float *dec = (float *)malloc(sizeof(float) * K);
+  for (int i = 0; i < K; i++) gam[i] = 1.0f;
+  for (int j = n - 1; j >= 0; j--) {
+    record_decay(sh, hv, j, dec);
+    for (int i = 0; i < K; i++) {
+      kd[(size_t)j * K + i] = gam[i] * hv->bk[(size_t)j * K + i];
+      gam[i] = gam[i] * dec[i];
+    }
+  }
+  for (int i = 0; i < K; i++)
+    for (int j = 0; j < V; j++) {
+      float base;
+      if (hv->S0) {
+        base = hv->S0[(size_t)i * V + j];                        /* quantization switched off */
+      } else {
+        float s = hv->B[j] / 127.0f;
+        base = hv->c[i] * ((float)hv->Z[(size_t)i * V + j] * s);
+        for (int h = 0; h < r; h++)
+          base = fmaf(lqo_f16_to_f32(hv->ck[(size_t)h * K + i]), lqo_f16_to_f32(hv->cu[(size_t)h * V + j]), base);
+      }
+      float x = gam[i] * base;
+      for (int jj = 0; jj < n; jj++) x = fmaf(kd[(size_t)jj * K + i], hv->bu[(size_t)jj * V + j], x);
+      S[(size_t)i * V + j] = x;
+    }
+  free(gam); free(kd); free(dec);
+}
+
+/* ------------------------------------------------------------------ */
+/* Window-boundary quantization of a dense state M (destroyed):        */
+/*   r Compensator Tokens, Eqs. 5-6, each the leading singular pair of  */
+/*   what is left, found by power iteration and removed with the values */
+/*   that are actually stored (fp16);                                   */
+/*   smoothing scales c, Sec. 3.4 (square root of the row mean |.|);    */
+/*   per-value-channel symmetric 8-bit codes, Appendix B.3.             */
+/* ------------------------------------------------------------------ */
+static void head_quantize(const lqo_shape *sh, float *M, const head_view *hv) {
+  int K = sh->d_k, V = sh->d_v;
+  float *w = (float *)malloc(sizeof(float) * V), *t = (float *)malloc(sizeof(float) * K);
+  float *col = (float *)malloc(sizeof(float) * K);
+  float *kf = (float *)malloc(sizeof(float) * K), *uf = (float *)malloc(sizeof(float) * V);
+
+  for (int h = 0; h < sh->r; h++) {
+    int vanished = 0;
+    for (int j = 0; j < V; j++) w[j] = 1.0f / sqrtf((float)V);
+    for (int it = 0; it < sh->n_iter; it++) {
+      for (int i = 0; i < K; i++) t[i] = lqo_csum_dot(M + (size_t)i * V, w, V);      /* t = M w      */
+      float nu = lqo_csum_dot(t, t, K);
+      if (nu < 1e-30f) { vanished = 1; break; }
+      float rinv = 1.0f / sqrtf(nu);
+      for (int i = 0; i < K; i++) t[i] = t[i] * rinv;                                   /* unit length  */
+      if (it + 1 < sh->n_iter)
+        for (int j = 0; j < V; j++) { column_of(M, K, V, j, col); w[j] = lqo_csum_dot(col, t, K); } /* w = M^T t */
+    }
+    for (int i = 0; i < K; i++) {
+      uint16_t bits = vanished ? 0 : lqo_f32_to_f16(clamp_f16_range(t[i]));
+      hv->ck[(size_t)h * K + i] = bits;
+      kf[i] = lqo_f16_to_f32(bits);
+    }
+    for (int j = 0; j < V; j++) {
+      uint16_t bits = 0;
+      if (!vanished) { column_of(M, K, V, j, col); bits = lqo_f32_to_f16(clamp_f16_range(lqo_csum_dot(col, kf, K))); }
+      hv->cu[(size_t)h * V + j] = bits;
+      uf[j] = lqo_f16_to_f32(bits);
+    }
+    for (int i = 0; i < K; i++)
+      for (int j = 0; j < V; j++) M[(size_t)i * V + j] = fmaf(-kf[i], uf[j], M[(size_t)i * V + j]);
+  }
+
+  /* M is now the residual R.  Smooth the key rows, then quantize each value channel. */
+  for (int i = 0; i < K; i++) {
+    float ci = 1.0f;
+    if (sh->smooth) {
+      float mean_abs = lqo_csum_abs(M + (size_t)i * V, V) / (float)V;
+      ci = fmaxf(sqrtf(mean_abs), 1e-6f);
+    }
+    hv->c[i] = ci;
+    float inv_c = 1.0f / ci;
+    for (int j = 0; j < V; j++) M[(size_t)i * V + j] = M[(size_t)i * V + j] * inv_c;
+  }
+  for (int j = 0; j < V; j++) {
+    float amax = 0.0f;
+    for (int i = 0; i < K; i++) amax = fmaxf(amax, fabsf(M[(size_t)i * V + j]));
+    hv->B[j] = amax;
+    float inv = amax > 0.0f ? 127.0f / amax : 0.0f;
+    for (int i = 0; i < K; i++) {
+      float z = rintf(M[(size_t)i * V + j] * inv);          /* ties to even */
+      z = fminf(fmaxf(z, -127.0f), 127.0f);
+      hv->Z[(size_t)i * V + j] = (int8_t)z;
+    }
+  }
+  free(w); free(t); free(col); free(kf); free(uf);
+}
+
+/* boundary: rebuild S_W from the window representation and start the next window from it */
+static void head_flush(const lqo_shape *sh, const head_view *hv, int n) {
+  int K = sh->d_k, V = sh->d_v;
+  float *S = (float *)malloc(sizeof(float) * (size_t)K * V);
+  head_reconstruct(sh, hv, n, S);
+  if (hv->S0) memcpy(hv->S0, S, sizeof(float) * (size_t)K * V);
+  else head_quantize(sh, S, hv);
+  free(S);
+}
+
+/* ------------------------------------------------------------------ */
+/* One decode token inside a window: the readout of Eq. 10 applied to   */
+/* x = alpha (.) k (for the correction u, Eq. 3) and to x = alpha (.) q */
+/* (for the output, using S_l^T q = S_{l-1}^T (alpha (.) q) + u (kt^T q)). */
+/* n records are already buffered; the new record goes to slot n.       */
+/* ------------------------------------------------------------------ */
+static void head_decode(const lqo_shape *sh, const head_view *hv, int n, const token_in *t, float *o) {
+  int K = sh->d_k, V = sh->d_v, r = sh->r;
+  float *kt = (float *)malloc(sizeof(float) * K), *g = (float *)malloc(sizeof(float) * K);
+  float *gk = (float *)malloc(sizeof(float) * K), *gq = (float *)malloc(sizeof(float) * K);
+  float *dec = (float *)malloc(sizeof(float) * K), *col = (float *)malloc(sizeof(float) * K);
+  float *pk = (float *)malloc(sizeof(float) * (n + r + 1)), *pq = (float *)malloc(sizeof(float) * (n + r + 1));
+  float *ck = (float *)malloc(sizeof(float) * K);
+  float *u = (float *)malloc(sizeof(float) * V);
+
+  for (int i = 0; i < K; i++) { kt[i] = t->beta * t->k[i]; g[i] = t->a[i]; }
+
+  /* real records, newest first; g is the decay from just after record j through the current token */
+  for (int j = n - 1; j >= 0; j--) {
+    for (int i = 0; i < K; i++) { gk[i] = g[i] * t->k[i]; gq[i] = g[i] * t->q[i]; }
+    pk[j] = lqo_csum_dot(hv->bk + (size_t)j * K, gk, K);
+    pq[j] = lqo_csum_dot(hv->bk + (size_t)j * K, gq, K);
+    record_decay(sh, hv, j, dec);
+    for (int i = 0; i < K; i++) g[i] = g[i] * dec[i];
+  }
+  /* g = Gamma_{1:l}: what the boundary state and its compensators have decayed by */
+  for (int i = 0; i < K; i++) { gk[i] = g[i] * t->k[i]; gq[i] = g[i] * t->q[i]; }
+
+  float *ptk = pk + n, *ptq = pq + n;      /* compensator projections */
+  if (!hv->S0)
+    for (int h = 0; h < r; h++) {
+      for (int i = 0; i < K; i++) ck[i] = lqo_f16_to_f32(hv->ck[(size_t)h * K + i]);
+      ptk[h] = lqo_csum_dot(ck, gk, K);
+      ptq[h] = lqo_csum_dot(ck, gq, K);
+    }
+
+  float ktq = lqo_csum_dot(kt, t->q, K);
+
+  /* boundary-state term: (B/127) Z^T (C Gamma x); with quantization off it is S0^T (Gamma x) */
+  float *xk = (float *)malloc(sizeof(float) * K), *xq = (float *)malloc(sizeof(float) * K);
+  for (int i = 0; i < K; i++) {
+    float ci = hv->S0 ? 1.0f : hv->c[i];
+    xk[i] = hv->S0 ? gk[i] : ci * gk[i];
+    xq[i] = hv->S0 ? gq[i] : ci * gq[i];
+  }
+  for (int j = 0; j < V; j++) {
+    float rk, rq;
+    if (hv->S0) {
+      column_of(hv->S0, K, V, j, col);
+      rk = lqo_csum_dot(col, xk, K);
+      rq = lqo_csum_dot(col, xq, K);
+    } else {
+      for (int i = 0; i < K; i++) col[i] = (float)hv->Z[(size_t)i * V + j];
+      float s = hv->B[j] / 127.0f;
+      rk = s * lqo_csum_dot(col, xk, K);
+      rq = s * lqo_csum_dot(col, xq, K);
+      for (int h = 0; h < r; h++) {
+        float uc = lqo_f16_to_f32(hv->cu[(size_t)h * V + j]);
+        rk = fmaf(uc, ptk[h], rk);
+        rq = fmaf(uc, ptq[h], rq);
+      }
+    }
+    for (int jj = 0; jj < n; jj++) {
+      rk = fmaf(hv->bu[(size_t)jj * V + j], pk[jj], rk);
+      rq = fmaf(hv->bu[(size_t)jj * V + j], pq[jj], rq);
+    }
+    u[j] = t->v[j] - rk;                 /* Eq. 3: u = v - S_{l-1}^T (alpha (.) k) */
+    o[j] = fmaf(u[j], ktq, rq);          /* o = S_{l-1}^T (alpha (.) q) + u (kt^T q) */
+  }
+
+  /* append the record (alpha, kt, u) */
+  if (sh->gate == LQO_GATE_DIAG) memcpy(hv->ba + (size_t)n * K, t->a, sizeof(float) * K);
+  else hv->ba[n] = t->a[0];
+  memcpy(hv->bk + (size_t)n * K, kt, sizeof(float) * K);
+  memcpy(hv->bu + (size_t)n * V, u, sizeof(float) * V);
+
+  free(kt); free(g); free(gk); free(gq); free(dec); free(col); free(pk); free(pq); free(ck); free(u);
+  free(xk); free(xq);
+}
+
+/* ------------------------------------------------------------------ */
+/* batch drivers (exported)                                            */
+/* ------------------------------------------------------------------ */
+
+static int shape_ok(const lqo_shape *sh) {
+  return sh && sh->batch >= 0 && sh->heads_v > 0 && sh->heads_qk > 0 && sh->heads_v % sh->heads_qk == 0 &&
+         sh->d_k > 0 && sh->d_v > 0 && sh->W > 0 && sh->r >= 0 && sh->n_iter >= 1 &&
+         (sh->gate == LQO_GATE_SCALAR || sh->gate == LQO_GATE_DIAG);
+}
+
+int lqo_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+/* Eq. 1 on a dense fp32 state (the unquantized trajectory). */
+int lqo_ref_step_f32(const lqo_shape *sh, float *S, const uint16_t *q, const uint16_t *k, const uint16_t *v,
+                     const uint16_t *beta, const uint16_t *alpha, float *o) {
+  if (!shape_ok(sh)) return 1;
+  long nh = (long)sh->batch * sh->heads_v;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (long bh = 0; bh < nh; bh++) {
+    int b = (int)(bh / sh->heads_v), h = (int)(bh % sh->heads_v);
+    token_in t = token_alloc(sh);
+    token_load(sh, b, h, q, k, v, beta, alpha, &t);
+    head_ref_step(sh, S + (size_t)bh * sh->d_k * sh->d_v, &t, o + (size_t)bh * sh->d_v);
+    token_free(&t);
+  }
+  return 0;
+}
+
+/* Eq. 2 with bf16 as the storage format: the state is rounded to bf16 after every token;
+ * the output is read from the updated state before it is rounded. */
+int lqo_ref_step_bf16(const lqo_shape *sh, uint16_t *S16, const uint16_t *q, const uint16_t *k, const uint16_t *v,
+                      const uint16_t *beta, const uint16_t *alpha, float *o) {
+  if (!shape_ok(sh)) return 1;
+  long nh = (long)sh->batch * sh->heads_v;
+  size_t KV = (size_t)sh->d_k * sh->d_v;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (long bh = 0; bh < nh; bh++) {
+    int b = (int)(bh / sh->heads_v), h = (int)(bh % sh->heads_v);
+    token_in t = token_alloc(sh);
+    token_load(sh, b, h, q, k, v, beta, alpha, &t);
+    float *S = (float *)malloc(sizeof(float) * KV);
+    for (size_t e = 0; e < KV; e++) S[e] = bf16_to_f32(S16[(size_t)bh * KV + e]);
+    head_ref_step(sh, S, &t, o + (size_t)bh * sh->d_v);
+    for (size_t e = 0; e < KV; e++) S16[(size_t)bh * KV + e] = lqo_f32_to_bf16(S[e]);
+    free(S);
+    token_free(&t);
+  }
+  return 0;
+}
+
+/* dense fp32 state -> window representation with an empty window */
+int lqo_quantize_state(const lqo_shape *sh, const float *S, lqo_state *st) {
+  if (!shape_ok(sh)) return 1;
+  long nh = (long)sh->batch * sh->heads_v;
+  size_t KV = (size_t)sh->d_k * sh->d_v;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (long bh = 0; bh < nh; bh++) {
+    head_view hv = view_of(sh, st, (int)(bh / sh->heads_v), (int)(bh % sh->heads_v));
+    if (hv.S0) { memcpy(hv.S0, S + (size_t)bh * KV, sizeof(float) * KV); continue; }
+    float *M = (float *)malloc(sizeof(float) * KV);
+    memcpy(M, S + (size_t)bh * KV, sizeof(float) * KV);
+    head_quantize(sh, M, &hv);
+    free(M);
+  }
+  for (int b = 0; b < sh->batch; b++) st->win_pos[b] = 0;
+  return 0;
+}
+
+/* window representation -> the dense state it stands for right now (all buffered records applied) */
+int lqo_dequantize_state(const lqo_shape *sh, const lqo_state *st, float *S) {
+  if (!shape_ok(sh)) return 1;
+  long nh = (long)sh->batch * sh->heads_v;
+  size_t KV = (size_t)sh->d_k * sh->d_v;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (long bh = 0; bh < nh; bh++) {
+    int b = (int)(bh / sh->heads_v);
+    head_view hv = view_of(sh, st, b, (int)(bh % sh->heads_v));
+    head_reconstruct(sh, &hv, st->win_pos[b], S + (size_t)bh * KV);
+  }
+  return 0;
+}
+
+/* Flush sequences whose window is full (force == 0) or that hold any record (force != 0). */
+int lqo_window_flush(const lqo_shape *sh, lqo_state *st, int force) {
+  if (!shape_ok(sh)) return 1;
+  long nh = (long)sh->batch * sh->heads_v;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (long bh = 0; bh < nh; bh++) {
+    int b = (int)(bh / sh->heads_v);
+    int n = st->win_pos[b];
+    if (n == sh->W || (force && n > 0)) {
+      head_view hv = view_of(sh, st, b, (int)(bh % sh->heads_v));
+      head_flush(sh, &hv, n);
+    }
+  }
+  for (int b = 0; b < sh->batch; b++) {
+    int n = st->win_pos[b];
+    if (n == sh->W || (force && n > 0)) st->win_pos[b] = 0;
+  }
+  return 0;
+}
+
+/* One decode token for every (sequence, value head); a window that becomes full is flushed at once
+ * (Eq. 4: the state is materialised and quantized only at l = p). */
+int lqo_decode_step(const lqo_shape *sh, lqo_state *st, const uint16_t *q, const uint16_t *k, const uint16_t *v,
+                    const uint16_t *beta, const uint16_t *alpha, float *o) {
+  if (!shape_ok(sh)) return 1;
+  for (int b = 0; b < sh->batch; b++)
+    if (st->win_pos[b] < 0 || st->win_pos[b] >= sh->W) return 2;
+  long nh = (long)sh->batch * sh->heads_v;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (long bh = 0; bh < nh; bh++) {
+    int b = (int)(bh / sh->heads_v), h = (int)(bh % sh->heads_v);
+    head_view hv = view_of(sh, st, b, h);
+    token_in t = token_alloc(sh);
+    token_load(sh, b, h, q, k, v, beta, alpha, &t);
+    head_decode(sh, &hv, st->win_pos[b], &t, o + (size_t)bh * sh->d_v);
+    token_free(&t);
+  }
+  for (int b = 0; b < sh->batch; b++) st->win_pos[b] += 1;
+  return lqo_window_flush(sh, st, 0);
+}

@@ -1,0 +1,104 @@
+"""Chain-level pins of the oracle: the window of one token is naive per-token requantization (Eq. 2), a forced
+flush keeps the state, the window position cycles, and the error ordering the paper reports (LeapQuant below
+per-window INT8 below per-step INT8) shows on a synthetic chain."""
+import numpy as np
+import pytest
+
+from oracle.lq_oracle import Shape, State
+from paper_2609_38166_b200 import synth
+from tests import refmath as rm
+
+
+def _shape(wl):
+    return Shape(wl.batch, wl.heads_v, wl.heads_qk, wl.d_k, wl.d_v, wl.W, wl.r, wl.n_iter, wl.gate, wl.smooth)
+
+
+def _naive_quant64(S):
+    """per-value-channel symmetric INT8 with residual smoothing and no compensators, in float64"""
+    c = np.maximum(np.sqrt(np.abs(S).mean(axis=1)), 1e-6)
+    X = S / c[:, None]
+    B = np.abs(X).max(axis=0)
+    Z = np.rint(X * np.where(B > 0, 127.0 / np.where(B > 0, B, 1), 0.0))
+    return Z, B, c
+
+
+@pytest.mark.parametrize("gate", [synth.GATE_SCALAR, synth.GATE_DIAG])
+def test_window_of_one_is_per_token_requantization(oracle, gate):
+    # Eq. 2 written on its own: dequantize, apply the model's update, quantize; every token
+    wl = synth.Workload("t", 1, 2, 2, 32, 32, W=1, r=0, gate=gate, seed=31)
+    sh = _shape(wl)
+    st = State(sh)
+    oracle.quantize_state(sh, np.zeros((1, 2, 32, 32), np.float32), st)
+    Z = np.zeros((2, 32, 32)); B = np.zeros((2, 32)); c = np.ones((2, 32))
+    off_by_one = total = 0
+    for step in range(30):
+        tok = synth.token_inputs(wl, step)
+        o = oracle.decode_step(sh, st, **tok)
+        assert st.win_pos[0] == 0
+        for h in range(2):
+            # restart the float64 chain from the oracle's stored state so that the comparison is per token
+            S_hat = c[h][:, None] * (Z[h] / 127.0) * B[h][None, :]
+            Sn, o64 = rm.native_step(S_hat, *rm.widen(tok, wl, 0, h), gate)
+            assert np.allclose(o[0, h], o64, rtol=1e-5, atol=1e-5)
+            Zn, Bn, cn = _naive_quant64(Sn)
+            d = np.abs(st.codes[0, h].astype(np.float64) - Zn)
+            assert d.max() <= 1
+            off_by_one += int((d > 0).sum()); total += d.size
+            assert np.allclose(st.col_scale[0, h], Bn, rtol=1e-5) and np.allclose(st.row_smooth[0, h], cn, rtol=1e-5)
+            Z[h], B[h], c[h] = st.codes[0, h], st.col_scale[0, h], st.row_smooth[0, h]
+    assert off_by_one <= 2e-3 * total     # only values within fp32 rounding of a tie may differ
+
+
+def test_forced_flush_keeps_the_state_and_empties_the_window(oracle):
+    wl = synth.Workload("t", 3, 2, 1, 64, 64, W=8, r=2, seed=32)
+    sh = _shape(wl)
+    st = State(sh)
+    oracle.quantize_state(sh, synth.dense_states(wl, 5), st)
+    for step in range(5):
+        oracle.decode_step(sh, st, **synth.token_inputs(wl, step))
+    assert np.all(st.win_pos == 5)
+    before = oracle.dequantize_state(sh, st)
+    oracle.window_flush(sh, st, force=False)          # nothing is full: no change
+    assert np.all(st.win_pos == 5) and np.array_equal(oracle.dequantize_state(sh, st), before)
+    oracle.window_flush(sh, st, force=True)
+    assert np.all(st.win_pos == 0)
+    after = oracle.dequantize_state(sh, st).astype(np.float64)
+    bound = st.row_smooth[..., None].astype(np.float64) * st.col_scale[:, :, None, :] / 254.0
+    assert np.all(np.abs(after - before) <= bound * (1 + 1e-4) + 1e-7)
+
+
+def test_staggered_sequences_flush_independently(oracle):
+    wl = synth.Workload("t", 4, 1, 1, 32, 32, W=4, r=1, seed=33)
+    sh = _shape(wl)
+    st = State(sh)
+    oracle.quantize_state(sh, synth.dense_states(wl, 6), st)
+    st.win_pos[:] = [0, 1, 2, 3]      # as if the sequences had started at different times
+    st.buf_a[...] = 1.0
+    codes0 = st.codes.copy()
+    oracle.decode_step(sh, st, **synth.token_inputs(wl, 0))
+    assert list(st.win_pos) == [1, 2, 3, 0]
+    assert np.array_equal(st.codes[:3], codes0[:3]) and not np.array_equal(st.codes[3], codes0[3])
+
+
+def test_error_ordering_on_a_chain(oracle):
+    """State error against the unquantized trajectory after a few hundred tokens: the full method is below
+    per-window INT8, which is below per-step INT8 (Sec. 3.2 and the component ablation)."""
+    base = synth.Workload("t", 4, 4, 4, 128, 128, W=16, r=4, seed=34, outlier_frac=0.02, outlier_mag=8.0)
+    variants = {"full": base, "window": base.with_(r=0, smooth=0), "step": base.with_(W=1, r=0, smooth=0)}
+    shf = _shape(base)
+    Sref = np.zeros((4, 4, 128, 128), np.float32)
+    states = {}
+    for name, wl in variants.items():
+        states[name] = State(_shape(wl))
+        oracle.quantize_state(_shape(wl), Sref, states[name])
+    err = {name: [] for name in variants}
+    for step in range(161):
+        tok = synth.token_inputs(base, step)
+        oref = oracle.ref_step_f32(shf, Sref, **tok)
+        for name, wl in variants.items():
+            o = oracle.decode_step(_shape(wl), states[name], **tok)
+            if step >= 32:
+                err[name].append(np.linalg.norm(o - oref) / np.linalg.norm(oref))
+    m = {k: float(np.mean(v)) for k, v in err.items()}
+    assert m["full"] < m["window"] < m["step"], m
+    assert m["full"] < 2e-3, m

@@ -1,0 +1,174 @@
+"""Pins for the oracle's recurrences: the dense reference step, the windowed decode step and the
+reconstruction, against the models' native updates written densely in float64, against closed-form
+special cases, and against brute force on tiny states."""
+import numpy as np
+import pytest
+
+from oracle.lq_oracle import Shape, State
+from paper_2609_38166_b200 import synth
+from tests import refmath as rm
+
+GATES = [synth.GATE_SCALAR, synth.GATE_DIAG]
+
+
+def _shape(wl):
+    return Shape(wl.batch, wl.heads_v, wl.heads_qk, wl.d_k, wl.d_v, wl.W, wl.r, wl.n_iter, wl.gate, wl.smooth)
+
+
+def _rel(a, b):
+    return float(np.linalg.norm(np.asarray(a, np.float64) - b) / (np.linalg.norm(b) + 1e-30))
+
+
+@pytest.mark.parametrize("gate", GATES)
+def test_native_update_equals_general_form(gate):
+    # the identity of Appendix A that lets GDN and KDA use Eq. 1; pure float64 mathematics
+    wl = synth.Workload("t", 1, 1, 1, 32, 24, gate=gate, seed=11)
+    S = np.random.default_rng(0).standard_normal((32, 24))
+    for step in range(5):
+        q, k, v, beta, alpha = rm.widen(synth.token_inputs(wl, step), wl)
+        S1, o1 = rm.native_step(S, q, k, v, beta, alpha, gate)
+        S2, o2 = rm.general_step(S, q, k, v, beta, alpha, gate)
+        assert np.allclose(S1, S2, rtol=0, atol=1e-12) and np.allclose(o1, o2, rtol=0, atol=1e-12)
+        S = S1
+
+
+@pytest.mark.parametrize("gate", GATES)
+def test_reference_step_follows_native_update(oracle, gate):
+    wl = synth.Workload("t", 2, 4, 2, 128, 128, gate=gate, seed=12)
+    sh = _shape(wl)
+    S = np.zeros((2, 4, 128, 128), np.float32)
+    S64 = np.zeros((2, 4, 128, 128))
+    for step in range(40):
+        tok = synth.token_inputs(wl, step)
+        o = oracle.ref_step_f32(sh, S, **tok)
+        for b in range(2):
+            for h in range(4):
+                S64[b, h], o64 = rm.native_step(S64[b, h], *rm.widen(tok, wl, b, h), gate)
+                assert np.allclose(o[b, h], o64, rtol=1e-5, atol=1e-5)
+    assert _rel(S, S64) < 1e-6
+
+
+def test_delta_rule_write_is_exact_recall(oracle):
+    # alpha = beta = 1 and |k| = 1: the update stores v under k, so reading with q = k returns v.
+    # Keys are +-1/8 on 64 channels, exactly representable and of unit length.
+    K = V = 64
+    sh = Shape(1, 1, 1, K, V, 4, 0, 1, synth.GATE_SCALAR, 1)
+    rng = np.random.default_rng(5)
+    S = rng.standard_normal((1, 1, K, V)).astype(np.float32)
+    one = synth.f32_to_bf16_bits(np.ones((1, 1), np.float32))
+    for _ in range(6):
+        k = (rng.integers(0, 2, (1, 1, K)) * 2 - 1).astype(np.float32) / 8.0
+        v = synth.f32_to_bf16_bits(rng.standard_normal((1, 1, V)).astype(np.float32))
+        kb = synth.f32_to_bf16_bits(k)
+        o = oracle.ref_step_f32(sh, S, kb, kb, v, one, one)
+        assert np.allclose(o, synth.bf16_bits_to_f32(v), rtol=0, atol=2e-5)
+
+
+@pytest.mark.parametrize("gate", GATES)
+@pytest.mark.parametrize("W", [1, 3, 16])
+def test_windowed_decode_without_quantizer_equals_dense_recurrence(oracle, gate, W):
+    # Eq. 4 / Eq. 9: with quant_b the identity the windowed form is the recurrence itself
+    wl = synth.Workload("t", 2, 2, 1, 128, 128, W=W, r=0, gate=gate, seed=13)
+    sh = _shape(wl)
+    st = State(sh, quant=False)
+    S64 = np.zeros((2, 2, 128, 128))
+    for step in range(2 * W + 5):
+        tok = synth.token_inputs(wl, step)
+        o = oracle.decode_step(sh, st, **tok)
+        for b in range(2):
+            for h in range(2):
+                S64[b, h], o64 = rm.native_step(S64[b, h], *rm.widen(tok, wl, b, h), gate)
+                assert np.allclose(o[b, h], o64, rtol=1e-5, atol=1e-5), (step, b, h)
+        assert np.all(st.win_pos == (step + 1) % W)
+        assert _rel(oracle.dequantize_state(sh, st), S64) < 1e-6
+
+
+@pytest.mark.parametrize("gate", GATES)
+def test_recall_special_case_holds_with_quantization_on(oracle, gate):
+    # With alpha = beta = 1, |k| = 1 and q = k the windowed output is v whatever the quantized state holds,
+    # because the same readout enters u and o and cancels.
+    K = V = 64
+    wl = synth.Workload("t", 1, 2, 2, K, V, W=4, r=2, gate=gate, seed=14)
+    sh = _shape(wl)
+    st = State(sh)
+    oracle.quantize_state(sh, synth.dense_states(wl, 1), st)
+    rng = np.random.default_rng(6)
+    one = synth.f32_to_bf16_bits(np.ones((1, 2), np.float32))
+    ones_a = one if gate == synth.GATE_SCALAR else synth.f32_to_bf16_bits(np.ones((1, 2, K), np.float32))
+    for _ in range(9):
+        kb = synth.f32_to_bf16_bits((rng.integers(0, 2, (1, 2, K)) * 2 - 1).astype(np.float32) / 8.0)
+        v = synth.f32_to_bf16_bits(rng.standard_normal((1, 2, V)).astype(np.float32))
+        o = oracle.decode_step(sh, st, kb, kb, v, one, ones_a)
+        assert np.allclose(o, synth.bf16_bits_to_f32(v), rtol=0, atol=1e-5)
+
+
+@pytest.mark.parametrize("gate", GATES)
+@pytest.mark.parametrize("dims", [(4, 4, 3, 1), (4, 4, 2, 2), (8, 16, 3, 2), (5, 3, 4, 1)])
+def test_brute_force_on_tiny_states(oracle, gate, dims):
+    """Materialise the state densely before every token (Eq. 7 written out in float64 from the stored arrays),
+    apply the native update, and compare the token's output and the record it appends."""
+    K, V, W, r = dims
+    wl = synth.Workload("t", 2, 2, 2, K, V, W=W, r=r, gate=gate, seed=15)
+    sh = _shape(wl)
+    st = State(sh)
+    oracle.quantize_state(sh, synth.dense_states(wl, 2, rank=2), st)
+    for step in range(3 * W + 1):
+        tok = synth.token_inputs(wl, step)
+        dense = np.zeros((2, 2, K, V))
+        for b in range(2):
+            n = int(st.win_pos[b])
+            for h in range(2):
+                S = rm.dequant_plain(st.codes[b, h], st.col_scale[b, h], st.row_smooth[b, h], st.comp_k[b, h],
+                                     st.comp_u[b, h])
+                for j in range(n):     # apply the buffered records in order (Eq. 3)
+                    a = st.buf_a[b, h, j].astype(np.float64)
+                    a = np.full(K, float(a)) if gate == synth.GATE_SCALAR else a
+                    S = a[:, None] * S + np.outer(st.buf_k[b, h, j].astype(np.float64),
+                                                  st.buf_u[b, h, j].astype(np.float64))
+                dense[b, h] = S
+        assert np.allclose(oracle.dequantize_state(sh, st), dense, rtol=1e-5, atol=1e-6)
+        n_before = st.win_pos.copy()
+        o = oracle.decode_step(sh, st, **tok)
+        for b in range(2):
+            for h in range(2):
+                q, k, v, beta, alpha = rm.widen(tok, wl, b, h)
+                Sn, o64 = rm.native_step(dense[b, h], q, k, v, beta, alpha, gate)
+                assert np.allclose(o[b, h], o64, rtol=1e-5, atol=1e-5), (step, b, h)
+                if n_before[b] + 1 < W:   # the record is still in the buffer: u = v - S^T (alpha (.) k)
+                    a = np.full(K, float(alpha)) if gate == synth.GATE_SCALAR else alpha
+                    u64 = v - dense[b, h].T @ (a * k)
+                    assert np.allclose(st.buf_u[b, h, n_before[b]], u64, rtol=1e-5, atol=1e-5)
+                    assert np.allclose(st.buf_k[b, h, n_before[b]], beta * k, rtol=1e-6, atol=0)
+        assert np.all(st.win_pos == (n_before + 1) % W)
+
+
+def test_grouped_heads_read_the_right_query_head(oracle):
+    # value head h uses q/k head h // (Hv/Hqk): make q/k heads wildly different and compare per head
+    wl = synth.Workload("t", 1, 4, 2, 16, 8, W=4, r=1, seed=16)
+    sh = _shape(wl)
+    S = np.zeros((1, 4, 16, 8), np.float32)
+    S64 = np.zeros((4, 16, 8))
+    for step in range(6):
+        tok = synth.token_inputs(wl, step)
+        o = oracle.ref_step_f32(sh, S, **tok)
+        for h in range(4):
+            S64[h], o64 = rm.native_step(S64[h], *rm.widen(tok, wl, 0, h), wl.gate)
+            assert np.allclose(o[0, h], o64, rtol=1e-5, atol=1e-6)
+
+
+def test_bf16_state_baseline_rounds_state_each_token(oracle):
+    wl = synth.Workload("t", 1, 2, 2, 32, 32, seed=17)
+    sh = _shape(wl)
+    S16 = np.zeros((1, 2, 32, 32), np.uint16)
+    S64 = np.zeros((2, 32, 32))
+    for step in range(10):
+        tok = synth.token_inputs(wl, step)
+        o = oracle.ref_step_bf16(sh, S16, **tok)
+        for h in range(2):
+            Sn, o64 = rm.native_step(S64[h], *rm.widen(tok, wl, 0, h), wl.gate)
+            assert np.allclose(o[0, h], o64, rtol=1e-5, atol=1e-6)
+            S64[h] = synth.bf16_bits_to_f32(synth.f32_to_bf16_bits(Sn.astype(np.float32))).astype(np.float64)
+            got = synth.bf16_bits_to_f32(S16[0, h]).astype(np.float64)
+            # equal up to an occasional one-ulp difference where the fp32 and fp64 values straddle a tie
+            assert np.mean(got != S64[h]) < 0.01 and np.allclose(got, S64[h], rtol=2.0 ** -7, atol=1e-8)
+            S64[h] = got
