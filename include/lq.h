@@ -1,0 +1,160 @@
+/*
+ * lq.h - C boundary of the B200 (sm_100a) per-window 8-bit decode step for
+ * Gated DeltaNet (scalar gate) and Kimi Delta Attention (per-channel gate)
+ * recurrent states.
+ *
+ * One value head owns a state S in R^{d_k x d_v} (Sec. 3.1, Eq. 1; row index =
+ * key channel, column index = value channel, readout o = S^T q).  Between
+ * window boundaries the state is held as
+ *     S_l = Gamma_{1:l} [ C (Z/127) B + Kc Uc^T ] + sum_j Gamma_{j+1:l} kt_j u_j^T      (Eq. 7)
+ * with Z the 8-bit codes, B the per-value-channel scale, C = Diag(c) the
+ * per-key-row smoothing scale (Sec. 3.4), (Kc, Uc) the r fp16 Compensator
+ * Tokens (Sec. 3.3) and (alpha_j, kt_j, u_j) the buffered records of the
+ * tokens decoded since the boundary (Sec. 3.2, Eq. 3).
+ *
+ * Conventions for every entry point
+ *  - All pointers are DEVICE pointers owned by the caller unless a parameter
+ *    is documented as a host pointer.  Arrays are dense, row-major, in the
+ *    layouts given below, and must be 16-byte aligned.
+ *  - The library allocates no device memory and never synchronises: work is
+ *    enqueued on `stream` and the call returns.  The lq_shape and lq_state
+ *    structs themselves are read on the host during the call only.
+ *  - bf16 and fp16 values travel as their 16-bit patterns (uint16_t).
+ *  - Errors are reported through the return value; nothing aborts or throws.
+ *    Argument errors are detected before anything is enqueued.
+ *  - Arithmetic is IEEE binary32.  Sums over a channel index are taken in a
+ *    fixed order (blocks of eight consecutive terms accumulated left to right
+ *    with fused multiply-add, block results combined as a balanced binary
+ *    tree over the block index), so results do not depend on the launch
+ *    configuration and are reproducible bit for bit.
+ *  - Supported shapes: d_k = d_v = 128, 1 <= W <= 64, 0 <= r <= 16,
+ *    n_iter >= 1, heads_v a multiple of heads_qk.  Anything else returns
+ *    LQ_ERR_UNSUPPORTED.
+ */
+#ifndef LQ_H_
+#define LQ_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  LQ_OK = 0,
+  LQ_ERR_NULL = 1,        /* a required pointer is null                         */
+  LQ_ERR_SHAPE = 2,       /* a dimension is non-positive or inconsistent        */
+  LQ_ERR_ALIGN = 3,       /* a pointer is not 16-byte aligned                   */
+  LQ_ERR_UNSUPPORTED = 4, /* valid request outside the supported shapes         */
+  LQ_ERR_CUDA = 5         /* the CUDA runtime reported an error on launch/copy  */
+} lq_status;
+
+typedef enum {
+  LQ_GATE_SCALAR = 0, /* GDN: D_t = alpha_t I;       alpha is [B,Hv]       */
+  LQ_GATE_DIAG = 1    /* KDA: D_t = Diag(alpha_t);   alpha is [B,Hv,d_k]   */
+} lq_gate;
+
+/* CUDA stream handle (a cudaStream_t); null is the default stream. */
+typedef struct CUstream_st *lq_stream;
+
+typedef struct {
+  int batch;    /* B: sequences                                                   */
+  int heads_v;  /* Hv: value heads per sequence, one state each                   */
+  int heads_qk; /* Hqk: query/key heads; value head h reads q/k head h/(Hv/Hqk)   */
+  int d_k, d_v; /* state is d_k x d_v                                             */
+  int W;        /* window length (the paper's p)                                  */
+  int r;        /* Compensator Tokens per state                                   */
+  int n_iter;   /* power-iteration steps per Compensator Token at a boundary      */
+  int gate;     /* lq_gate                                                        */
+  int smooth;   /* 1: residual smoothing (Sec. 3.4); 0: c = 1 (ablation)          */
+} lq_shape;
+
+/* Window representation of B x Hv states.  h is the value head. */
+typedef struct {
+  int8_t *codes;      /* [B,Hv,d_k,d_v]  Z, symmetric, in [-127,127]                        */
+  float *col_scale;   /* [B,Hv,d_v]      B: dequant(Z) = (Z/127) B  (Appendix B.3)           */
+  float *row_smooth;  /* [B,Hv,d_k]      c > 0 (Sec. 3.4)                                    */
+  uint16_t *comp_k;   /* [B,Hv,r,d_k]    fp16, unit-length key side of the compensators     */
+  uint16_t *comp_u;   /* [B,Hv,r,d_v]    fp16, value side (carries the magnitude)           */
+  float *buf_k;       /* [B,Hv,W,d_k]    write keys kt = beta*k of the buffered records     */
+  float *buf_u;       /* [B,Hv,W,d_v]    corrections u = v - S^T(alpha.k)  (Eq. 3)          */
+  float *buf_a;       /* [B,Hv,W] (scalar gate) or [B,Hv,W,d_k] (diagonal gate): decays     */
+  int32_t *win_pos;   /* [B]             records buffered per sequence, 0..W-1 between calls.
+                                         Bits 16 and up are used as a scratch counter while a
+                                         call runs and are zero again when it has finished.   */
+} lq_state;
+
+/*
+ * One decode token for every (sequence, value head): Eq. 10 (the readout of the smoothed, compensated
+ * window representation) applied to alpha.k gives the correction u of Eq. 3, applied to alpha.q gives
+ * the output through S_l^T q = S_{l-1}^T (alpha.q) + u (kt^T q); the record (alpha, kt, u) is appended
+ * to the buffer and win_pos advances.  A sequence whose window becomes full (win_pos reaches W) is
+ * taken through the boundary in the same call, as Eq. 4 prescribes: see lq_window_flush.
+ *   q, k  : bf16 [B,Hqk,d_k]     v : bf16 [B,Hv,d_v]     beta : bf16 [B,Hv]
+ *   alpha : bf16 [B,Hv] or [B,Hv,d_k], the decay multiplier itself (not its logarithm)
+ *   o     : fp32 [B,Hv,d_v], written
+ * A sequence that enters with win_pos >= W (possible only if the caller set it) gets no token: its `o`
+ * rows are not written and nothing is appended; with win_pos == W it is taken through the boundary by
+ * this call like by lq_window_flush.
+ * Calls on the same state must be ordered by the stream.
+ */
+lq_status lq_decode_step(const lq_shape *shape, const lq_state *state, const uint16_t *q, const uint16_t *k,
+                         const uint16_t *v, const uint16_t *beta, const uint16_t *alpha, float *o, lq_stream stream);
+
+/*
+ * Same as lq_decode_step, but the token's inputs and the output live in HOST memory (pinned memory makes
+ * the copies asynchronous): q_h, k_h, v_h, beta_h, alpha_h are copied into the device staging buffer
+ * `stage` on `stream`, the step runs, and `o` is copied to o_h.  `stage` is a device buffer of at least
+ * lq_decode_stage_bytes(shape) bytes, 16-byte aligned, owned by the caller.  The host arrays must stay
+ * valid until the stream has passed the call.
+ */
+lq_status lq_decode_step_host(const lq_shape *shape, const lq_state *state, const uint16_t *q_h,
+                              const uint16_t *k_h, const uint16_t *v_h, const uint16_t *beta_h,
+                              const uint16_t *alpha_h, float *o_h, void *stage, lq_stream stream);
+/* Bytes of device staging lq_decode_step_host needs for `shape` (0 if the shape is invalid). */
+uint64_t lq_decode_stage_bytes(const lq_shape *shape);
+
+/*
+ * Window boundary (Secs. 3.2-3.4): for every sequence with win_pos == W, or, when force != 0, with
+ * win_pos > 0, rebuild the dense state from the window representation (Eq. 7), refit the r Compensator
+ * Tokens by power iteration and remove them (Eqs. 5-6), recompute the smoothing scales from the
+ * residual, requantize it to 8 bits, and set win_pos = 0.  Other sequences are not touched.
+ */
+lq_status lq_window_flush(const lq_shape *shape, const lq_state *state, int force, lq_stream stream);
+
+/*
+ * Start a window from dense states: S fp32 [B,Hv,d_k,d_v] (read only) is split into compensators,
+ * smoothing scales and 8-bit codes exactly as at a window boundary; win_pos is set to 0 for all B
+ * sequences.  The record buffers are not read or written.
+ */
+lq_status lq_quantize_state(const lq_shape *shape, const float *S, const lq_state *state, lq_stream stream);
+
+/*
+ * The dense state the window representation currently stands for, all buffered records applied (Eq. 7
+ * with l = win_pos): written to S fp32 [B,Hv,d_k,d_v].  The state is not modified.
+ */
+lq_status lq_dequantize_state(const lq_shape *shape, const lq_state *state, float *S, lq_stream stream);
+
+/*
+ * Speed and accuracy baselines: the same token on an unquantized dense state (Eq. 1 with the GDN / KDA
+ * coefficients of Table 4), read and written in full every token.  S is [B,Hv,d_k,d_v], fp32 or bf16
+ * (rounded to nearest even after every token, the "BF16 per-step" setting); o is computed from the
+ * updated state before it is rounded.  Only batch, heads_v, heads_qk, d_k, d_v and gate of `shape` are used.
+ */
+lq_status lq_ref_decode_step_f32(const lq_shape *shape, float *S, const uint16_t *q, const uint16_t *k,
+                                 const uint16_t *v, const uint16_t *beta, const uint16_t *alpha, float *o,
+                                 lq_stream stream);
+lq_status lq_ref_decode_step_bf16(const lq_shape *shape, uint16_t *S, const uint16_t *q, const uint16_t *k,
+                                  const uint16_t *v, const uint16_t *beta, const uint16_t *alpha, float *o,
+                                  lq_stream stream);
+
+/* Kernels one lq_decode_step call launches for `shape` (used to report launch counts). */
+int lq_decode_launches(const lq_shape *shape);
+
+const char *lq_status_string(lq_status status);
+int lq_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LQ_H_ */

@@ -1,0 +1,365 @@
+// C boundary of the library: argument checks, launch configuration, and the kernels that wrap the
+// device routines of lq_decode.cuh and lq_boundary.cuh.  Declarations and contracts: include/lq.h.
+#include <cstdio>
+
+#include "lq_boundary.cuh"
+#include "lq_decode.cuh"
+
+namespace lq {
+
+// ---------------------------------------------------------------------------------------------
+// Boundary kernels: a CTA of 256 threads walks over heads (grid-stride) and takes those that need work.
+// MODE 0: flush (window representation -> dense -> new window representation)
+// MODE 1: quantize dense fp32 states         MODE 2: dequantize to dense fp32 states
+// ---------------------------------------------------------------------------------------------
+template <int GATE, int MODE>
+__global__ void __launch_bounds__(256) boundary_kernel(const Params p) {
+  extern __shared__ float4 lq_smem4[];
+  const BoundarySmem sm(reinterpret_cast<float *>(lq_smem4), p.W, p.r, GATE == LQ_GATE_DIAG);
+  const Tile t;
+  const size_t nh = (size_t)p.batch * p.heads_v;
+  for (size_t bh = blockIdx.x; bh < nh; bh += gridDim.x) {
+    const int b = static_cast<int>(bh / p.heads_v);
+    int n = 0;
+    if (MODE != 1) {
+      n = p.win_pos[b] & 0xFFFF;
+      if (MODE == 0 && !(n == p.W || (p.force && n > 0))) continue;
+      if (n > p.W) n = p.W;
+    }
+    float M[8][8];
+    if (MODE == 1) {
+      const float *S = p.S + bh * (size_t)(D * D);
+#pragma unroll
+      for (int a = 0; a < 8; a++) load8(S + (8 * t.ty + a) * D + 8 * t.tx, M[a]);
+    } else {
+      __syncthreads();                       // the previous head's use of shared memory is over
+      reconstruct_tile<GATE>(p, sm, t, bh, n, M);
+    }
+    if (MODE == 2) {
+      float *S = p.S + bh * (size_t)(D * D);
+#pragma unroll
+      for (int a = 0; a < 8; a++) store8(S + (8 * t.ty + a) * D + 8 * t.tx, M[a]);
+      continue;
+    }
+    quantize_tile(p, sm, t, bh, M);
+    __syncthreads();
+    if (t.tid == 0) {
+      if (MODE == 0) arrive_and_set(p.win_pos, b, p.heads_v, 0);
+      else p.win_pos[b] = 0;                 // nobody reads win_pos in this mode
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Baseline: Eq. 1 on a dense state that is read and written in full every token.
+// ---------------------------------------------------------------------------------------------
+template <int GATE, bool BF16>
+__global__ void __launch_bounds__(256) ref_kernel(const Params p) {
+  __shared__ __align__(16) float kt_s[D], q_s[D], bv_s[D], a_s[D], part_s[8 * D];
+  const Tile t;
+  const size_t bh = blockIdx.x;
+  const int b = static_cast<int>(bh / p.heads_v), hv = static_cast<int>(bh % p.heads_v);
+  float M[8][8];
+  if (BF16) {
+    const uint16_t *S = p.S16 + bh * (size_t)(D * D);
+#pragma unroll
+    for (int a = 0; a < 8; a++) {
+      const uint4 w = *reinterpret_cast<const uint4 *>(S + (8 * t.ty + a) * D + 8 * t.tx);
+      const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+      for (int e = 0; e < 4; e++) {
+        M[a][2 * e] = __uint_as_float(ws[e] << 16);
+        M[a][2 * e + 1] = __uint_as_float(ws[e] & 0xFFFF0000u);
+      }
+    }
+  } else {
+    const float *S = p.S + bh * (size_t)(D * D);
+#pragma unroll
+    for (int a = 0; a < 8; a++) load8(S + (8 * t.ty + a) * D + 8 * t.tx, M[a]);
+  }
+  if (t.tid < D) {
+    const int group = p.heads_v / p.heads_qk;
+    const size_t qk_off = ((size_t)b * p.heads_qk + hv / group) * D;
+    const float k_i = bf16_bits(p.k[qk_off + t.tid]);
+    const float a_i = GATE == LQ_GATE_DIAG ? bf16_bits(p.alpha[bh * D + t.tid]) : bf16_bits(p.alpha[bh]);
+    kt_s[t.tid] = bf16_bits(p.beta[bh]) * k_i;
+    bv_s[t.tid] = a_i * k_i;
+    a_s[t.tid] = a_i;
+    q_s[t.tid] = bf16_bits(p.q[qk_off + t.tid]);
+  }
+  __syncthreads();
+  float x[8], pc[8], u[8], o[8], kt[8], ai[8];
+  load8(bv_s + 8 * t.ty, x);
+  col_blocks(M, x, pc);
+  col_tree(pc, part_s, t, u);                            // S^T (alpha.k)
+#pragma unroll
+  for (int c = 0; c < 8; c++) u[c] = bf16_bits(p.v[bh * D + 8 * t.tx + c]) - u[c];
+  load8(kt_s + 8 * t.ty, kt);
+  load8(a_s + 8 * t.ty, ai);
+#pragma unroll
+  for (int a = 0; a < 8; a++)
+#pragma unroll
+    for (int c = 0; c < 8; c++) M[a][c] = fmaf(kt[a], u[c], ai[a] * M[a][c]);
+  load8(q_s + 8 * t.ty, x);
+  col_blocks(M, x, pc);
+  __syncthreads();                                       // part_s is reused
+  col_tree(pc, part_s, t, o);
+  if (t.ty == 0) store8(p.o + bh * D + 8 * t.tx, o);
+  if (BF16) {
+    uint16_t *S = p.S16 + bh * (size_t)(D * D);
+#pragma unroll
+    for (int a = 0; a < 8; a++) {
+      uint32_t ws[4];
+#pragma unroll
+      for (int e = 0; e < 4; e++)
+        ws[e] = (uint32_t)to_bf16_bits(M[a][2 * e]) | ((uint32_t)to_bf16_bits(M[a][2 * e + 1]) << 16);
+      *reinterpret_cast<uint4 *>(S + (8 * t.ty + a) * D + 8 * t.tx) = make_uint4(ws[0], ws[1], ws[2], ws[3]);
+    }
+  } else {
+    float *S = p.S + bh * (size_t)(D * D);
+#pragma unroll
+    for (int a = 0; a < 8; a++) store8(S + (8 * t.ty + a) * D + 8 * t.tx, M[a]);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------------
+static bool aligned16(const void *ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15u) == 0; }
+
+static lq_status check_shape(const lq_shape *s) {
+  if (!s) return LQ_ERR_NULL;
+  if (s->batch < 0 || s->heads_v <= 0 || s->heads_qk <= 0 || s->d_k <= 0 || s->d_v <= 0 || s->W <= 0 || s->r < 0 ||
+      s->n_iter < 1 || s->heads_v % s->heads_qk != 0 || (s->gate != LQ_GATE_SCALAR && s->gate != LQ_GATE_DIAG))
+    return LQ_ERR_SHAPE;
+  if (s->d_k != D || s->d_v != D || s->W > MAX_W || s->r > MAX_R) return LQ_ERR_UNSUPPORTED;
+  return LQ_OK;
+}
+
+static lq_status check_ptrs(std::initializer_list<const void *> ptrs) {
+  for (const void *q : ptrs)
+    if (!q) return LQ_ERR_NULL;
+  for (const void *q : ptrs)
+    if (!aligned16(q)) return LQ_ERR_ALIGN;
+  return LQ_OK;
+}
+
+// arrays that are only read or written one element at a time need their natural alignment only
+static lq_status check_scalar_ptrs(std::initializer_list<const void *> ptrs, unsigned elem_bytes) {
+  for (const void *q : ptrs)
+    if (!q) return LQ_ERR_NULL;
+  for (const void *q : ptrs)
+    if (reinterpret_cast<uintptr_t>(q) & (elem_bytes - 1)) return LQ_ERR_ALIGN;
+  return LQ_OK;
+}
+
+static lq_status check_state(const lq_shape *s, const lq_state *st, bool need_buffers) {
+  if (!st) return LQ_ERR_NULL;
+  lq_status rc = check_ptrs({st->codes, st->col_scale, st->row_smooth});
+  if (rc != LQ_OK) return rc;
+  if ((rc = check_scalar_ptrs({st->win_pos}, 4)) != LQ_OK) return rc;
+  if (s->r > 0 && (rc = check_ptrs({st->comp_k, st->comp_u})) != LQ_OK) return rc;
+  if (need_buffers && (rc = check_ptrs({st->buf_k, st->buf_u, st->buf_a})) != LQ_OK) return rc;
+  return LQ_OK;
+}
+
+static Params make_params(const lq_shape *s, const lq_state *st) {
+  Params p{};
+  p.batch = s->batch; p.heads_v = s->heads_v; p.heads_qk = s->heads_qk; p.W = s->W; p.r = s->r;
+  p.n_iter = s->n_iter; p.smooth = s->smooth; p.force = 0;
+  if (st) {
+    p.codes = st->codes; p.col_scale = st->col_scale; p.row_smooth = st->row_smooth;
+    p.comp_k = st->comp_k; p.comp_u = st->comp_u; p.buf_k = st->buf_k; p.buf_u = st->buf_u; p.buf_a = st->buf_a;
+    p.win_pos = st->win_pos;
+  }
+  return p;
+}
+
+static int sm_count() {
+  static int cached = 0;
+  if (!cached) {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
+      cached = n;
+    else
+      return 148;
+  }
+  return cached;
+}
+
+template <typename K>
+static lq_status launch(K kernel, int grid, int block, size_t smem, cudaStream_t stream, const Params &p) {
+  if (grid <= 0) return LQ_OK;
+  if (smem > 48 * 1024 &&
+      cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess) {
+    cudaGetLastError();
+    return LQ_ERR_CUDA;
+  }
+  kernel<<<grid, block, smem, stream>>>(p);
+  return cudaGetLastError() == cudaSuccess ? LQ_OK : LQ_ERR_CUDA;
+}
+
+template <int MODE>
+static lq_status launch_boundary(const lq_shape *s, const Params &p, cudaStream_t stream) {
+  const bool diag = s->gate == LQ_GATE_DIAG;
+  const size_t smem = BoundarySmem::bytes(s->W, s->r, diag);
+  const long nh = (long)s->batch * s->heads_v;
+  const int grid = static_cast<int>(nh < 4L * sm_count() ? nh : 4L * sm_count());
+  return diag ? launch(boundary_kernel<LQ_GATE_DIAG, MODE>, grid, 256, smem, stream, p)
+              : launch(boundary_kernel<LQ_GATE_SCALAR, MODE>, grid, 256, smem, stream, p);
+}
+
+}  // namespace lq
+
+using namespace lq;
+
+extern "C" {
+
+lq_status lq_decode_step(const lq_shape *shape, const lq_state *state, const uint16_t *q, const uint16_t *k,
+                         const uint16_t *v, const uint16_t *beta, const uint16_t *alpha, float *o, lq_stream stream) {
+  lq_status rc = check_shape(shape);
+  if (rc != LQ_OK) return rc;
+  if ((rc = check_state(shape, state, true)) != LQ_OK) return rc;
+  if ((rc = check_ptrs({q, k, v, o})) != LQ_OK) return rc;
+  if ((rc = check_scalar_ptrs({beta}, 2)) != LQ_OK) return rc;
+  if ((rc = shape->gate == LQ_GATE_DIAG ? check_ptrs({alpha}) : check_scalar_ptrs({alpha}, 2)) != LQ_OK) return rc;
+  Params p = make_params(shape, state);
+  p.q = q; p.k = k; p.v = v; p.beta = beta; p.alpha = alpha; p.o = o;
+  const bool diag = shape->gate == LQ_GATE_DIAG;
+  const int nh = shape->batch * shape->heads_v;
+  const size_t smem = DecodeSmem::bytes(shape->W, shape->r, diag);
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  rc = diag ? launch(decode_kernel<LQ_GATE_DIAG>, nh, 128, smem, st, p)
+            : launch(decode_kernel<LQ_GATE_SCALAR>, nh, 128, smem, st, p);
+  if (rc != LQ_OK) return rc;
+  return launch_boundary<0>(shape, p, st);     // sequences whose window just became full
+}
+
+uint64_t lq_decode_stage_bytes(const lq_shape *s) {
+  if (check_shape(s) != LQ_OK) return 0;
+  const uint64_t B = s->batch, Hv = s->heads_v, Hqk = s->heads_qk, K = s->d_k, V = s->d_v;
+  auto up = [](uint64_t x) { return (x + 255) / 256 * 256; };
+  const uint64_t na = s->gate == LQ_GATE_DIAG ? B * Hv * K : B * Hv;
+  return 2 * up(2 * B * Hqk * K) + up(2 * B * Hv * V) + up(2 * B * Hv) + up(2 * na) + up(4 * B * Hv * V);
+}
+
+lq_status lq_decode_step_host(const lq_shape *shape, const lq_state *state, const uint16_t *q_h, const uint16_t *k_h,
+                              const uint16_t *v_h, const uint16_t *beta_h, const uint16_t *alpha_h, float *o_h,
+                              void *stage, lq_stream stream) {
+  lq_status rc = check_shape(shape);
+  if (rc != LQ_OK) return rc;
+  if (!q_h || !k_h || !v_h || !beta_h || !alpha_h || !o_h || !stage) return LQ_ERR_NULL;
+  if (!aligned16(stage)) return LQ_ERR_ALIGN;
+  const uint64_t B = shape->batch, Hv = shape->heads_v, Hqk = shape->heads_qk, K = shape->d_k, V = shape->d_v;
+  auto up = [](uint64_t x) { return (x + 255) / 256 * 256; };
+  const uint64_t nqk = 2 * B * Hqk * K, nv = 2 * B * Hv * V, nb = 2 * B * Hv;
+  const uint64_t na = 2 * (shape->gate == LQ_GATE_DIAG ? B * Hv * K : B * Hv), no = 4 * B * Hv * V;
+  char *base = static_cast<char *>(stage);
+  uint16_t *q_d = reinterpret_cast<uint16_t *>(base); base += up(nqk);
+  uint16_t *k_d = reinterpret_cast<uint16_t *>(base); base += up(nqk);
+  uint16_t *v_d = reinterpret_cast<uint16_t *>(base); base += up(nv);
+  uint16_t *b_d = reinterpret_cast<uint16_t *>(base); base += up(nb);
+  uint16_t *a_d = reinterpret_cast<uint16_t *>(base); base += up(na);
+  float *o_d = reinterpret_cast<float *>(base);
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (B == 0) return LQ_OK;
+  if (cudaMemcpyAsync(q_d, q_h, nqk, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(k_d, k_h, nqk, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(v_d, v_h, nv, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(b_d, beta_h, nb, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(a_d, alpha_h, na, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+    cudaGetLastError();
+    return LQ_ERR_CUDA;
+  }
+  rc = lq_decode_step(shape, state, q_d, k_d, v_d, b_d, a_d, o_d, stream);
+  if (rc != LQ_OK) return rc;
+  if (cudaMemcpyAsync(o_h, o_d, no, cudaMemcpyDeviceToHost, st) != cudaSuccess) {
+    cudaGetLastError();
+    return LQ_ERR_CUDA;
+  }
+  return LQ_OK;
+}
+
+lq_status lq_window_flush(const lq_shape *shape, const lq_state *state, int force, lq_stream stream) {
+  lq_status rc = check_shape(shape);
+  if (rc != LQ_OK) return rc;
+  if ((rc = check_state(shape, state, true)) != LQ_OK) return rc;
+  Params p = make_params(shape, state);
+  p.force = force ? 1 : 0;
+  return launch_boundary<0>(shape, p, reinterpret_cast<cudaStream_t>(stream));
+}
+
+lq_status lq_quantize_state(const lq_shape *shape, const float *S, const lq_state *state, lq_stream stream) {
+  lq_status rc = check_shape(shape);
+  if (rc != LQ_OK) return rc;
+  if ((rc = check_state(shape, state, false)) != LQ_OK) return rc;
+  if ((rc = check_ptrs({S})) != LQ_OK) return rc;
+  Params p = make_params(shape, state);
+  p.S = const_cast<float *>(S);
+  return launch_boundary<1>(shape, p, reinterpret_cast<cudaStream_t>(stream));
+}
+
+lq_status lq_dequantize_state(const lq_shape *shape, const lq_state *state, float *S, lq_stream stream) {
+  lq_status rc = check_shape(shape);
+  if (rc != LQ_OK) return rc;
+  if ((rc = check_state(shape, state, true)) != LQ_OK) return rc;
+  if ((rc = check_ptrs({S})) != LQ_OK) return rc;
+  Params p = make_params(shape, state);
+  p.S = S;
+  return launch_boundary<2>(shape, p, reinterpret_cast<cudaStream_t>(stream));
+}
+
+static lq_status ref_step(const lq_shape *shape, float *S, uint16_t *S16, const uint16_t *q, const uint16_t *k,
+                          const uint16_t *v, const uint16_t *beta, const uint16_t *alpha, float *o, lq_stream stream) {
+  lq_shape s = *shape;
+  s.W = 1; s.r = 0; s.n_iter = 1;      // unused by the baseline
+  lq_status rc = check_shape(&s);
+  if (rc != LQ_OK) return rc;
+  if ((rc = check_ptrs({S ? (const void *)S : (const void *)S16, q, k, v, o})) != LQ_OK) return rc;
+  if ((rc = check_scalar_ptrs({beta}, 2)) != LQ_OK) return rc;
+  if ((rc = s.gate == LQ_GATE_DIAG ? check_ptrs({alpha}) : check_scalar_ptrs({alpha}, 2)) != LQ_OK) return rc;
+  Params p = make_params(&s, nullptr);
+  p.S = S; p.S16 = S16; p.q = q; p.k = k; p.v = v; p.beta = beta; p.alpha = alpha; p.o = o;
+  const int nh = s.batch * s.heads_v;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const bool diag = s.gate == LQ_GATE_DIAG;
+  if (S16) return diag ? launch(ref_kernel<LQ_GATE_DIAG, true>, nh, 256, 0, st, p)
+                       : launch(ref_kernel<LQ_GATE_SCALAR, true>, nh, 256, 0, st, p);
+  return diag ? launch(ref_kernel<LQ_GATE_DIAG, false>, nh, 256, 0, st, p)
+              : launch(ref_kernel<LQ_GATE_SCALAR, false>, nh, 256, 0, st, p);
+}
+
+lq_status lq_ref_decode_step_f32(const lq_shape *shape, float *S, const uint16_t *q, const uint16_t *k,
+                                 const uint16_t *v, const uint16_t *beta, const uint16_t *alpha, float *o,
+                                 lq_stream stream) {
+  if (!shape) return LQ_ERR_NULL;
+  if (!S) return LQ_ERR_NULL;
+  return ref_step(shape, S, nullptr, q, k, v, beta, alpha, o, stream);
+}
+
+lq_status lq_ref_decode_step_bf16(const lq_shape *shape, uint16_t *S, const uint16_t *q, const uint16_t *k,
+                                  const uint16_t *v, const uint16_t *beta, const uint16_t *alpha, float *o,
+                                  lq_stream stream) {
+  if (!shape) return LQ_ERR_NULL;
+  if (!S) return LQ_ERR_NULL;
+  return ref_step(shape, nullptr, S, q, k, v, beta, alpha, o, stream);
+}
+
+int lq_decode_launches(const lq_shape *shape) { return check_shape(shape) == LQ_OK && shape->batch > 0 ? 2 : 0; }
+
+const char *lq_status_string(lq_status status) {
+  switch (status) {
+    case LQ_OK: return "ok";
+    case LQ_ERR_NULL: return "null pointer";
+    case LQ_ERR_SHAPE: return "invalid shape";
+    case LQ_ERR_ALIGN: return "pointer not 16-byte aligned";
+    case LQ_ERR_UNSUPPORTED: return "shape not supported";
+    case LQ_ERR_CUDA: return "CUDA runtime error";
+  }
+  return "unknown status";
+}
+
+int lq_version(void) { return 1; }
+
+}  // extern "C"

@@ -1,0 +1,264 @@
+// Window-boundary work on one 128x128 state held as 8x8 register tiles by a CTA of 256 threads:
+// reconstruction of the dense state from the window representation (Eq. 7) and its quantization
+// (Compensator-Token fit by power iteration with deflation, Eqs. 5-6; residual smoothing, Sec. 3.4;
+// per-value-channel symmetric 8-bit codes, Appendix B.3).
+#pragma once
+#include "lq_common.cuh"
+
+namespace lq {
+
+// Shared-memory plan of the boundary kernels (floats).
+struct BoundarySmem {
+  float *kd;     // [W][128]  buffered write keys, turned in place into Gamma_{j+1:n} kt_j
+  float *bu;     // [W][128]  buffered corrections u_j
+  float *ba;     // [W][128]  diagonal-gate decays of the records (diagonal gate only), else [W]
+  float *ck;     // [r][128]  compensator keys widened to fp32
+  float *cu;     // [r][128]  compensator values widened to fp32
+  float *vec;    // [128]     row-sum results (t of the power iteration, row mean-abs)
+  float *part;   // [8][128]  per-warp column partial sums
+  float *gam;    // [128]     Gamma_{1:n}
+  float *cs;     // [128]     smoothing scales c
+  float *ss;     // [128]     B_j / 127
+  __device__ __forceinline__ BoundarySmem(float *base, int W, int r, bool diag) {
+    kd = base; bu = kd + W * D; ba = bu + W * D; ck = ba + (diag ? W * D : MAX_W);
+    cu = ck + r * D; vec = cu + r * D; part = vec + D; gam = part + 8 * D; cs = gam + D; ss = cs + D;
+  }
+  static size_t bytes(int W, int r, bool diag) {
+    return sizeof(float) * (size_t)(2 * W * D + (diag ? W * D : MAX_W) + 2 * r * D + D + 8 * D + 3 * D);
+  }
+};
+
+// Eq. 7 for the tile of thread t: M = Gamma_{1:n}[C (Z/127) B + Kc Uc^T] + sum_j Gamma_{j+1:n} kt_j u_j^T,
+// evaluated per element as  base = c_i*(Z_ij*s_j); base = fma(kc_hi, uc_hj, base) for h = 0..r-1;
+// x = gamma_i*base; x = fma(kd_ji, u_jj, x) for j = 0..n-1.  No sum crosses threads.
+// Leaves the CTA's shared memory holding the records; ends after its last read of it (no trailing barrier).
+template <int GATE>
+__device__ __forceinline__ void reconstruct_tile(const Params &p, const BoundarySmem &sm, const Tile &t, size_t bh,
+                                                 int n, float (&M)[8][8]) {
+  const int W = p.W, r = p.r;
+  // this thread's codes: 8 rows x 8 bytes, issued first so that they fly while the records are staged
+  uint2 z[8];
+  {
+    const int8_t *Z = p.codes + bh * (size_t)(D * D);
+#pragma unroll
+    for (int a = 0; a < 8; a++) z[a] = *reinterpret_cast<const uint2 *>(Z + (8 * t.ty + a) * D + 8 * t.tx);
+  }
+  // stage the n records, the compensators and the scales in shared memory
+  {
+    const float *bk = p.buf_k + bh * (size_t)(W * D), *bu = p.buf_u + bh * (size_t)(W * D);
+    for (int e = t.tid; e < n * (D / 4); e += 256) {
+      cp_async16(sm.kd + 4 * e, bk + 4 * e);
+      cp_async16(sm.bu + 4 * e, bu + 4 * e);
+    }
+    if (GATE == LQ_GATE_DIAG) {
+      const float *ba = p.buf_a + bh * (size_t)(W * D);
+      for (int e = t.tid; e < n * (D / 4); e += 256) cp_async16(sm.ba + 4 * e, ba + 4 * e);
+    } else if (t.tid < n) {
+      sm.ba[t.tid] = p.buf_a[bh * (size_t)W + t.tid];
+    }
+    cp_async_commit();
+    const uint16_t *gk = p.comp_k + bh * (size_t)(r * D), *gu = p.comp_u + bh * (size_t)(r * D);
+    for (int e = t.tid; e < r * D; e += 256) {
+      sm.ck[e] = f16_bits(gk[e]);
+      sm.cu[e] = f16_bits(gu[e]);
+    }
+    if (t.tid < D) {
+      sm.cs[t.tid] = p.row_smooth[bh * D + t.tid];
+      sm.ss[t.tid] = p.col_scale[bh * D + t.tid] / 127.0f;
+    }
+    cp_async_wait_all();
+  }
+  __syncthreads();
+  // cumulative decays, newest record first (Appendix B.2): kd_j = Gamma_{j+1:n} kt_j, gam = Gamma_{1:n}
+  if (t.tid < D) {
+    const int i = t.tid;
+    float g = 1.0f;
+    for (int j = n - 1; j >= 0; j--) {
+      sm.kd[j * D + i] = g * sm.kd[j * D + i];
+      g = g * (GATE == LQ_GATE_DIAG ? sm.ba[j * D + i] : sm.ba[j]);
+    }
+    sm.gam[i] = g;
+  }
+  __syncthreads();
+
+  float ci[8], gi[8], sj[8];
+  load8(sm.cs + 8 * t.ty, ci);
+  load8(sm.gam + 8 * t.ty, gi);
+  load8(sm.ss + 8 * t.tx, sj);
+#pragma unroll
+  for (int a = 0; a < 8; a++) {
+    const uint32_t lo = z[a].x, hi = z[a].y;
+#pragma unroll
+    for (int b = 0; b < 8; b++) {
+      const uint32_t word = b < 4 ? lo : hi;
+      const float zf = static_cast<float>(static_cast<int8_t>((word >> (8 * (b & 3))) & 0xFF));
+      M[a][b] = ci[a] * (zf * sj[b]);
+    }
+  }
+  for (int h = 0; h < r; h++) {
+    float kc[8], uc[8];
+    load8(sm.ck + h * D + 8 * t.ty, kc);
+    load8(sm.cu + h * D + 8 * t.tx, uc);
+#pragma unroll
+    for (int a = 0; a < 8; a++)
+#pragma unroll
+      for (int b = 0; b < 8; b++) M[a][b] = fmaf(kc[a], uc[b], M[a][b]);
+  }
+#pragma unroll
+  for (int a = 0; a < 8; a++)
+#pragma unroll
+    for (int b = 0; b < 8; b++) M[a][b] = gi[a] * M[a][b];
+  for (int j = 0; j < n; j++) {
+    float kj[8], uj[8];
+    load8(sm.kd + j * D + 8 * t.ty, kj);
+    load8(sm.bu + j * D + 8 * t.tx, uj);
+#pragma unroll
+    for (int a = 0; a < 8; a++)
+#pragma unroll
+      for (int b = 0; b < 8; b++) M[a][b] = fmaf(kj[a], uj[b], M[a][b]);
+  }
+}
+
+// Quantize the dense state held in M (destroyed) and write codes, scales and compensators of head bh.
+// Uses sm.vec and sm.part; begins with a barrier so that it may follow any other use of shared memory.
+__device__ __forceinline__ void quantize_tile(const Params &p, const BoundarySmem &sm, const Tile &t, size_t bh,
+                                              float (&M)[8][8]) {
+  const int r = p.r;
+  __syncthreads();
+  int h = 0;
+  for (; h < r; h++) {
+    float w[8], tn[8];
+    const float w0 = 1.0f / sqrtf(static_cast<float>(D));
+#pragma unroll
+    for (int b = 0; b < 8; b++) w[b] = w0;
+    bool vanished = false;
+    for (int it = 0; it < p.n_iter; it++) {
+      float pr[8];
+      row_blocks(M, w, pr);                                   // t = M w
+      int sel;
+      const float tv = row_tree(pr, t.lane, sel);
+      if (t.tx < 8) sm.vec[8 * t.ty + sel] = tv;
+      __syncthreads();
+      const float nu = dot128_shared(sm.vec, sm.vec, t.lane & 15);
+      if (nu < 1e-30f) { vanished = true; break; }            // same value in every thread
+      const float rinv = 1.0f / sqrtf(nu);
+      load8(sm.vec + 8 * t.ty, tn);
+#pragma unroll
+      for (int a = 0; a < 8; a++) tn[a] = tn[a] * rinv;
+      if (it + 1 < p.n_iter) {
+        float pc[8];
+        col_blocks(M, tn, pc);                                // w = M^T t
+        col_tree(pc, sm.part, t, w);
+      }
+    }
+    if (vanished) break;
+    // store the key side in fp16 and continue with the stored values
+    float kf[8], uf[8];
+    uint16_t kb[8], ub[8];
+#pragma unroll
+    for (int a = 0; a < 8; a++) { kb[a] = to_f16_bits_sat(tn[a]); kf[a] = f16_bits(kb[a]); }
+    {
+      float pc[8], uraw[8];
+      col_blocks(M, kf, pc);                                  // value side = M^T k
+      col_tree(pc, sm.part, t, uraw);
+#pragma unroll
+      for (int b = 0; b < 8; b++) { ub[b] = to_f16_bits_sat(uraw[b]); uf[b] = f16_bits(ub[b]); }
+    }
+    if (t.tx == 0) {
+      uint4 pk = make_uint4(kb[0] | (uint32_t)kb[1] << 16, kb[2] | (uint32_t)kb[3] << 16, kb[4] | (uint32_t)kb[5] << 16,
+                            kb[6] | (uint32_t)kb[7] << 16);
+      *reinterpret_cast<uint4 *>(p.comp_k + (bh * r + h) * (size_t)D + 8 * t.ty) = pk;
+    }
+    if (t.ty == 0) {
+      uint4 pu = make_uint4(ub[0] | (uint32_t)ub[1] << 16, ub[2] | (uint32_t)ub[3] << 16, ub[4] | (uint32_t)ub[5] << 16,
+                            ub[6] | (uint32_t)ub[7] << 16);
+      *reinterpret_cast<uint4 *>(p.comp_u + (bh * r + h) * (size_t)D + 8 * t.tx) = pu;
+    }
+#pragma unroll
+    for (int a = 0; a < 8; a++)
+#pragma unroll
+      for (int b = 0; b < 8; b++) M[a][b] = fmaf(-kf[a], uf[b], M[a][b]);
+  }
+  // a vanished component means nothing is left to fit: this and all later compensators are zero
+  for (; h < r; h++) {
+    if (t.tx == 0) *reinterpret_cast<uint4 *>(p.comp_k + (bh * r + h) * (size_t)D + 8 * t.ty) = make_uint4(0, 0, 0, 0);
+    if (t.ty == 0) *reinterpret_cast<uint4 *>(p.comp_u + (bh * r + h) * (size_t)D + 8 * t.tx) = make_uint4(0, 0, 0, 0);
+  }
+
+  // residual smoothing: c_i = max(sqrt(mean_j |R_ij|), 1e-6)
+  float c[8];
+  __syncthreads();   // every read of sm.vec / sm.part above is done
+  if (p.smooth) {
+    float pr[8];
+#pragma unroll
+    for (int a = 0; a < 8; a++) {
+      float s = fabsf(M[a][0]);
+#pragma unroll
+      for (int b = 1; b < 8; b++) s = s + fabsf(M[a][b]);
+      pr[a] = s;
+    }
+    int sel;
+    const float tot = row_tree(pr, t.lane, sel);
+    if (t.tx < 8) sm.vec[8 * t.ty + sel] = fmaxf(sqrtf(tot / static_cast<float>(D)), 1e-6f);
+    __syncthreads();
+    load8(sm.vec + 8 * t.ty, c);
+  } else {
+#pragma unroll
+    for (int a = 0; a < 8; a++) c[a] = 1.0f;
+  }
+  if (t.tx == 0) store8(p.row_smooth + bh * D + 8 * t.ty, c);
+#pragma unroll
+  for (int a = 0; a < 8; a++) {
+    const float inv_c = 1.0f / c[a];
+#pragma unroll
+    for (int b = 0; b < 8; b++) M[a][b] = M[a][b] * inv_c;
+  }
+  // per-value-channel scale: column maximum of |X| (exact in any order)
+  float amax[8];
+  {
+    float4 q;
+    float m[8];
+#pragma unroll
+    for (int b = 0; b < 8; b++) {
+      float s = fabsf(M[0][b]);
+#pragma unroll
+      for (int a = 1; a < 8; a++) s = fmaxf(s, fabsf(M[a][b]));
+      m[b] = fmaxf(s, __shfl_xor_sync(FULL, s, 16));
+    }
+    if (t.lane < 16) {
+      q = make_float4(m[0], m[1], m[2], m[3]);
+      *reinterpret_cast<float4 *>(sm.part + t.warp * D + 8 * t.tx) = q;
+      q = make_float4(m[4], m[5], m[6], m[7]);
+      *reinterpret_cast<float4 *>(sm.part + t.warp * D + 8 * t.tx + 4) = q;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int b = 0; b < 8; b++) amax[b] = 0.0f;
+#pragma unroll
+    for (int wv = 0; wv < 8; wv++) {
+      float x[8];
+      load8(sm.part + wv * D + 8 * t.tx, x);
+#pragma unroll
+      for (int b = 0; b < 8; b++) amax[b] = fmaxf(amax[b], x[b]);
+    }
+  }
+  if (t.ty == 0) store8(p.col_scale + bh * D + 8 * t.tx, amax);
+  float inv[8];
+#pragma unroll
+  for (int b = 0; b < 8; b++) inv[b] = amax[b] > 0.0f ? 127.0f / amax[b] : 0.0f;
+  int8_t *Z = p.codes + bh * (size_t)(D * D);
+#pragma unroll
+  for (int a = 0; a < 8; a++) {
+    uint32_t w2[2] = {0u, 0u};
+#pragma unroll
+    for (int b = 0; b < 8; b++) {
+      float zf = rintf(M[a][b] * inv[b]);                     // ties to even
+      zf = fminf(fmaxf(zf, -127.0f), 127.0f);
+      const uint32_t byte = static_cast<uint32_t>(static_cast<int>(zf)) & 0xFFu;
+      w2[b >> 2] |= byte << (8 * (b & 3));
+    }
+    *reinterpret_cast<uint2 *>(Z + (8 * t.ty + a) * D + 8 * t.tx) = make_uint2(w2[0], w2[1]);
+  }
+}
+
+}  // namespace lq

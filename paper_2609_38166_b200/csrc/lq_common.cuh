@@ -1,0 +1,192 @@
+// Device helpers shared by the sm_100a kernels of the per-window 8-bit decode step.
+//
+// Everything is compiled with -fmad=false: a product is fused with an addition only where fmaf() is
+// written, so that every value is reproducible bit for bit.  Sums over a channel index follow one
+// fixed order: blocks of eight consecutive terms accumulated left to right (first product rounded, the
+// rest folded in with fmaf), block results added as a balanced binary tree over the block index.
+// The thread mappings below are chosen so that this order is the natural one: a thread owns one block
+// of eight, neighbouring lanes own neighbouring blocks, and butterfly exchanges with lane masks
+// 1, 2, 4, ... walk up the tree.
+#pragma once
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/lq.h"
+
+namespace lq {
+
+constexpr int D = 128;       // d_k = d_v of the supported shape
+constexpr int MAX_W = 64;
+constexpr int MAX_R = 16;
+constexpr unsigned FULL = 0xffffffffu;
+
+// Launch-time description of one call, passed to the kernels by value.
+struct Params {
+  int batch, heads_v, heads_qk, W, r, n_iter, smooth, force;
+  int8_t *codes;
+  float *col_scale, *row_smooth;
+  uint16_t *comp_k, *comp_u;
+  float *buf_k, *buf_u, *buf_a;
+  int32_t *win_pos;
+  const uint16_t *q, *k, *v, *beta, *alpha;
+  float *o;
+  float *S;          // dense fp32 states (quantize / dequantize / fp32 baseline)
+  uint16_t *S16;     // dense bf16 states (bf16 baseline)
+};
+
+__device__ __forceinline__ float bf16_bits(uint16_t h) { return __uint_as_float(static_cast<uint32_t>(h) << 16); }
+__device__ __forceinline__ float f16_bits(uint16_t h) { return __half2float(__ushort_as_half(h)); }
+// binary32 -> binary16 bits, nearest even, clamped to the finite range first
+__device__ __forceinline__ uint16_t to_f16_bits_sat(float x) {
+  x = fminf(fmaxf(x, -65504.0f), 65504.0f);
+  return __half_as_ushort(__float2half_rn(x));
+}
+// binary32 -> bfloat16 bits, nearest even (finite inputs)
+__device__ __forceinline__ uint16_t to_bf16_bits(float x) {
+  uint32_t u = __float_as_uint(x);
+  u += 0x7FFFu + ((u >> 16) & 1u);
+  return static_cast<uint16_t>(u >> 16);
+}
+
+// ---- asynchronous global -> shared copies (16 bytes each) ----
+__device__ __forceinline__ void cp_async16(void *smem, const void *gmem) {
+  unsigned s = static_cast<unsigned>(__cvta_generic_to_shared(smem));
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;\n" ::: "memory"); }
+
+// ---- sum of sixteen block results held by sixteen neighbouring lanes (tree levels 1, 2, 4, 8) ----
+__device__ __forceinline__ float tree16(float x) {
+  x = x + __shfl_xor_sync(FULL, x, 1);
+  x = x + __shfl_xor_sync(FULL, x, 2);
+  x = x + __shfl_xor_sync(FULL, x, 4);
+  x = x + __shfl_xor_sync(FULL, x, 8);
+  return x;
+}
+
+// Dot product of two 128-vectors in shared memory, computed by sixteen neighbouring lanes
+// (lane c = lane & 15 owns block c); every one of the sixteen lanes returns the sum.
+__device__ __forceinline__ float dot128_shared(const float *a, const float *b, int c) {
+  const float4 a0 = *reinterpret_cast<const float4 *>(a + 8 * c), a1 = *reinterpret_cast<const float4 *>(a + 8 * c + 4);
+  const float4 b0 = *reinterpret_cast<const float4 *>(b + 8 * c), b1 = *reinterpret_cast<const float4 *>(b + 8 * c + 4);
+  float s = a0.x * b0.x;
+  s = fmaf(a0.y, b0.y, s); s = fmaf(a0.z, b0.z, s); s = fmaf(a0.w, b0.w, s);
+  s = fmaf(a1.x, b1.x, s); s = fmaf(a1.y, b1.y, s); s = fmaf(a1.z, b1.z, s); s = fmaf(a1.w, b1.w, s);
+  return tree16(s);
+}
+
+// =====================================================================================
+// 8x8 register tiles: a CTA of 256 threads holds one 128x128 state, thread (ty, tx) owning rows
+// 8ty..8ty+7 and columns 8tx..8tx+7, with tx = lane & 15 and ty = 2*warp + (lane >> 4).
+// =====================================================================================
+struct Tile {
+  int tid, lane, warp, tx, ty;
+  __device__ __forceinline__ Tile() {
+    tid = threadIdx.x; lane = tid & 31; warp = tid >> 5; tx = lane & 15; ty = tid >> 4;
+  }
+};
+
+__device__ __forceinline__ void load8(const float *src, float (&x)[8]) {
+  const float4 lo = *reinterpret_cast<const float4 *>(src), hi = *reinterpret_cast<const float4 *>(src + 4);
+  x[0] = lo.x; x[1] = lo.y; x[2] = lo.z; x[3] = lo.w; x[4] = hi.x; x[5] = hi.y; x[6] = hi.z; x[7] = hi.w;
+}
+__device__ __forceinline__ void store8(float *dst, const float (&x)[8]) {
+  *reinterpret_cast<float4 *>(dst) = make_float4(x[0], x[1], x[2], x[3]);
+  *reinterpret_cast<float4 *>(dst + 4) = make_float4(x[4], x[5], x[6], x[7]);
+}
+
+// Row sums.  In: p[a] = this thread's block result for row 8ty+a (block index tx).
+// Out: the full sum of row 8ty+sel, the same value in lanes tx and tx^8; sel depends on tx & 7 only.
+// Halving exchanges: after the step with mask m a lane keeps the rows whose partner-combined sums it owns.
+__device__ __forceinline__ float row_tree(const float (&p)[8], int lane, int &sel) {
+  float q4[4], q2[2], q1;
+  const bool u0 = lane & 1, u1 = lane & 2, u2 = lane & 4;
+#pragma unroll
+  for (int e = 0; e < 4; e++) {
+    const float keep = u0 ? p[e + 4] : p[e], send = u0 ? p[e] : p[e + 4];
+    q4[e] = keep + __shfl_xor_sync(FULL, send, 1);
+  }
+#pragma unroll
+  for (int e = 0; e < 2; e++) {
+    const float keep = u1 ? q4[e + 2] : q4[e], send = u1 ? q4[e] : q4[e + 2];
+    q2[e] = keep + __shfl_xor_sync(FULL, send, 2);
+  }
+  {
+    const float keep = u2 ? q2[1] : q2[0], send = u2 ? q2[0] : q2[1];
+    q1 = keep + __shfl_xor_sync(FULL, send, 4);
+  }
+  q1 = q1 + __shfl_xor_sync(FULL, q1, 8);
+  sel = (u0 ? 4 : 0) + (u1 ? 2 : 0) + (u2 ? 1 : 0);
+  return q1;
+}
+
+// Column sums.  In: p[b] = this thread's block result for column 8tx+b (block index ty).
+// part: 8*128 floats of shared memory.  Out: w[b] = full sum of column 8tx+b, in every thread.
+// Contains one __syncthreads(); `part` may be rewritten after the next barrier of the CTA.
+__device__ __forceinline__ void col_tree(const float (&p)[8], float *part, const Tile &t, float (&w)[8]) {
+  const bool up = t.lane & 16;
+  float4 q;
+  {
+    float r[4];
+#pragma unroll
+    for (int e = 0; e < 4; e++) {
+      const float keep = up ? p[e + 4] : p[e], send = up ? p[e] : p[e + 4];
+      r[e] = keep + __shfl_xor_sync(FULL, send, 16);      // rows 16w..16w+7 with rows 16w+8..16w+15
+    }
+    q = make_float4(r[0], r[1], r[2], r[3]);
+  }
+  *reinterpret_cast<float4 *>(part + t.warp * D + 8 * t.tx + (up ? 4 : 0)) = q;
+  __syncthreads();
+  // ((w0+w1)+(w2+w3)) + ((w4+w5)+(w6+w7)), four warps at a time to keep few values live
+  float half[2][8];
+#pragma unroll
+  for (int g = 0; g < 2; g++) {
+    float pr[2][8];
+#pragma unroll
+    for (int pair = 0; pair < 2; pair++) {
+      float x0[8], x1[8];
+      load8(part + (4 * g + 2 * pair) * D + 8 * t.tx, x0);
+      load8(part + (4 * g + 2 * pair + 1) * D + 8 * t.tx, x1);
+#pragma unroll
+      for (int b = 0; b < 8; b++) pr[pair][b] = x0[b] + x1[b];
+    }
+#pragma unroll
+    for (int b = 0; b < 8; b++) half[g][b] = pr[0][b] + pr[1][b];
+  }
+#pragma unroll
+  for (int b = 0; b < 8; b++) w[b] = half[0][b] + half[1][b];
+}
+
+// p[b] = block result over this thread's eight rows of  sum_a M[a][b] * x[a]
+__device__ __forceinline__ void col_blocks(const float (&M)[8][8], const float (&x)[8], float (&p)[8]) {
+#pragma unroll
+  for (int b = 0; b < 8; b++) {
+    float s = M[0][b] * x[0];
+#pragma unroll
+    for (int a = 1; a < 8; a++) s = fmaf(M[a][b], x[a], s);
+    p[b] = s;
+  }
+}
+// p[a] = block result over this thread's eight columns of  sum_b M[a][b] * x[b]
+__device__ __forceinline__ void row_blocks(const float (&M)[8][8], const float (&x)[8], float (&p)[8]) {
+#pragma unroll
+  for (int a = 0; a < 8; a++) {
+    float s = M[a][0] * x[0];
+#pragma unroll
+    for (int b = 1; b < 8; b++) s = fmaf(M[a][b], x[b], s);
+    p[a] = s;
+  }
+}
+
+// Last-arrival bookkeeping on win_pos[b]: bits 16.. count the heads of sequence b that are done with
+// the value in bits 0..15.  The head that arrives last (all heads_v have read the old value by then)
+// stores the new value and thereby clears the counter.  Call from one thread per head, after a
+// __syncthreads() that follows the head's last global write.
+__device__ __forceinline__ void arrive_and_set(int32_t *win_pos, int b, int heads_v, int new_value) {
+  const int old = atomicAdd(win_pos + b, 0x10000);
+  if ((old >> 16) == heads_v - 1) win_pos[b] = new_value;
+}
+
+}  // namespace lq
