@@ -16,6 +16,13 @@
  * -ffp-contract=off so that a product is fused with an addition only where
  * fmaf() is written.  bf16 inputs and fp16 compensators are widened exactly.
  *
+ * The boundary-state term of the readout, (B/127) Z^T (C Gamma x) in Appendix
+ * B.3, is an integer payload times a vector.  The paper leaves its arithmetic
+ * open; here the vector C Gamma x is taken in block fixed point (30 bits below
+ * the power of two that bounds its largest entry) and the products with the
+ * 8-bit codes are accumulated exactly, as integers.  The term is then free of
+ * summation order, and it is more accurate than an fp32 accumulation.
+ *
  * Summation order.  The paper never says in which order a sum is taken, yet
  * the 8-bit codes and the fp16 compensators are step functions of fp32
  * values, so the order has to be part of the definition.  Every reduction in
@@ -31,7 +38,8 @@
  *   reference recurrence, windowed decode, reconstruction, quantizer,
  *   smoothing, rank-r fit as a Frobenius minimiser        : pinned
  *   the constants n_iter, the all-equal start vector, the 1e-30 zero guard,
- *   the 1e-6 smoothing floor, the summation tree          : parity unpinned
+ *   the 1e-6 smoothing floor, the summation tree, the 30-bit fixed-point
+ *   grid of the readout vector                             : parity unpinned
  *   (the paper fixes none of them; they are this build's definition).
  */
 #include <math.h>
@@ -193,6 +201,25 @@ float lqo_csum_abs(const float *x, int n) {
 /* column j of a row-major d_k x d_v matrix, gathered so that it can be summed */
 static void column_of(const float *M, int d_k, int d_v, int j, float *out) {
   for (int i = 0; i < d_k; i++) out[i] = M[(size_t)i * d_v + j];
+}
+
+/* ------------------------------------------------------------------ */
+/* block fixed point for the readout vector                            */
+/* ------------------------------------------------------------------ */
+
+/* X_i = rint(x_i * 2^(29-e)) with 2^e <= max|x| < 2^(e+1), so that |X_i| <= 2^30; returns 2^(e-29), the
+ * factor that takes integers back (0 when the vector is zero or below 2^-96, in which case X = 0). */
+static float block_fixed_point(const float *x, int n, int32_t *X) {
+  float xmax = 0.0f;
+  for (int i = 0; i < n; i++) xmax = fmaxf(xmax, fabsf(x[i]));
+  if (!(xmax >= 0x1p-96f)) {
+    for (int i = 0; i < n; i++) X[i] = 0;
+    return 0.0f;
+  }
+  int e = (int)((f32_bits(xmax) >> 23) & 0xFF) - 127;       /* floor(log2 xmax); xmax is a normal number */
+  float scale = bits_f32((uint32_t)(29 - e + 127) << 23);   /* 2^(29-e) */
+  for (int i = 0; i < n; i++) X[i] = (int32_t)rintf(x[i] * scale);
+  return bits_f32((uint32_t)(e - 29 + 127) << 23);          /* 2^(e-29) */
 }
 
 /* ------------------------------------------------------------------ */
@@ -430,13 +457,16 @@ static void head_decode(const lqo_shape *sh, const head_view *hv, int n, const t
 
   float ktq = lqo_csum_dot(kt, t->q, K);
 
-  /* boundary-state term: (B/127) Z^T (C Gamma x); with quantization off it is S0^T (Gamma x) */
+  /* boundary-state term: (B/127) Z^T (C Gamma x), the vector in block fixed point and the sum exact;
+   * with quantization off it is S0^T (Gamma x) in fp32 */
   float *xk = (float *)malloc(sizeof(float) * K), *xq = (float *)malloc(sizeof(float) * K);
+  int32_t *Xk = (int32_t *)malloc(sizeof(int32_t) * K), *Xq = (int32_t *)malloc(sizeof(int32_t) * K);
   for (int i = 0; i < K; i++) {
-    float ci = hv->S0 ? 1.0f : hv->c[i];
-    xk[i] = hv->S0 ? gk[i] : ci * gk[i];
-    xq[i] = hv->S0 ? gq[i] : ci * gq[i];
+    xk[i] = hv->S0 ? gk[i] : hv->c[i] * gk[i];
+    xq[i] = hv->S0 ? gq[i] : hv->c[i] * gq[i];
   }
+  float back_k = 0.0f, back_q = 0.0f;
+  if (!hv->S0) { back_k = block_fixed_point(xk, K, Xk); back_q = block_fixed_point(xq, K, Xq); }
   for (int j = 0; j < V; j++) {
     float rk, rq;
     if (hv->S0) {
@@ -444,10 +474,14 @@ static void head_decode(const lqo_shape *sh, const head_view *hv, int n, const t
       rk = lqo_csum_dot(col, xk, K);
       rq = lqo_csum_dot(col, xq, K);
     } else {
-      for (int i = 0; i < K; i++) col[i] = (float)hv->Z[(size_t)i * V + j];
+      int64_t tk = 0, tq = 0;
+      for (int i = 0; i < K; i++) {
+        tk += (int64_t)hv->Z[(size_t)i * V + j] * Xk[i];
+        tq += (int64_t)hv->Z[(size_t)i * V + j] * Xq[i];
+      }
       float s = hv->B[j] / 127.0f;
-      rk = s * lqo_csum_dot(col, xk, K);
-      rq = s * lqo_csum_dot(col, xq, K);
+      rk = s * ((float)tk * back_k);
+      rq = s * ((float)tq * back_q);
       for (int h = 0; h < r; h++) {
         float uc = lqo_f16_to_f32(hv->cu[(size_t)h * V + j]);
         rk = fmaf(uc, ptk[h], rk);
@@ -469,7 +503,7 @@ static void head_decode(const lqo_shape *sh, const head_view *hv, int n, const t
   memcpy(hv->bu + (size_t)n * V, u, sizeof(float) * V);
 
   free(kt); free(g); free(gk); free(gq); free(dec); free(col); free(pk); free(pq); free(ck); free(u);
-  free(xk); free(xq);
+  free(xk); free(xq); free(Xk); free(Xq);
 }
 
 /* ------------------------------------------------------------------ */

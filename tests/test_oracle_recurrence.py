@@ -172,3 +172,26 @@ def test_bf16_state_baseline_rounds_state_each_token(oracle):
             # equal up to an occasional one-ulp difference where the fp32 and fp64 values straddle a tie
             assert np.mean(got != S64[h]) < 0.01 and np.allclose(got, S64[h], rtol=2.0 ** -7, atol=1e-8)
             S64[h] = got
+
+
+def test_boundary_term_is_exact_up_to_the_fixed_point_grid(oracle):
+    """(B/127) Z^T (C Gamma x) with the vector on a 30-bit block fixed-point grid and exact integer sums:
+    against float64 the error is the grid's (2^-29 of the largest entry per term) plus two fp32 roundings,
+    far below what an fp32 accumulation of 128 terms leaves."""
+    wl = synth.Workload("t", 2, 2, 2, 128, 128, W=4, r=0, seed=18)
+    sh = _shape(wl)
+    st = State(sh)
+    oracle.quantize_state(sh, synth.dense_states(wl, 3), st)
+    tok = synth.token_inputs(wl, 0)
+    oracle.decode_step(sh, st, **tok)          # n = 0, r = 0: u = v - (B/127) Z^T (c . alpha k)
+    for b in range(2):
+        for h in range(2):
+            q, k, v, beta, alpha = rm.widen(tok, wl, b, h)
+            c = st.row_smooth[b, h].astype(np.float64)
+            x = (c.astype(np.float32) * (np.float32(alpha) * k.astype(np.float32))).astype(np.float64)
+            s = (st.col_scale[b, h] / np.float32(127.0)).astype(np.float64)
+            Z = st.codes[b, h].astype(np.float64)
+            exact = s * (Z.T @ x)
+            got = v - st.buf_u[b, h, 0].astype(np.float64)
+            grid = 2.0 ** -29 * 2 * np.abs(x).max() * np.abs(Z).sum(axis=0) * s
+            assert np.all(np.abs(got - exact) <= grid + 3 * 2.0 ** -24 * (np.abs(exact) + np.abs(v)))
