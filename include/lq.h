@@ -71,7 +71,8 @@ typedef struct {
 
 /* Window representation of B x Hv states.  h is the value head. */
 typedef struct {
-  int8_t *codes;      /* [B,Hv,d_k,d_v]  Z, symmetric, in [-127,127]                        */
+  int8_t *codes;      /* [B,Hv,d_v,d_k]  Z^T: code of S[i][j] at [j][i] (value-channel major, so that
+                                         the key index is contiguous); symmetric, in [-127,127]  */
   float *col_scale;   /* [B,Hv,d_v]      B: dequant(Z) = (Z/127) B  (Appendix B.3)           */
   float *row_smooth;  /* [B,Hv,d_k]      c > 0 (Sec. 3.4)                                    */
   uint16_t *comp_k;   /* [B,Hv,r,d_k]    fp16, unit-length key side of the compensators     */

@@ -13,7 +13,7 @@ namespace lq {
 // MODE 1: quantize dense fp32 states         MODE 2: dequantize to dense fp32 states
 // ---------------------------------------------------------------------------------------------
 template <int GATE, int MODE>
-__global__ void __launch_bounds__(256) boundary_kernel(const Params p) {
+__global__ void __launch_bounds__(256, 2) boundary_kernel(const Params p) {
   extern __shared__ float4 lq_smem4[];
   const BoundarySmem sm(reinterpret_cast<float *>(lq_smem4), p.W, p.r, GATE == LQ_GATE_DIAG);
   const Tile t;
@@ -54,8 +54,8 @@ __global__ void __launch_bounds__(256) boundary_kernel(const Params p) {
 // Baseline: Eq. 1 on a dense state that is read and written in full every token.
 // ---------------------------------------------------------------------------------------------
 template <int GATE, bool BF16>
-__global__ void __launch_bounds__(256) ref_kernel(const Params p) {
-  __shared__ __align__(16) float kt_s[D], q_s[D], bv_s[D], a_s[D], part_s[8 * D];
+__global__ void __launch_bounds__(256, 2) ref_kernel(const Params p) {
+  __shared__ __align__(16) float kt_s[D], q_s[D], bv_s[D], a_s[D], col_s[D], part_s[8 * D];
   const Tile t;
   const size_t bh = blockIdx.x;
   const int b = static_cast<int>(bh / p.heads_v), hv = static_cast<int>(bh % p.heads_v);
@@ -91,7 +91,7 @@ __global__ void __launch_bounds__(256) ref_kernel(const Params p) {
   float x[8], pc[8], u[8], o[8], kt[8], ai[8];
   load8(bv_s + 8 * t.ty, x);
   col_blocks(M, x, pc);
-  col_tree(pc, part_s, t, u);                            // S^T (alpha.k)
+  col_tree(pc, part_s, col_s, t, u);                           // S^T (alpha.k)
 #pragma unroll
   for (int c = 0; c < 8; c++) u[c] = bf16_bits(p.v[bh * D + 8 * t.tx + c]) - u[c];
   load8(kt_s + 8 * t.ty, kt);
@@ -102,8 +102,7 @@ __global__ void __launch_bounds__(256) ref_kernel(const Params p) {
     for (int c = 0; c < 8; c++) M[a][c] = fmaf(kt[a], u[c], ai[a] * M[a][c]);
   load8(q_s + 8 * t.ty, x);
   col_blocks(M, x, pc);
-  __syncthreads();                                       // part_s is reused
-  col_tree(pc, part_s, t, o);
+  col_tree(pc, part_s, col_s, t, o);
   if (t.ty == 0) store8(p.o + bh * D + 8 * t.tx, o);
   if (BF16) {
     uint16_t *S = p.S16 + bh * (size_t)(D * D);

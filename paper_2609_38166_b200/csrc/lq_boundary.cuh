@@ -15,16 +15,17 @@ struct BoundarySmem {
   float *ck;     // [r][128]  compensator keys widened to fp32
   float *cu;     // [r][128]  compensator values widened to fp32
   float *vec;    // [128]     row-sum results (t of the power iteration, row mean-abs)
+  float *colv;   // [128]     column-sum results
   float *part;   // [8][128]  per-warp column partial sums
   float *gam;    // [128]     Gamma_{1:n}
   float *cs;     // [128]     smoothing scales c
   float *ss;     // [128]     B_j / 127
   __device__ __forceinline__ BoundarySmem(float *base, int W, int r, bool diag) {
     kd = base; bu = kd + W * D; ba = bu + W * D; ck = ba + (diag ? W * D : MAX_W);
-    cu = ck + r * D; vec = cu + r * D; part = vec + D; gam = part + 8 * D; cs = gam + D; ss = cs + D;
+    cu = ck + r * D; vec = cu + r * D; colv = vec + D; part = colv + D; gam = part + 8 * D; cs = gam + D; ss = cs + D;
   }
   static size_t bytes(int W, int r, bool diag) {
-    return sizeof(float) * (size_t)(2 * W * D + (diag ? W * D : MAX_W) + 2 * r * D + D + 8 * D + 3 * D);
+    return sizeof(float) * (size_t)(2 * W * D + (diag ? W * D : MAX_W) + 2 * r * D + 2 * D + 8 * D + 3 * D);
   }
 };
 
@@ -36,12 +37,13 @@ template <int GATE>
 __device__ __forceinline__ void reconstruct_tile(const Params &p, const BoundarySmem &sm, const Tile &t, size_t bh,
                                                  int n, float (&M)[8][8]) {
   const int W = p.W, r = p.r;
-  // this thread's codes: 8 rows x 8 bytes, issued first so that they fly while the records are staged
+  // this thread's codes: the layout is value-channel major (Z^T), so a column of the tile is 8 contiguous
+  // bytes; issued first so that they fly while the records are staged
   uint2 z[8];
   {
-    const int8_t *Z = p.codes + bh * (size_t)(D * D);
+    const int8_t *ZT = p.codes + bh * (size_t)(D * D);
 #pragma unroll
-    for (int a = 0; a < 8; a++) z[a] = *reinterpret_cast<const uint2 *>(Z + (8 * t.ty + a) * D + 8 * t.tx);
+    for (int b = 0; b < 8; b++) z[b] = *reinterpret_cast<const uint2 *>(ZT + (8 * t.tx + b) * D + 8 * t.ty);
   }
   // stage the n records, the compensators and the scales in shared memory
   {
@@ -86,12 +88,12 @@ __device__ __forceinline__ void reconstruct_tile(const Params &p, const Boundary
   load8(sm.gam + 8 * t.ty, gi);
   load8(sm.ss + 8 * t.tx, sj);
 #pragma unroll
-  for (int a = 0; a < 8; a++) {
-    const uint32_t lo = z[a].x, hi = z[a].y;
+  for (int b = 0; b < 8; b++) {
+    const uint32_t lo = z[b].x, hi = z[b].y;
 #pragma unroll
-    for (int b = 0; b < 8; b++) {
-      const uint32_t word = b < 4 ? lo : hi;
-      const float zf = static_cast<float>(static_cast<int8_t>((word >> (8 * (b & 3))) & 0xFF));
+    for (int a = 0; a < 8; a++) {
+      const uint32_t word = a < 4 ? lo : hi;
+      const float zf = static_cast<float>(static_cast<int8_t>((word >> (8 * (a & 3))) & 0xFF));
       M[a][b] = ci[a] * (zf * sj[b]);
     }
   }
@@ -148,7 +150,7 @@ __device__ __forceinline__ void quantize_tile(const Params &p, const BoundarySme
       if (it + 1 < p.n_iter) {
         float pc[8];
         col_blocks(M, tn, pc);                                // w = M^T t
-        col_tree(pc, sm.part, t, w);
+        col_tree(pc, sm.part, sm.colv, t, w);
       }
     }
     if (vanished) break;
@@ -160,7 +162,7 @@ __device__ __forceinline__ void quantize_tile(const Params &p, const BoundarySme
     {
       float pc[8], uraw[8];
       col_blocks(M, kf, pc);                                  // value side = M^T k
-      col_tree(pc, sm.part, t, uraw);
+      col_tree(pc, sm.part, sm.colv, t, uraw);
 #pragma unroll
       for (int b = 0; b < 8; b++) { ub[b] = to_f16_bits_sat(uraw[b]); uf[b] = f16_bits(ub[b]); }
     }
@@ -246,18 +248,18 @@ __device__ __forceinline__ void quantize_tile(const Params &p, const BoundarySme
   float inv[8];
 #pragma unroll
   for (int b = 0; b < 8; b++) inv[b] = amax[b] > 0.0f ? 127.0f / amax[b] : 0.0f;
-  int8_t *Z = p.codes + bh * (size_t)(D * D);
+  int8_t *ZT = p.codes + bh * (size_t)(D * D);
 #pragma unroll
-  for (int a = 0; a < 8; a++) {
+  for (int b = 0; b < 8; b++) {
     uint32_t w2[2] = {0u, 0u};
 #pragma unroll
-    for (int b = 0; b < 8; b++) {
+    for (int a = 0; a < 8; a++) {
       float zf = rintf(M[a][b] * inv[b]);                     // ties to even
       zf = fminf(fmaxf(zf, -127.0f), 127.0f);
       const uint32_t byte = static_cast<uint32_t>(static_cast<int>(zf)) & 0xFFu;
-      w2[b >> 2] |= byte << (8 * (b & 3));
+      w2[a >> 2] |= byte << (8 * (a & 3));
     }
-    *reinterpret_cast<uint2 *>(Z + (8 * t.ty + a) * D + 8 * t.tx) = make_uint2(w2[0], w2[1]);
+    *reinterpret_cast<uint2 *>(ZT + (8 * t.tx + b) * D + 8 * t.ty) = make_uint2(w2[0], w2[1]);
   }
 }
 

@@ -123,11 +123,11 @@ __device__ __forceinline__ float row_tree(const float (&p)[8], int lane, int &se
 }
 
 // Column sums.  In: p[b] = this thread's block result for column 8tx+b (block index ty).
-// part: 8*128 floats of shared memory.  Out: w[b] = full sum of column 8tx+b, in every thread.
-// Contains one __syncthreads(); `part` may be rewritten after the next barrier of the CTA.
-__device__ __forceinline__ void col_tree(const float (&p)[8], float *part, const Tile &t, float (&w)[8]) {
+// part: 8*128 floats and out: 128 floats of shared memory.  Returns w[b] = full sum of column 8tx+b in
+// every thread.  Tree levels: ty^1 inside the warp (lane^16), then warps (0,1)(2,3)(4,5)(6,7), pairs of
+// pairs, halves.  Contains two __syncthreads(); `part` and `out` may be rewritten after the CTA's next barrier.
+__device__ __forceinline__ void col_tree(const float (&p)[8], float *part, float *out, const Tile &t, float (&w)[8]) {
   const bool up = t.lane & 16;
-  float4 q;
   {
     float r[4];
 #pragma unroll
@@ -135,28 +135,15 @@ __device__ __forceinline__ void col_tree(const float (&p)[8], float *part, const
       const float keep = up ? p[e + 4] : p[e], send = up ? p[e] : p[e + 4];
       r[e] = keep + __shfl_xor_sync(FULL, send, 16);      // rows 16w..16w+7 with rows 16w+8..16w+15
     }
-    q = make_float4(r[0], r[1], r[2], r[3]);
+    *reinterpret_cast<float4 *>(part + t.warp * D + 8 * t.tx + (up ? 4 : 0)) = make_float4(r[0], r[1], r[2], r[3]);
   }
-  *reinterpret_cast<float4 *>(part + t.warp * D + 8 * t.tx + (up ? 4 : 0)) = q;
   __syncthreads();
-  // ((w0+w1)+(w2+w3)) + ((w4+w5)+(w6+w7)), four warps at a time to keep few values live
-  float half[2][8];
-#pragma unroll
-  for (int g = 0; g < 2; g++) {
-    float pr[2][8];
-#pragma unroll
-    for (int pair = 0; pair < 2; pair++) {
-      float x0[8], x1[8];
-      load8(part + (4 * g + 2 * pair) * D + 8 * t.tx, x0);
-      load8(part + (4 * g + 2 * pair + 1) * D + 8 * t.tx, x1);
-#pragma unroll
-      for (int b = 0; b < 8; b++) pr[pair][b] = x0[b] + x1[b];
-    }
-#pragma unroll
-    for (int b = 0; b < 8; b++) half[g][b] = pr[0][b] + pr[1][b];
+  if (t.tid < D) {
+    const float *c = part + t.tid;
+    out[t.tid] = ((c[0] + c[D]) + (c[2 * D] + c[3 * D])) + ((c[4 * D] + c[5 * D]) + (c[6 * D] + c[7 * D]));
   }
-#pragma unroll
-  for (int b = 0; b < 8; b++) w[b] = half[0][b] + half[1][b];
+  __syncthreads();
+  load8(out + 8 * t.tx, w);
 }
 
 // p[b] = block result over this thread's eight rows of  sum_a M[a][b] * x[a]

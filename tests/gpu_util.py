@@ -34,12 +34,17 @@ def tok_dev(tok: dict) -> dict:
 
 def state_to_dev(ost: OState, lsh) -> "lq.State":
     st = lq.State(lsh)
-    st.codes.copy_(dev(ost.codes)); st.col_scale.copy_(dev(ost.col_scale)); st.row_smooth.copy_(dev(ost.row_smooth))
+    st.codes.copy_(dev(np.ascontiguousarray(ost.codes.transpose(0, 1, 3, 2)))); st.col_scale.copy_(dev(ost.col_scale)); st.row_smooth.copy_(dev(ost.row_smooth))
     if lsh.r > 0:
         st.comp_k.copy_(dev(ost.comp_k).view(torch.float16)); st.comp_u.copy_(dev(ost.comp_u).view(torch.float16))
     st.buf_k.copy_(dev(ost.buf_k)); st.buf_u.copy_(dev(ost.buf_u)); st.buf_a.copy_(dev(ost.buf_a))
     st.win_pos.copy_(dev(ost.win_pos))
     return st
+
+
+def gpu_codes(st) -> np.ndarray:
+    """the library keeps Z^T ([B,Hv,d_v,d_k]); returns Z as [B,Hv,d_k,d_v] like the oracle"""
+    return np.ascontiguousarray(host(st.codes).transpose(0, 1, 3, 2))
 
 
 def code_mismatch(gpu_codes: np.ndarray, ref_codes: np.ndarray):
@@ -53,7 +58,7 @@ def assert_state_parity(st: "lq.State", ost: OState, r: int, what: str = "", exa
     within 1e-3 relative / 1e-5 absolute.  With `exact` (the default) every array must match bit for bit,
     which the fixed summation order makes possible."""
     torch.cuda.synchronize()
-    frac, worst = code_mismatch(host(st.codes), ost.codes)
+    frac, worst = code_mismatch(gpu_codes(st), ost.codes)
     assert worst <= 1 and frac <= 1e-4, (what, frac, worst)
     pairs = [("col_scale", host(st.col_scale), ost.col_scale), ("row_smooth", host(st.row_smooth), ost.row_smooth),
              ("buf_k", host(st.buf_k), ost.buf_k), ("buf_u", host(st.buf_u), ost.buf_u),

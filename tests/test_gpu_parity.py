@@ -168,7 +168,8 @@ def test_forced_flush_and_skip_of_full_windows(oracle):
     assert torch.all(o[1] == 7.0) and not torch.any(o[0] == 7.0)
     assert st.win_pos.tolist() == [1, 0, 1, 1]
     oracle.window_flush(osh, ost, force=False)
-    for name in ("codes", "col_scale", "row_smooth"):
+    assert np.array_equal(gu.gpu_codes(st)[1], ost.codes[1])
+    for name in ("col_scale", "row_smooth"):
         assert np.array_equal(gu.host(getattr(st, name))[1], getattr(ost, name)[1]), name
     assert np.array_equal(gu.host(st.comp_u)[1], ost.comp_u[1])
 
@@ -193,7 +194,7 @@ def test_sub_batches_by_pointer_offset(oracle):
         getattr(ost_sub, name)[...] = getattr(ost, name)[2:5]
     want = oracle.decode_step(osub, ost_sub, **{k: np.ascontiguousarray(v[2:5]) for k, v in tok.items()})
     _close(gu.host(o)[2:5], want, "sub-batch o")
-    assert np.array_equal(gu.host(st.codes)[2:5], ost_sub.codes)
+    assert np.array_equal(gu.gpu_codes(st)[2:5], ost_sub.codes)
     assert st.win_pos.tolist() == [3, 3, 0, 0, 0, 3]
 
 
