@@ -149,6 +149,13 @@ lq_status lq_ref_decode_step_bf16(const lq_shape *shape, uint16_t *S, const uint
                                   const uint16_t *v, const uint16_t *beta, const uint16_t *alpha, float *o,
                                   lq_stream stream);
 
+/*
+ * Device-side error flags of the current device (0 = none), written to *flags (a host pointer).  Waits inside
+ * the kernels are bounded; bit 0 is set when a decode warp gave up waiting for its asynchronous copies, in
+ * which case the outputs of that launch are not valid.  The call synchronises the device.
+ */
+lq_status lq_check_device(int *flags);
+
 /* Kernels one lq_decode_step call launches for `shape` (used to report launch counts). */
 int lq_decode_launches(const lq_shape *shape);
 

@@ -1,5 +1,6 @@
 // C boundary of the library: argument checks, launch configuration, and the kernels that wrap the
 // device routines of lq_decode.cuh and lq_boundary.cuh.  Declarations and contracts: include/lq.h.
+#include <algorithm>
 #include <cstdio>
 
 #include "lq_boundary.cuh"
@@ -226,11 +227,14 @@ lq_status lq_decode_step(const lq_shape *shape, const lq_state *state, const uin
   Params p = make_params(shape, state);
   p.q = q; p.k = k; p.v = v; p.beta = beta; p.alpha = alpha; p.o = o;
   const bool diag = shape->gate == LQ_GATE_DIAG;
-  const int nh = shape->batch * shape->heads_v;
-  const size_t smem = DecodeSmem::bytes(shape->W, shape->r, diag);
+  const long nh = (long)shape->batch * shape->heads_v;
+  // one-warp CTAs, each with a shared-memory slot that holds a whole head; as many per SM as fit
+  const size_t smem = DecodeSlot(shape->W, shape->r, diag).bytes;
+  const long per_sm = std::max<long>(1, std::min<long>(32, (227 * 1024) / (long)(smem + 1024)));
+  const int grid = static_cast<int>(std::min<long>(nh, per_sm * sm_count()));
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-  rc = diag ? launch(decode_kernel<LQ_GATE_DIAG>, nh, 128, smem, st, p)
-            : launch(decode_kernel<LQ_GATE_SCALAR>, nh, 128, smem, st, p);
+  rc = diag ? launch(decode_kernel<LQ_GATE_DIAG>, grid, 32, smem, st, p)
+            : launch(decode_kernel<LQ_GATE_SCALAR>, grid, 32, smem, st, p);
   if (rc != LQ_OK) return rc;
   return launch_boundary<0>(shape, p, st);     // sequences whose window just became full
 }
@@ -343,6 +347,17 @@ lq_status lq_ref_decode_step_bf16(const lq_shape *shape, uint16_t *S, const uint
   if (!shape) return LQ_ERR_NULL;
   if (!S) return LQ_ERR_NULL;
   return ref_step(shape, nullptr, S, q, k, v, beta, alpha, o, stream);
+}
+
+lq_status lq_check_device(int *flags) {
+  if (!flags) return LQ_ERR_NULL;
+  int v = 0;
+  if (cudaMemcpyFromSymbol(&v, g_device_error, sizeof(int)) != cudaSuccess) {
+    cudaGetLastError();
+    return LQ_ERR_CUDA;
+  }
+  *flags = v;
+  return LQ_OK;
 }
 
 int lq_decode_launches(const lq_shape *shape) { return check_shape(shape) == LQ_OK && shape->batch > 0 ? 2 : 0; }

@@ -1,43 +1,52 @@
-// Decode: one token for one (sequence, value head), done by a team of 128 threads (4 warps).
+// Decode: one token for one (sequence, value head), done by ONE WARP.
 //
 // Eq. 10 (readout of the smoothed, compensated window representation) evaluated for x = alpha.k and
 // x = alpha.q in one pass over the 8-bit codes:
 //   S_{l-1}^T (alpha.x) = (B/127) Z^T (C Gamma_{1:l} x) + Uc (Kc^T Gamma_{1:l} x) + sum_j u_j (kt_j^T Gamma_{j+1:l} x)
 // then u = v - S_{l-1}^T(alpha.k) (Eq. 3), o = S_{l-1}^T(alpha.q) + u (kt^T q), and the record is appended.
 //
-// The first term is a dense int8 contraction, Z^T [128 x 128] against the two vectors.  The vectors are
-// put on a 30-bit block fixed-point grid and split into four signed base-256 digits each, which gives an
-// int8 operand of 128 x 8; the tensor cores (mma.sync m16n8k32, s8 x s8 -> s32) then produce exact
-// integer sums, which are recombined in 64-bit integers and rounded to fp32 once.  The result does not
-// depend on the order of accumulation.  The codes are stored value-channel major (Z^T, [d_v][d_k]), so
-// that the key index, the contraction index, is contiguous in memory as the MMA operand layout needs.
+// Data movement: everything a head needs (16 KiB of codes, the two scale vectors, the compensators and the
+// n buffered records) is brought into the warp's own shared-memory slot by TMA bulk copies that complete on
+// an mbarrier; the warp loads the token's vectors meanwhile, waits once, and computes out of shared memory.
+// A warp therefore keeps a whole head (about 27 KB at W = 16) in flight, and nothing in the kernel needs a
+// CTA-wide barrier: warps are independent workers that walk over the heads with a grid stride.
 //
-// All 16 KiB of codes of a head are requested by eight 16-byte loads per thread at entry and consumed
-// after the (much smaller) record walk, so a team has its whole state in flight at once.
+// Arithmetic: the first term is a dense int8 contraction, Z^T [128 x 128] against the two vectors.  The
+// vectors are put on a 30-bit block fixed-point grid and split into four signed base-256 digits each, which
+// gives an int8 operand of 128 x 8; the tensor cores (mma.sync m16n8k32, s8 x s8 -> s32) produce exact
+// integer sums, recombined in 64-bit integers and rounded to fp32 once, so the result does not depend on
+// the order of accumulation.  The codes are stored value-channel major (Z^T, [d_v][d_k]): the contraction
+// index is then contiguous, as the MMA operand layout needs.  The small dot products against records and
+// compensators run on the fp32 pipes in the library's fixed summation order.
 #pragma once
 #include "lq_common.cuh"
 
 namespace lq {
 
-struct DecodeSmem {
-  float *bk, *bu, *ba;      // staged records: [W][128], [W][128], [W][128] (diag) or [MAX_W] (scalar)
-  float *ck, *cu;           // compensators widened to fp32: [r][128] each
-  float *kf, *qf, *kt;      // token vectors
-  float *gk, *gq;           // Gamma_{1:l} k, Gamma_{1:l} q
-  float *yk, *yq;           // exact integer sums of the state stream, rounded to fp32
-  float *pk, *pq;           // [MAX_W + MAX_R + 1] projections; the last used slot of pq holds kt^T q
-  float *gs;                // [MAX_W] scalar-gate decays Gamma_{j+1:l}
-  float *wmax;              // [4 warps][2] per-warp maxima of |C Gamma k|, |C Gamma q|
-  int8_t *digits;           // [8][128] digit planes: plane 4v+d = digit d of vector v (0: k, 1: q)
-  __device__ __forceinline__ DecodeSmem(float *base, int W, int r, bool diag) {
-    bk = base; bu = bk + W * D; ba = bu + W * D; ck = ba + (diag ? W * D : MAX_W); cu = ck + r * D;
-    kf = cu + r * D; qf = kf + D; kt = qf + D; gk = kt + D; gq = gk + D; yk = gq + D; yq = yk + D;
-    pk = yq + D; pq = pk + (MAX_W + MAX_R + 16); gs = pq + (MAX_W + MAX_R + 16); wmax = gs + MAX_W;
-    digits = reinterpret_cast<int8_t *>(wmax + 8);
-  }
-  static size_t bytes(int W, int r, bool diag) {
-    return sizeof(float) * (size_t)(2 * W * D + (diag ? W * D : MAX_W) + 2 * r * D + 7 * D +
-                                    2 * (MAX_W + MAX_R + 16) + MAX_W + 8) + 8 * D;
+// Set when a bounded wait gave up (bit 0: a decode warp's wait for its bulk copies).  Never cleared by kernels.
+__device__ int g_device_error = 0;
+
+// ---- per-warp shared-memory slot ----
+struct DecodeSlot {
+  // byte offsets inside a slot; every region starts on a 16-byte boundary
+  int zt, cs, bs, ck, cu, bk, bu, ba, digits, y, pk, pq, gs, mbar, bytes;
+  __host__ __device__ DecodeSlot(int W, int r, bool diag) {
+    int o = 0;
+    zt = o; o += D * D;                 // codes, Z^T
+    cs = o; o += 4 * D;                 // row_smooth
+    bs = o; o += 4 * D;                 // col_scale
+    ck = o; o += 2 * D * r;             // compensator keys, fp16
+    cu = o; o += 2 * D * r;             // compensator values, fp16
+    bk = o; o += 4 * D * W;             // buffered write keys
+    bu = o; o += 4 * D * W;             // buffered corrections
+    ba = o; o += diag ? 4 * D * W : 0;  // buffered diagonal decays, turned in place into Gamma_{j+1:l}
+    digits = o; o += 8 * D;             // digit planes: plane 4v+d = digit d of vector v (0: k, 1: q)
+    y = o; o += 2 * 4 * D;              // exact integer sums of the state stream, rounded to fp32: [2][128]
+    pk = o; o += 4 * (MAX_W + MAX_R + 16);
+    pq = o; o += 4 * (MAX_W + MAX_R + 16);   // projections; pq[n+r] holds kt^T q
+    gs = o; o += 4 * MAX_W;             // scalar-gate decays Gamma_{j+1:l}
+    mbar = o; o += 16;
+    bytes = (o + 127) / 128 * 128;
   }
 };
 
@@ -58,227 +67,312 @@ __device__ __forceinline__ void fixed_point_scales(float xmax, float &scale, flo
   back = __uint_as_float(static_cast<uint32_t>(e - 29 + 127) << 23);
 }
 
-// X = d0 + 256 d1 + 65536 d2 + 2^24 d3 with every digit in [-128, 127] (|X| <= 2^30)
-__device__ __forceinline__ void store_digits(int X, int8_t *plane0, int i) {
+// ---- mbarrier / TMA bulk copy (1-D) ----
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
+  asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+// global -> shared bulk copy; addresses and size are multiples of 16 bytes
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+// Bounded wait for phase `parity`; false if the limit ran out (the caller then reports and bails out).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  for (int spin = 0; spin < (1 << 20); spin++) {
+    uint32_t done;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(done)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    if (done) return true;
+  }
+  return false;
+}
+
+__device__ __forceinline__ void widen8_bf16(const uint4 w, float (&x)[8]) {
+  const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
-  for (int d = 0; d < 4; d++) {
-    const int dig = (X << 24) >> 24;      // sign-extended low byte
-    plane0[d * D + i] = static_cast<int8_t>(dig);
-    X = (X - dig) >> 8;
+  for (int e = 0; e < 4; e++) {
+    x[2 * e] = __uint_as_float(ws[e] << 16);
+    x[2 * e + 1] = __uint_as_float(ws[e] & 0xFFFF0000u);
+  }
+}
+__device__ __forceinline__ void widen8_f16(const uint4 w, float (&x)[8]) {
+  const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+  for (int e = 0; e < 4; e++) {
+    const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&ws[e]));
+    x[2 * e] = f.x;
+    x[2 * e + 1] = f.y;
   }
 }
 
-// The work of one team on head bh; tid in [0,128) is the thread's index within the team and `bar` the id
-// of the named barrier the team synchronises on (all 128 threads of the team must call this function).
+// Persistent kernel of one-warp CTAs: warp `gw` of the grid takes heads gw, gw + nwarps, ...
 template <int GATE>
-__device__ __forceinline__ void decode_head(const Params &p, const DecodeSmem &sm, const size_t bh, const int tid,
-                                            const int bar, const int n) {
+__global__ void __launch_bounds__(32) decode_kernel(const Params p) {
+  extern __shared__ __align__(128) unsigned char lq_smem_raw[];
   const int W = p.W, r = p.r;
-  const int lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
-  const int b = static_cast<int>(bh / p.heads_v), hv = static_cast<int>(bh % p.heads_v);
-  auto team_sync = [&]() { asm volatile("bar.sync %0, 128;\n" ::"r"(bar) : "memory"); };
+  const DecodeSlot L(W, r, GATE == LQ_GATE_DIAG);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int c = lane & 15, half = lane >> 4, g = lane >> 2, t = lane & 3;
+  unsigned char *slot = lq_smem_raw + (size_t)warp * L.bytes;
+  const int8_t *zt = reinterpret_cast<const int8_t *>(slot + L.zt);
+  const float *cs = reinterpret_cast<const float *>(slot + L.cs), *bs = reinterpret_cast<const float *>(slot + L.bs);
+  const uint16_t *ckh = reinterpret_cast<const uint16_t *>(slot + L.ck), *cuh = reinterpret_cast<const uint16_t *>(slot + L.cu);
+  const float *bk = reinterpret_cast<const float *>(slot + L.bk), *bu = reinterpret_cast<const float *>(slot + L.bu);
+  float *ba = reinterpret_cast<float *>(slot + L.ba);
+  int8_t *digits = reinterpret_cast<int8_t *>(slot + L.digits);
+  float *y = reinterpret_cast<float *>(slot + L.y), *pk = reinterpret_cast<float *>(slot + L.pk);
+  float *pq = reinterpret_cast<float *>(slot + L.pq), *gs = reinterpret_cast<float *>(slot + L.gs);
+  const uint32_t bar = smem_addr(slot + L.mbar), slot_a = smem_addr(slot);
 
-  // (1) the codes.  Warp w owns value channels 32w..32w+31 as two 16-row MMA tiles; a thread's 16 bytes of
-  // a row hold the key channels 64p+16t..64p+16t+15, which serve as the A fragments of two k-blocks.
-  uint4 zlo[2][2], zhi[2][2];
-  {
-    const int8_t *ZT = p.codes + bh * (size_t)(D * D);
-#pragma unroll
-    for (int mt = 0; mt < 2; mt++)
-#pragma unroll
-      for (int pp = 0; pp < 2; pp++) {
-        const int j = 32 * warp + 16 * mt + g;
-        zlo[mt][pp] = *reinterpret_cast<const uint4 *>(ZT + j * D + 64 * pp + 16 * t);
-        zhi[mt][pp] = *reinterpret_cast<const uint4 *>(ZT + (j + 8) * D + 64 * pp + 16 * t);
-      }
-  }
+  if (lane == 0) mbar_init(bar, 1);
+  __syncwarp();
+  uint32_t parity = 0;
 
-  // (2) records of the window so far -> shared memory, asynchronously
-  {
-    const float *bk = p.buf_k + bh * (size_t)(W * D), *bu = p.buf_u + bh * (size_t)(W * D);
-    for (int e = tid; e < n * (D / 4); e += 128) {
-      cp_async16(sm.bk + 4 * e, bk + 4 * e);
-      cp_async16(sm.bu + 4 * e, bu + 4 * e);
-    }
-    if (GATE == LQ_GATE_DIAG) {
-      const float *ba = p.buf_a + bh * (size_t)(W * D);
-      for (int e = tid; e < n * (D / 4); e += 128) cp_async16(sm.ba + 4 * e, ba + 4 * e);
-    } else if (tid < n) {
-      sm.ba[tid] = p.buf_a[bh * (size_t)W + tid];
-    }
-    cp_async_commit();
-  }
-
-  // (3) the token: thread i holds key channel i and value channel i
+  const size_t nh = (size_t)p.batch * p.heads_v;
+  const size_t nwarps = (size_t)gridDim.x * (blockDim.x >> 5);
   const int group = p.heads_v / p.heads_qk;
-  const size_t qk_off = ((size_t)b * p.heads_qk + hv / group) * D;
-  const float k_i = bf16_bits(p.k[qk_off + tid]), q_i = bf16_bits(p.q[qk_off + tid]);
-  const float v_j = bf16_bits(p.v[bh * D + tid]);
-  const float beta = bf16_bits(p.beta[bh]);
-  const float a_i = GATE == LQ_GATE_DIAG ? bf16_bits(p.alpha[bh * D + tid]) : bf16_bits(p.alpha[bh]);
-  const float kt_i = beta * k_i;
-  const float c_i = p.row_smooth[bh * D + tid];
-  const float s_j = p.col_scale[bh * D + tid] / 127.0f;
-  sm.kf[tid] = k_i; sm.qf[tid] = q_i; sm.kt[tid] = kt_i;
-  {
-    const uint16_t *gk = p.comp_k + bh * (size_t)(r * D), *gu = p.comp_u + bh * (size_t)(r * D);
-    for (int h = 0; h < r; h++) {
-      sm.ck[h * D + tid] = f16_bits(gk[h * D + tid]);
-      sm.cu[h * D + tid] = f16_bits(gu[h * D + tid]);
-    }
-  }
-  cp_async_wait_all();
-  team_sync();
 
-  // (4) cumulative decays from the newest record back (Appendix B.2).  After the loop gam = Gamma_{1:l}.
-  float gam = a_i;
-  if (GATE == LQ_GATE_DIAG) {
-    for (int j = n - 1; j >= 0; j--) {
-      const float aj = sm.ba[j * D + tid];
-      sm.ba[j * D + tid] = gam;            // Gamma_{j+1:l} for channel i, in place of the record's decay
-      gam = gam * aj;
-    }
-  } else {
-    for (int j = n - 1; j >= 0; j--) {     // every thread runs the same scalar chain
-      if (tid == 0) sm.gs[j] = gam;
-      gam = gam * sm.ba[j];
-    }
-  }
-  const float gk_i = gam * k_i, gq_i = gam * q_i;
-  const float xk_i = c_i * gk_i, xq_i = c_i * gq_i;
-  sm.gk[tid] = gk_i; sm.gq[tid] = gq_i;
-  {
-    float mk = fabsf(xk_i), mq = fabsf(xq_i);
-#pragma unroll
-    for (int m = 16; m >= 1; m >>= 1) {
-      mk = fmaxf(mk, __shfl_xor_sync(FULL, mk, m));
-      mq = fmaxf(mq, __shfl_xor_sync(FULL, mq, m));
-    }
-    if (lane == 0) { sm.wmax[2 * warp] = mk; sm.wmax[2 * warp + 1] = mq; }
-  }
-  team_sync();
+  for (size_t bh = (size_t)blockIdx.x * (blockDim.x >> 5) + warp; bh < nh; bh += nwarps) {
+    const int b = static_cast<int>(bh / p.heads_v), hv = static_cast<int>(bh % p.heads_v);
+    const int n = p.win_pos[b] & 0xFFFF;     // bits 16.. are the arrival counter of this launch
+    if (n >= W) continue;                    // nothing can be appended: the sequence gets no token
 
-  // (4b) the two vectors on their fixed-point grids, as digit planes for the B operand
-  float back_k, back_q;
-  {
-    const float xmk = fmaxf(fmaxf(sm.wmax[0], sm.wmax[2]), fmaxf(sm.wmax[4], sm.wmax[6]));
-    const float xmq = fmaxf(fmaxf(sm.wmax[1], sm.wmax[3]), fmaxf(sm.wmax[5], sm.wmax[7]));
-    float scale_k, scale_q;
-    fixed_point_scales(xmk, scale_k, back_k);
-    fixed_point_scales(xmq, scale_q, back_q);
-    store_digits(__float2int_rn(xk_i * scale_k), sm.digits, tid);
-    store_digits(__float2int_rn(xq_i * scale_q), sm.digits + 4 * D, tid);
-  }
+    // (1) request the head: bulk copies into the slot, completion counted in bytes on the mbarrier
+    if (lane == 0) {
+      // the slot was last touched through ordinary loads and stores; order them before the async writes
+      asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+      const uint32_t rec = 4u * D * n;
+      uint32_t total = D * D + 8u * D + 4u * D * r + 2u * rec + (GATE == LQ_GATE_DIAG ? rec : 0u);
+      mbar_expect_tx(bar, total);
+      bulk_g2s(slot_a + L.zt, p.codes + bh * (size_t)(D * D), D * D, bar);
+      bulk_g2s(slot_a + L.cs, p.row_smooth + bh * D, 4 * D, bar);
+      bulk_g2s(slot_a + L.bs, p.col_scale + bh * D, 4 * D, bar);
+      if (r > 0) {
+        bulk_g2s(slot_a + L.ck, p.comp_k + bh * (size_t)(r * D), 2 * D * r, bar);
+        bulk_g2s(slot_a + L.cu, p.comp_u + bh * (size_t)(r * D), 2 * D * r, bar);
+      }
+      if (n > 0) {
+        bulk_g2s(slot_a + L.bk, p.buf_k + bh * (size_t)(W * D), rec, bar);
+        bulk_g2s(slot_a + L.bu, p.buf_u + bh * (size_t)(W * D), rec, bar);
+        if (GATE == LQ_GATE_DIAG) bulk_g2s(slot_a + L.ba, p.buf_a + bh * (size_t)(W * D), rec, bar);
+      }
+    }
 
-  // (5) projections: one dot product pair per group of sixteen lanes (lane c owns block c of eight terms).
-  // The trip count is the same for both halves of a warp (the shuffles of tree16 name all 32 lanes): a
-  // half without a dot product of its own recomputes the last one and does not store it.
-  {
-    const int c = tid & 15, total = n + r + 1;
-    for (int jb = 2 * warp; jb < total; jb += 8) {
-      const int jown = jb + (lane >> 4);
-      const int j = jown < total ? jown : total - 1;
-      float a8[8], bk8[8], bq8[8];
-      if (j < n) {
-        load8(sm.bk + j * D + 8 * c, a8);
-        float k8[8], q8[8];
-        load8(sm.kf + 8 * c, k8);
-        load8(sm.qf + 8 * c, q8);
-        if (GATE == LQ_GATE_DIAG) {
-          float g8[8];
-          load8(sm.ba + j * D + 8 * c, g8);
+    // (2) the token, straight into registers.  Lane c (and its twin c+16) owns key channels 8c..8c+7;
+    // lane l owns value channels 4l..4l+3.
+    float k8[8], q8[8], kt8[8], a8[8], v4[4];
+    {
+      const size_t qk_off = ((size_t)b * p.heads_qk + hv / group) * D;
+      widen8_bf16(*reinterpret_cast<const uint4 *>(p.k + qk_off + 8 * c), k8);
+      widen8_bf16(*reinterpret_cast<const uint4 *>(p.q + qk_off + 8 * c), q8);
+      const uint2 vw = *reinterpret_cast<const uint2 *>(p.v + bh * D + 4 * lane);
+      v4[0] = __uint_as_float(vw.x << 16); v4[1] = __uint_as_float(vw.x & 0xFFFF0000u);
+      v4[2] = __uint_as_float(vw.y << 16); v4[3] = __uint_as_float(vw.y & 0xFFFF0000u);
+      const float beta = bf16_bits(p.beta[bh]);
+      if (GATE == LQ_GATE_DIAG) {
+        widen8_bf16(*reinterpret_cast<const uint4 *>(p.alpha + bh * D + 8 * c), a8);
+      } else {
+        const float a = bf16_bits(p.alpha[bh]);
 #pragma unroll
-          for (int e = 0; e < 8; e++) { bk8[e] = g8[e] * k8[e]; bq8[e] = g8[e] * q8[e]; }
-        } else {
-          const float gj = sm.gs[j];
+        for (int e = 0; e < 8; e++) a8[e] = a;
+      }
 #pragma unroll
-          for (int e = 0; e < 8; e++) { bk8[e] = gj * k8[e]; bq8[e] = gj * q8[e]; }
+      for (int e = 0; e < 8; e++) kt8[e] = beta * k8[e];
+    }
+    float ba_lo = 1.0f, ba_hi = 1.0f;        // scalar gate: decay of record `lane` and of record `lane + 32`
+    if (GATE == LQ_GATE_SCALAR) {
+      if (lane < n) ba_lo = p.buf_a[bh * (size_t)W + lane];
+      if (lane + 32 < n) ba_hi = p.buf_a[bh * (size_t)W + lane + 32];
+    }
+
+    // (3) wait for the slot (bounded: a copy that never lands must not hang the GPU)
+    if (!mbar_wait(bar, parity)) {
+      if (lane == 0) atomicOr(&g_device_error, 1);
+      mbar_wait(bar, parity);                // one more bounded wait for the copies in flight, then give up
+      return;
+    }
+    parity ^= 1u;
+
+    // (4) cumulative decays from the newest record back (Appendix B.2).  After the loop g8 = Gamma_{1:l}.
+    float g8[8];
+#pragma unroll
+    for (int e = 0; e < 8; e++) g8[e] = a8[e];
+    if (GATE == LQ_GATE_DIAG) {
+      for (int j = n - 1; j >= 0; j--) {
+        float aj[8];
+        load8(ba + j * D + 8 * c, aj);
+        __syncwarp();                        // both twins have read the decay before one of them replaces it
+        if (half == 0) store8(ba + j * D + 8 * c, g8);   // Gamma_{j+1:l} in place of the record's decay
+#pragma unroll
+        for (int e = 0; e < 8; e++) g8[e] = g8[e] * aj[e];
+      }
+    } else {
+      float gsc = a8[0];
+      for (int j = n - 1; j >= 0; j--) {     // every lane runs the same scalar chain
+        if (lane == (j & 31)) gs[j] = gsc;
+        gsc = gsc * __shfl_sync(FULL, j < 32 ? ba_lo : ba_hi, j & 31);
+      }
+#pragma unroll
+      for (int e = 0; e < 8; e++) g8[e] = gsc;
+    }
+    float gk8[8], gq8[8];
+#pragma unroll
+    for (int e = 0; e < 8; e++) { gk8[e] = g8[e] * k8[e]; gq8[e] = g8[e] * q8[e]; }
+
+    // (4b) C Gamma k (lanes 0..15) and C Gamma q (lanes 16..31) on their fixed-point grids, as digit planes
+    float back_own;
+    {
+      float c8[8], x8[8];
+      load8(cs + 8 * c, c8);
+      float m = 0.0f;
+#pragma unroll
+      for (int e = 0; e < 8; e++) {
+        x8[e] = c8[e] * (half ? gq8[e] : gk8[e]);
+        m = fmaxf(m, fabsf(x8[e]));
+      }
+#pragma unroll
+      for (int s = 1; s <= 8; s <<= 1) m = fmaxf(m, __shfl_xor_sync(FULL, m, s));
+      float scale;
+      fixed_point_scales(m, scale, back_own);
+      uint32_t lo[4] = {0u, 0u, 0u, 0u}, hi[4] = {0u, 0u, 0u, 0u};      // [digit]: bytes of elements 0..3 / 4..7
+#pragma unroll
+      for (int e = 0; e < 8; e++) {
+        int X = __float2int_rn(x8[e] * scale);
+#pragma unroll
+        for (int d = 0; d < 4; d++) {       // X = d0 + 256 d1 + 65536 d2 + 2^24 d3, digits in [-128, 127]
+          const int dig = (X << 24) >> 24;
+          const uint32_t byte = static_cast<uint32_t>(dig) & 0xFFu;
+          if (e < 4) lo[d] |= byte << (8 * e); else hi[d] |= byte << (8 * (e - 4));
+          X = (X - dig) >> 8;
         }
-      } else if (j < n + r) {
-        load8(sm.ck + (j - n) * D + 8 * c, a8);
-        load8(sm.gk + 8 * c, bk8);
-        load8(sm.gq + 8 * c, bq8);
-      } else {                               // kt^T q, stored in the pq slot; the pk slot is unused
-        load8(sm.kt + 8 * c, a8);
-        load8(sm.qf + 8 * c, bq8);
-#pragma unroll
-        for (int e = 0; e < 8; e++) bk8[e] = bq8[e];
       }
-      float sk = a8[0] * bk8[0], sq = a8[0] * bq8[0];
 #pragma unroll
-      for (int e = 1; e < 8; e++) { sk = fmaf(a8[e], bk8[e], sk); sq = fmaf(a8[e], bq8[e], sq); }
-      sk = tree16(sk);
-      sq = tree16(sq);
-      if (c == 0 && jown < total) { sm.pk[j] = sk; sm.pq[j] = sq; }
+      for (int d = 0; d < 4; d++)
+        *reinterpret_cast<uint2 *>(digits + (4 * half + d) * D + 8 * c) = make_uint2(lo[d], hi[d]);
     }
-  }
-  team_sync();                               // digit planes (and projections) are complete
+    const float back_other = __shfl_xor_sync(FULL, back_own, 16);
+    const float back_k = half ? back_other : back_own, back_q = half ? back_own : back_other;
+    __syncwarp();                            // in-place decays, gs and digit planes are visible to the warp
 
-  // (6) the state stream on the tensor cores
-  {
-    uint4 bf[2];
+    // (5) projections: the two halves of the warp take one dot-product pair each per trip (lane c owns block
+    // c of eight terms).  Both halves make the same number of trips: the shuffles name all 32 lanes.
+    {
+      const int total = n + r + 1;
+      for (int jb = 0; jb < total; jb += 2) {
+        const int jown = jb + half;
+        const int j = jown < total ? jown : total - 1;
+        float x8[8], yk8[8], yq8[8];
+        if (j < n) {
+          load8(bk + j * D + 8 * c, x8);
+          if (GATE == LQ_GATE_DIAG) {
+            float gj8[8];
+            load8(ba + j * D + 8 * c, gj8);
 #pragma unroll
-    for (int pp = 0; pp < 2; pp++) bf[pp] = *reinterpret_cast<const uint4 *>(sm.digits + g * D + 64 * pp + 16 * t);
+            for (int e = 0; e < 8; e++) { yk8[e] = gj8[e] * k8[e]; yq8[e] = gj8[e] * q8[e]; }
+          } else {
+            const float gj = gs[j];
 #pragma unroll
-    for (int mt = 0; mt < 2; mt++) {
-      int c4[4] = {0, 0, 0, 0};
+            for (int e = 0; e < 8; e++) { yk8[e] = gj * k8[e]; yq8[e] = gj * q8[e]; }
+          }
+        } else if (j < n + r) {
+          widen8_f16(*reinterpret_cast<const uint4 *>(ckh + (j - n) * D + 8 * c), x8);
 #pragma unroll
-      for (int pp = 0; pp < 2; pp++) {
-        mma_s8(c4, zlo[mt][pp].x, zhi[mt][pp].x, zlo[mt][pp].y, zhi[mt][pp].y, bf[pp].x, bf[pp].y);
-        mma_s8(c4, zlo[mt][pp].z, zhi[mt][pp].z, zlo[mt][pp].w, zhi[mt][pp].w, bf[pp].z, bf[pp].w);
-      }
-      // c4[0], c4[1]: row g, planes 2t, 2t+1;  c4[2], c4[3]: row g+8.  Planes 4v..4v+3 are the digits of
-      // vector v, so lanes t = 0, 1 carry the k sums and t = 2, 3 the q sums: even t the low digit pair.
-      long long lo = static_cast<long long>(c4[0]) + (static_cast<long long>(c4[1]) << 8);
-      long long hi = static_cast<long long>(c4[2]) + (static_cast<long long>(c4[3]) << 8);
-      if (t & 1) { lo <<= 16; hi <<= 16; }
-      lo += __shfl_xor_sync(FULL, lo, 1);
-      hi += __shfl_xor_sync(FULL, hi, 1);
-      if (!(t & 1)) {
-        float *dst = (t & 2) ? sm.yq : sm.yk;
-        const int j = 32 * warp + 16 * mt + g;
-        dst[j] = __ll2float_rn(lo);
-        dst[j + 8] = __ll2float_rn(hi);
+          for (int e = 0; e < 8; e++) { yk8[e] = gk8[e]; yq8[e] = gq8[e]; }
+        } else {                             // kt^T q, kept in the pq slot; the pk slot is unused
+#pragma unroll
+          for (int e = 0; e < 8; e++) { x8[e] = kt8[e]; yk8[e] = q8[e]; yq8[e] = q8[e]; }
+        }
+        float sk = x8[0] * yk8[0], sq = x8[0] * yq8[0];
+#pragma unroll
+        for (int e = 1; e < 8; e++) { sk = fmaf(x8[e], yk8[e], sk); sq = fmaf(x8[e], yq8[e], sq); }
+        sk = tree16(sk);
+        sq = tree16(sq);
+        if (c == 0 && jown < total) { pk[j] = sk; pq[j] = sq; }
       }
     }
-  }
-  team_sync();
 
-  // (7) per value channel j = tid: scale the sums, add compensator and record terms, emit u and o
-  {
-    const int j = tid;
-    float rk = s_j * (sm.yk[j] * back_k), rq = s_j * (sm.yq[j] * back_q);
-    for (int h = 0; h < r; h++) {
-      const float uc = sm.cu[h * D + j];
-      rk = fmaf(uc, sm.pk[n + h], rk);
-      rq = fmaf(uc, sm.pq[n + h], rq);
+    // (6) the state stream on the tensor cores: eight 16-row tiles of Z^T, K = 128 as four k-blocks.
+    // A thread's 16 bytes of a row hold key channels 64p+16t..64p+16t+15 and serve two k-blocks; the digit
+    // planes are read with the same permutation of the key index.
+    {
+      uint4 bf[2];
+#pragma unroll
+      for (int pp = 0; pp < 2; pp++) bf[pp] = *reinterpret_cast<const uint4 *>(digits + g * D + 64 * pp + 16 * t);
+#pragma unroll 2
+      for (int mt = 0; mt < 8; mt++) {
+        int c4[4] = {0, 0, 0, 0};
+        const int j = 16 * mt + g;
+#pragma unroll
+        for (int pp = 0; pp < 2; pp++) {
+          const uint4 zlo = *reinterpret_cast<const uint4 *>(zt + j * D + 64 * pp + 16 * t);
+          const uint4 zhi = *reinterpret_cast<const uint4 *>(zt + (j + 8) * D + 64 * pp + 16 * t);
+          mma_s8(c4, zlo.x, zhi.x, zlo.y, zhi.y, bf[pp].x, bf[pp].y);
+          mma_s8(c4, zlo.z, zhi.z, zlo.w, zhi.w, bf[pp].z, bf[pp].w);
+        }
+        // c4[0], c4[1]: row g, planes 2t, 2t+1;  c4[2], c4[3]: row g+8.  Planes 4v..4v+3 are the digits of
+        // vector v: lanes t = 0, 1 carry the k sums and t = 2, 3 the q sums, even t the low digit pair.
+        long long lo = static_cast<long long>(c4[0]) + (static_cast<long long>(c4[1]) << 8);
+        long long hi = static_cast<long long>(c4[2]) + (static_cast<long long>(c4[3]) << 8);
+        if (t & 1) { lo <<= 16; hi <<= 16; }
+        lo += __shfl_xor_sync(FULL, lo, 1);
+        hi += __shfl_xor_sync(FULL, hi, 1);
+        if (!(t & 1)) {
+          float *dst = y + (t >> 1) * D;
+          dst[j] = __ll2float_rn(lo);
+          dst[j + 8] = __ll2float_rn(hi);
+        }
+      }
     }
-    for (int jj = 0; jj < n; jj++) {
-      const float uj = sm.bu[jj * D + j];
-      rk = fmaf(uj, sm.pk[jj], rk);
-      rq = fmaf(uj, sm.pq[jj], rq);
-    }
-    const float u = v_j - rk;
-    const float o = fmaf(u, sm.pq[n + r], rq);
-    p.o[bh * D + j] = o;
-    p.buf_u[(bh * W + n) * (size_t)D + j] = u;
-    p.buf_k[(bh * W + n) * (size_t)D + j] = kt_i;
-    if (GATE == LQ_GATE_DIAG) p.buf_a[(bh * W + n) * (size_t)D + j] = a_i;
-    else if (tid == 0) p.buf_a[bh * W + n] = a_i;
-  }
-}
+    __syncwarp();
 
-template <int GATE>
-__global__ void __launch_bounds__(128) decode_kernel(const Params p) {
-  extern __shared__ float4 lq_smem4[];
-  const DecodeSmem sm(reinterpret_cast<float *>(lq_smem4), p.W, p.r, GATE == LQ_GATE_DIAG);
-  const size_t bh = blockIdx.x;
-  const int b = static_cast<int>(bh / p.heads_v);
-  const int n = p.win_pos[b] & 0xFFFF;       // bits 16.. are the arrival counter of this launch
-  if (n >= p.W) return;                      // nothing can be appended: the sequence gets no token
-  decode_head<GATE>(p, sm, bh, threadIdx.x, 1, n);
-  __syncthreads();
-  if (threadIdx.x == 0) arrive_and_set(p.win_pos, b, p.heads_v, n + 1);
+    // (7) per value channel (lane l: channels 4l..4l+3): scale the sums, add compensator and record terms
+    {
+      const float4 yk4 = *reinterpret_cast<const float4 *>(y + 4 * lane);
+      const float4 yq4 = *reinterpret_cast<const float4 *>(y + D + 4 * lane);
+      const float4 b4 = *reinterpret_cast<const float4 *>(bs + 4 * lane);
+      const float s4[4] = {b4.x / 127.0f, b4.y / 127.0f, b4.z / 127.0f, b4.w / 127.0f};
+      float rk[4] = {s4[0] * (yk4.x * back_k), s4[1] * (yk4.y * back_k), s4[2] * (yk4.z * back_k), s4[3] * (yk4.w * back_k)};
+      float rq[4] = {s4[0] * (yq4.x * back_q), s4[1] * (yq4.y * back_q), s4[2] * (yq4.z * back_q), s4[3] * (yq4.w * back_q)};
+      for (int h = 0; h < r; h++) {
+        const uint2 w = *reinterpret_cast<const uint2 *>(cuh + h * D + 4 * lane);
+        const float2 f01 = __half22float2(*reinterpret_cast<const __half2 *>(&w.x));
+        const float2 f23 = __half22float2(*reinterpret_cast<const __half2 *>(&w.y));
+        const float uc[4] = {f01.x, f01.y, f23.x, f23.y};
+        const float pkh = pk[n + h], pqh = pq[n + h];
+#pragma unroll
+        for (int e = 0; e < 4; e++) { rk[e] = fmaf(uc[e], pkh, rk[e]); rq[e] = fmaf(uc[e], pqh, rq[e]); }
+      }
+      for (int jj = 0; jj < n; jj++) {
+        const float4 u4 = *reinterpret_cast<const float4 *>(bu + jj * D + 4 * lane);
+        const float uj[4] = {u4.x, u4.y, u4.z, u4.w};
+        const float pkj = pk[jj], pqj = pq[jj];
+#pragma unroll
+        for (int e = 0; e < 4; e++) { rk[e] = fmaf(uj[e], pkj, rk[e]); rq[e] = fmaf(uj[e], pqj, rq[e]); }
+      }
+      const float ktq = pq[n + r];
+      float u[4], o[4];
+#pragma unroll
+      for (int e = 0; e < 4; e++) { u[e] = v4[e] - rk[e]; o[e] = fmaf(u[e], ktq, rq[e]); }
+      *reinterpret_cast<float4 *>(p.o + bh * D + 4 * lane) = make_float4(o[0], o[1], o[2], o[3]);
+      *reinterpret_cast<float4 *>(p.buf_u + (bh * W + n) * (size_t)D + 4 * lane) = make_float4(u[0], u[1], u[2], u[3]);
+      if (half == 0) {
+        store8(p.buf_k + (bh * W + n) * (size_t)D + 8 * c, kt8);
+        if (GATE == LQ_GATE_DIAG) store8(p.buf_a + (bh * W + n) * (size_t)D + 8 * c, a8);
+        else if (lane == 0) p.buf_a[bh * W + n] = a8[0];
+      }
+    }
+    __syncwarp();
+    if (lane == 0) arrive_and_set(p.win_pos, b, p.heads_v, n + 1);
+  }
 }
 
 }  // namespace lq

@@ -21,7 +21,7 @@ _lib = None
 
 EXPORTS = ["lq_decode_step", "lq_decode_step_host", "lq_decode_stage_bytes", "lq_window_flush",
            "lq_quantize_state", "lq_dequantize_state", "lq_ref_decode_step_f32", "lq_ref_decode_step_bf16",
-           "lq_decode_launches", "lq_status_string", "lq_version"]
+           "lq_decode_launches", "lq_check_device", "lq_status_string", "lq_version"]
 
 
 class LqError(RuntimeError):
@@ -52,7 +52,7 @@ def lib() -> C.CDLL:
         L.lq_decode_stage_bytes.argtypes = [C.c_void_p]
         L.lq_decode_launches.restype = C.c_int
         L.lq_decode_launches.argtypes = [C.c_void_p]
-        for name in ("lq_decode_step", "lq_decode_step_host", "lq_window_flush", "lq_quantize_state",
+        for name in ("lq_decode_step", "lq_decode_step_host", "lq_check_device", "lq_window_flush", "lq_quantize_state",
                      "lq_dequantize_state", "lq_ref_decode_step_f32", "lq_ref_decode_step_bf16"):
             getattr(L, name).restype = C.c_int
         _lib = L
@@ -191,6 +191,13 @@ def ref_decode_step_bf16(sh: Shape, S16, q, k, v, beta, alpha, o, stream=None):
     s = sh.c()
     _check(lib().lq_ref_decode_step_bf16(C.byref(s), _ptr(S16), _ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(alpha),
                                          _ptr(o), _stream(stream)), "lq_ref_decode_step_bf16")
+
+
+def check_device() -> int:
+    """lq_check_device: synchronises the device and returns the kernels' error flags (0 = none)."""
+    flags = C.c_int(0)
+    _check(lib().lq_check_device(C.byref(flags)), "lq_check_device")
+    return int(flags.value)
 
 
 def version() -> int:
