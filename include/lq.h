@@ -69,21 +69,38 @@ typedef struct {
   int smooth;   /* 1: residual smoothing (Sec. 3.4); 0: c = 1 (ablation)          */
 } lq_shape;
 
-/* Window representation of B x Hv states.  h is the value head. */
+/*
+ * Window representation of B x Hv states, laid out for bulk transfers: everything that is read once per
+ * token and head is contiguous.
+ *
+ * heads: one block of lq_head_bytes(shape) bytes per (sequence, value head), [B,Hv] blocks back to back:
+ *     offset 0                        codes      int8 [d_v][d_k]  Z^T: the code of S[i][j] sits at [j][i]
+ *                                                (value-channel major, so that the key index is contiguous);
+ *                                                symmetric, in [-127,127]
+ *     + d_k*d_v                       col_scale  fp32 [d_v]       step of the code per value channel, B_j/127:
+ *                                                dequant(Z)_ij = Z_ij * col_scale_j  (Appendix B.3)
+ *     + 4*d_v                         row_smooth fp32 [d_k]       c > 0 (Sec. 3.4)
+ *     + 4*d_k                         comp_k     fp16 [r][d_k]    unit-length key side of the compensators
+ *     + 2*r*d_k                       comp_u     fp16 [r][d_v]    value side (carries the magnitude)
+ *   (17408 + 512 r bytes at d_k = d_v = 128: 19456 for r = 4, i.e. 1.19 bytes per state element.)
+ *
+ * records: one row of lq_record_floats(shape) fp32 values per buffered record, [B,Hv,W] rows:
+ *     kt[d_k] | u[d_v]                write key kt = beta*k and correction u = v - S^T(alpha.k)  (Eq. 3)
+ *     | alpha[d_k]                    diagonal gate only: the record's decay
+ * decays: scalar gate only, fp32 [B,Hv,W]: the decay of each buffered record (ignored for the diagonal gate).
+ * win_pos: int32 [B], records buffered per sequence, 0..W-1 between calls.  Bits 16 and up are used as a
+ *     scratch counter while a call runs and are zero again when it has finished.
+ */
 typedef struct {
-  int8_t *codes;      /* [B,Hv,d_v,d_k]  Z^T: code of S[i][j] at [j][i] (value-channel major, so that
-                                         the key index is contiguous); symmetric, in [-127,127]  */
-  float *col_scale;   /* [B,Hv,d_v]      B: dequant(Z) = (Z/127) B  (Appendix B.3)           */
-  float *row_smooth;  /* [B,Hv,d_k]      c > 0 (Sec. 3.4)                                    */
-  uint16_t *comp_k;   /* [B,Hv,r,d_k]    fp16, unit-length key side of the compensators     */
-  uint16_t *comp_u;   /* [B,Hv,r,d_v]    fp16, value side (carries the magnitude)           */
-  float *buf_k;       /* [B,Hv,W,d_k]    write keys kt = beta*k of the buffered records     */
-  float *buf_u;       /* [B,Hv,W,d_v]    corrections u = v - S^T(alpha.k)  (Eq. 3)          */
-  float *buf_a;       /* [B,Hv,W] (scalar gate) or [B,Hv,W,d_k] (diagonal gate): decays     */
-  int32_t *win_pos;   /* [B]             records buffered per sequence, 0..W-1 between calls.
-                                         Bits 16 and up are used as a scratch counter while a
-                                         call runs and are zero again when it has finished.   */
+  uint8_t *heads;
+  float *records;
+  float *decays;
+  int32_t *win_pos;
 } lq_state;
+
+/* Size in bytes of one head block, and the number of fp32 values in one record row (0 for an invalid shape). */
+uint64_t lq_head_bytes(const lq_shape *shape);
+uint64_t lq_record_floats(const lq_shape *shape);
 
 /*
  * One decode token for every (sequence, value head): Eq. 10 (the readout of the smoothed, compensated

@@ -67,7 +67,7 @@ typedef struct {
 
 typedef struct {
   int8_t *codes;        /* [B,Hv,d_k,d_v]  Z                                */
-  float *col_scale;     /* [B,Hv,d_v]      B, per value channel             */
+  float *col_scale;     /* [B,Hv,d_v]      code step B_j/127, per value ch. */
   float *row_smooth;    /* [B,Hv,d_k]      c, per key row                   */
   uint16_t *comp_k;     /* [B,Hv,r,d_k]    fp16 bit patterns                */
   uint16_t *comp_u;     /* [B,Hv,r,d_v]    fp16 bit patterns                */
@@ -309,7 +309,7 @@ static void head_ref_step(const lqo_shape *sh, float *S, const token_in *t, floa
 /* Reconstruction of the state after the n buffered records, Eq. 7      */
 /* (Eq. 4 when there is no smoothing and no compensator):               */
 /*   S_n = Gamma_{1:n} [ C dequant(Z) + Kc Uc^T ] + sum_j Gamma_{j+1:n} kt_j u_j^T
- * with dequant(Z) = (Z/127) B (Appendix B.3).  The cumulative decays are
+ * with dequant(Z) = (Z/127) B (Appendix B.3; B/127 is what is stored).  The cumulative decays are
  * built up record by record from the newest one, as Appendix B.2 describes. */
 /* ------------------------------------------------------------------ */
 static void head_reconstruct(const lqo_shape *sh, const head_view *hv, int n, float *S) {
@@ -331,7 +331,7 @@ static void head_reconstruct(const lqo_shape *sh, const head_view *hv, int n, fl
       if (hv->S0) {
         base = hv->S0[(size_t)i * V + j];                        /* quantization switched off */
       } else {
-        float s = hv->B[j] / 127.0f;
+        float s = hv->B[j];                                       /* the stored step B_j/127 */
         base = hv->c[i] * ((float)hv->Z[(size_t)i * V + j] * s);
         for (int h = 0; h < r; h++)
           base = fmaf(lqo_f16_to_f32(hv->ck[(size_t)h * K + i]), lqo_f16_to_f32(hv->cu[(size_t)h * V + j]), base);
@@ -398,7 +398,7 @@ static void head_quantize(const lqo_shape *sh, float *M, const head_view *hv) {
   for (int j = 0; j < V; j++) {
     float amax = 0.0f;
     for (int i = 0; i < K; i++) amax = fmaxf(amax, fabsf(M[(size_t)i * V + j]));
-    hv->B[j] = amax;
+    hv->B[j] = amax / 127.0f;                 /* stored as the step of the code: dequant = Z * step */
     float inv = amax > 0.0f ? 127.0f / amax : 0.0f;
     for (int i = 0; i < K; i++) {
       float z = rintf(M[(size_t)i * V + j] * inv);          /* ties to even */
@@ -479,7 +479,7 @@ static void head_decode(const lqo_shape *sh, const head_view *hv, int n, const t
         tk += (int64_t)hv->Z[(size_t)i * V + j] * Xk[i];
         tq += (int64_t)hv->Z[(size_t)i * V + j] * Xq[i];
       }
-      float s = hv->B[j] / 127.0f;
+      float s = hv->B[j];
       rk = s * ((float)tk * back_k);
       rq = s * ((float)tq * back_q);
       for (int h = 0; h < r; h++) {

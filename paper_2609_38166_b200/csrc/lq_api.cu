@@ -155,11 +155,13 @@ static lq_status check_scalar_ptrs(std::initializer_list<const void *> ptrs, uns
 
 static lq_status check_state(const lq_shape *s, const lq_state *st, bool need_buffers) {
   if (!st) return LQ_ERR_NULL;
-  lq_status rc = check_ptrs({st->codes, st->col_scale, st->row_smooth});
+  lq_status rc = check_ptrs({st->heads});
   if (rc != LQ_OK) return rc;
   if ((rc = check_scalar_ptrs({st->win_pos}, 4)) != LQ_OK) return rc;
-  if (s->r > 0 && (rc = check_ptrs({st->comp_k, st->comp_u})) != LQ_OK) return rc;
-  if (need_buffers && (rc = check_ptrs({st->buf_k, st->buf_u, st->buf_a})) != LQ_OK) return rc;
+  if (need_buffers) {
+    if ((rc = check_ptrs({st->records})) != LQ_OK) return rc;
+    if (s->gate == LQ_GATE_SCALAR && (rc = check_scalar_ptrs({st->decays}, 4)) != LQ_OK) return rc;
+  }
   return LQ_OK;
 }
 
@@ -168,9 +170,7 @@ static Params make_params(const lq_shape *s, const lq_state *st) {
   p.batch = s->batch; p.heads_v = s->heads_v; p.heads_qk = s->heads_qk; p.W = s->W; p.r = s->r;
   p.n_iter = s->n_iter; p.smooth = s->smooth; p.force = 0;
   if (st) {
-    p.codes = st->codes; p.col_scale = st->col_scale; p.row_smooth = st->row_smooth;
-    p.comp_k = st->comp_k; p.comp_u = st->comp_u; p.buf_k = st->buf_k; p.buf_u = st->buf_u; p.buf_a = st->buf_a;
-    p.win_pos = st->win_pos;
+    p.heads = st->heads; p.records = st->records; p.decays = st->decays; p.win_pos = st->win_pos;
   }
   return p;
 }
@@ -198,6 +198,24 @@ static lq_status launch(K kernel, int grid, int block, size_t smem, cudaStream_t
   }
   kernel<<<grid, block, smem, stream>>>(p);
   return cudaGetLastError() == cudaSuccess ? LQ_OK : LQ_ERR_CUDA;
+}
+
+// grid = min(work items, CTAs that fit on the device at once), for kernels that stride over their work
+template <typename K>
+static lq_status launch_persistent(K kernel, long items, int block, size_t smem, cudaStream_t stream, const Params &p) {
+  if (items <= 0) return LQ_OK;
+  if (smem > 48 * 1024 &&
+      cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess) {
+    cudaGetLastError();
+    return LQ_ERR_CUDA;
+  }
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, block, smem) != cudaSuccess || per_sm < 1) {
+    cudaGetLastError();
+    return LQ_ERR_CUDA;
+  }
+  const long resident = (long)per_sm * sm_count();
+  return launch(kernel, static_cast<int>(items < resident ? items : resident), block, smem, stream, p);
 }
 
 template <int MODE>
@@ -228,15 +246,19 @@ lq_status lq_decode_step(const lq_shape *shape, const lq_state *state, const uin
   p.q = q; p.k = k; p.v = v; p.beta = beta; p.alpha = alpha; p.o = o;
   const bool diag = shape->gate == LQ_GATE_DIAG;
   const long nh = (long)shape->batch * shape->heads_v;
-  // one-warp CTAs, each with a shared-memory slot that holds a whole head; as many per SM as fit
+  // persistent two-warp CTAs, each with its own shared-memory slot: as many as are resident at once
   const size_t smem = DecodeSlot(shape->W, shape->r, diag).bytes;
-  const long per_sm = std::max<long>(1, std::min<long>(32, (227 * 1024) / (long)(smem + 1024)));
-  const int grid = static_cast<int>(std::min<long>(nh, per_sm * sm_count()));
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-  rc = diag ? launch(decode_kernel<LQ_GATE_DIAG>, grid, 32, smem, st, p)
-            : launch(decode_kernel<LQ_GATE_SCALAR>, grid, 32, smem, st, p);
+  rc = diag ? launch_persistent(decode_kernel<LQ_GATE_DIAG>, nh, 64, smem, st, p)
+            : launch_persistent(decode_kernel<LQ_GATE_SCALAR>, nh, 64, smem, st, p);
   if (rc != LQ_OK) return rc;
   return launch_boundary<0>(shape, p, st);     // sequences whose window just became full
+}
+
+uint64_t lq_head_bytes(const lq_shape *s) { return check_shape(s) == LQ_OK ? (uint64_t)head_bytes(s->r) : 0; }
+
+uint64_t lq_record_floats(const lq_shape *s) {
+  return check_shape(s) == LQ_OK ? (uint64_t)record_floats(s->gate == LQ_GATE_DIAG) : 0;
 }
 
 uint64_t lq_decode_stage_bytes(const lq_shape *s) {
@@ -359,6 +381,15 @@ lq_status lq_check_device(int *flags) {
   *flags = v;
   return LQ_OK;
 }
+
+#ifdef LQ_TIMING
+// development aid: copies the phase counters to host memory and clears them
+int lq_debug_phase_cycles(unsigned long long *out) {
+  unsigned long long zero[32] = {0};
+  if (cudaMemcpyFromSymbol(out, g_phase_cycles, sizeof(zero)) != cudaSuccess) return 1;
+  return cudaMemcpyToSymbol(g_phase_cycles, zero, sizeof(zero)) != cudaSuccess;
+}
+#endif
 
 int lq_decode_launches(const lq_shape *shape) { return check_shape(shape) == LQ_OK && shape->batch > 0 ? 2 : 0; }
 

@@ -19,7 +19,7 @@ struct BoundarySmem {
   float *part;   // [8][128]  per-warp column partial sums
   float *gam;    // [128]     Gamma_{1:n}
   float *cs;     // [128]     smoothing scales c
-  float *ss;     // [128]     B_j / 127
+  float *ss;     // [128]     code steps s_j = B_j / 127
   __device__ __forceinline__ BoundarySmem(float *base, int W, int r, bool diag) {
     kd = base; bu = kd + W * D; ba = bu + W * D; ck = ba + (diag ? W * D : MAX_W);
     cu = ck + r * D; vec = cu + r * D; colv = vec + D; part = colv + D; gam = part + 8 * D; cs = gam + D; ss = cs + D;
@@ -30,43 +30,42 @@ struct BoundarySmem {
 };
 
 // Eq. 7 for the tile of thread t: M = Gamma_{1:n}[C (Z/127) B + Kc Uc^T] + sum_j Gamma_{j+1:n} kt_j u_j^T,
-// evaluated per element as  base = c_i*(Z_ij*s_j); base = fma(kc_hi, uc_hj, base) for h = 0..r-1;
+// evaluated per element as  base = c_i*(Z_ij*s_j) with s_j the stored code step; base = fma(kc_hi, uc_hj, base) for h = 0..r-1;
 // x = gamma_i*base; x = fma(kd_ji, u_jj, x) for j = 0..n-1.  No sum crosses threads.
 // Leaves the CTA's shared memory holding the records; ends after its last read of it (no trailing barrier).
 template <int GATE>
 __device__ __forceinline__ void reconstruct_tile(const Params &p, const BoundarySmem &sm, const Tile &t, size_t bh,
                                                  int n, float (&M)[8][8]) {
   const int W = p.W, r = p.r;
+  constexpr bool DIAG = GATE == LQ_GATE_DIAG;
+  constexpr int RF = record_floats(DIAG);
   // this thread's codes: the layout is value-channel major (Z^T), so a column of the tile is 8 contiguous
   // bytes; issued first so that they fly while the records are staged
   uint2 z[8];
   {
-    const int8_t *ZT = p.codes + bh * (size_t)(D * D);
+    const int8_t *ZT = p.codes(bh);
 #pragma unroll
     for (int b = 0; b < 8; b++) z[b] = *reinterpret_cast<const uint2 *>(ZT + (8 * t.tx + b) * D + 8 * t.ty);
   }
   // stage the n records, the compensators and the scales in shared memory
   {
-    const float *bk = p.buf_k + bh * (size_t)(W * D), *bu = p.buf_u + bh * (size_t)(W * D);
+    const float *rec = p.record(bh, 0, DIAG);
     for (int e = t.tid; e < n * (D / 4); e += 256) {
-      cp_async16(sm.kd + 4 * e, bk + 4 * e);
-      cp_async16(sm.bu + 4 * e, bu + 4 * e);
+      const int j = e / (D / 4), q4 = 4 * (e % (D / 4));
+      cp_async16(sm.kd + j * D + q4, rec + j * RF + REC_KT + q4);
+      cp_async16(sm.bu + j * D + q4, rec + j * RF + REC_U + q4);
+      if (DIAG) cp_async16(sm.ba + j * D + q4, rec + j * RF + REC_A + q4);
     }
-    if (GATE == LQ_GATE_DIAG) {
-      const float *ba = p.buf_a + bh * (size_t)(W * D);
-      for (int e = t.tid; e < n * (D / 4); e += 256) cp_async16(sm.ba + 4 * e, ba + 4 * e);
-    } else if (t.tid < n) {
-      sm.ba[t.tid] = p.buf_a[bh * (size_t)W + t.tid];
-    }
+    if (!DIAG && t.tid < n) sm.ba[t.tid] = p.decays[bh * (size_t)W + t.tid];
     cp_async_commit();
-    const uint16_t *gk = p.comp_k + bh * (size_t)(r * D), *gu = p.comp_u + bh * (size_t)(r * D);
+    const uint16_t *gk = p.comp_k(bh), *gu = p.comp_u(bh);
     for (int e = t.tid; e < r * D; e += 256) {
       sm.ck[e] = f16_bits(gk[e]);
       sm.cu[e] = f16_bits(gu[e]);
     }
     if (t.tid < D) {
-      sm.cs[t.tid] = p.row_smooth[bh * D + t.tid];
-      sm.ss[t.tid] = p.col_scale[bh * D + t.tid] / 127.0f;
+      sm.cs[t.tid] = p.row_smooth(bh)[t.tid];
+      sm.ss[t.tid] = p.col_scale(bh)[t.tid];
     }
     cp_async_wait_all();
   }
@@ -169,12 +168,12 @@ __device__ __forceinline__ void quantize_tile(const Params &p, const BoundarySme
     if (t.tx == 0) {
       uint4 pk = make_uint4(kb[0] | (uint32_t)kb[1] << 16, kb[2] | (uint32_t)kb[3] << 16, kb[4] | (uint32_t)kb[5] << 16,
                             kb[6] | (uint32_t)kb[7] << 16);
-      *reinterpret_cast<uint4 *>(p.comp_k + (bh * r + h) * (size_t)D + 8 * t.ty) = pk;
+      *reinterpret_cast<uint4 *>(p.comp_k(bh) + h * D + 8 * t.ty) = pk;
     }
     if (t.ty == 0) {
       uint4 pu = make_uint4(ub[0] | (uint32_t)ub[1] << 16, ub[2] | (uint32_t)ub[3] << 16, ub[4] | (uint32_t)ub[5] << 16,
                             ub[6] | (uint32_t)ub[7] << 16);
-      *reinterpret_cast<uint4 *>(p.comp_u + (bh * r + h) * (size_t)D + 8 * t.tx) = pu;
+      *reinterpret_cast<uint4 *>(p.comp_u(bh) + h * D + 8 * t.tx) = pu;
     }
 #pragma unroll
     for (int a = 0; a < 8; a++)
@@ -183,8 +182,8 @@ __device__ __forceinline__ void quantize_tile(const Params &p, const BoundarySme
   }
   // a vanished component means nothing is left to fit: this and all later compensators are zero
   for (; h < r; h++) {
-    if (t.tx == 0) *reinterpret_cast<uint4 *>(p.comp_k + (bh * r + h) * (size_t)D + 8 * t.ty) = make_uint4(0, 0, 0, 0);
-    if (t.ty == 0) *reinterpret_cast<uint4 *>(p.comp_u + (bh * r + h) * (size_t)D + 8 * t.tx) = make_uint4(0, 0, 0, 0);
+    if (t.tx == 0) *reinterpret_cast<uint4 *>(p.comp_k(bh) + h * D + 8 * t.ty) = make_uint4(0, 0, 0, 0);
+    if (t.ty == 0) *reinterpret_cast<uint4 *>(p.comp_u(bh) + h * D + 8 * t.tx) = make_uint4(0, 0, 0, 0);
   }
 
   // residual smoothing: c_i = max(sqrt(mean_j |R_ij|), 1e-6)
@@ -208,7 +207,7 @@ __device__ __forceinline__ void quantize_tile(const Params &p, const BoundarySme
 #pragma unroll
     for (int a = 0; a < 8; a++) c[a] = 1.0f;
   }
-  if (t.tx == 0) store8(p.row_smooth + bh * D + 8 * t.ty, c);
+  if (t.tx == 0) store8(p.row_smooth(bh) + 8 * t.ty, c);
 #pragma unroll
   for (int a = 0; a < 8; a++) {
     const float inv_c = 1.0f / c[a];
@@ -244,11 +243,16 @@ __device__ __forceinline__ void quantize_tile(const Params &p, const BoundarySme
       for (int b = 0; b < 8; b++) amax[b] = fmaxf(amax[b], x[b]);
     }
   }
-  if (t.ty == 0) store8(p.col_scale + bh * D + 8 * t.tx, amax);
+  if (t.ty == 0) {                                            // stored as the step of the code, B_j / 127
+    float step[8];
+#pragma unroll
+    for (int b = 0; b < 8; b++) step[b] = amax[b] / 127.0f;
+    store8(p.col_scale(bh) + 8 * t.tx, step);
+  }
   float inv[8];
 #pragma unroll
   for (int b = 0; b < 8; b++) inv[b] = amax[b] > 0.0f ? 127.0f / amax[b] : 0.0f;
-  int8_t *ZT = p.codes + bh * (size_t)(D * D);
+  int8_t *ZT = p.codes(bh);
 #pragma unroll
   for (int b = 0; b < 8; b++) {
     uint32_t w2[2] = {0u, 0u};

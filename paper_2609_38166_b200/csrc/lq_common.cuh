@@ -21,18 +21,38 @@ constexpr int MAX_W = 64;
 constexpr int MAX_R = 16;
 constexpr unsigned FULL = 0xffffffffu;
 
+// Byte offsets inside a head block and float offsets inside a record row (d_k = d_v = 128).
+constexpr int HB_CODES = 0;
+constexpr int HB_COL_SCALE = D * D;
+constexpr int HB_ROW_SMOOTH = HB_COL_SCALE + 4 * D;
+constexpr int HB_COMP_K = HB_ROW_SMOOTH + 4 * D;
+__host__ __device__ constexpr int hb_comp_u(int r) { return HB_COMP_K + 2 * D * r; }
+__host__ __device__ constexpr int head_bytes(int r) { return HB_COMP_K + 4 * D * r; }
+__host__ __device__ constexpr int record_floats(bool diag) { return diag ? 3 * D : 2 * D; }
+constexpr int REC_KT = 0, REC_U = D, REC_A = 2 * D;
+
 // Launch-time description of one call, passed to the kernels by value.
 struct Params {
   int batch, heads_v, heads_qk, W, r, n_iter, smooth, force;
-  int8_t *codes;
-  float *col_scale, *row_smooth;
-  uint16_t *comp_k, *comp_u;
-  float *buf_k, *buf_u, *buf_a;
+  uint8_t *heads;    // [B*Hv] head blocks of head_bytes(r)
+  float *records;    // [B*Hv][W] record rows of record_floats(gate)
+  float *decays;     // scalar gate: [B*Hv][W]
   int32_t *win_pos;
   const uint16_t *q, *k, *v, *beta, *alpha;
   float *o;
   float *S;          // dense fp32 states (quantize / dequantize / fp32 baseline)
   uint16_t *S16;     // dense bf16 states (bf16 baseline)
+
+  __device__ __forceinline__ uint8_t *head(size_t bh) const { return heads + bh * (size_t)head_bytes(r); }
+  __device__ __forceinline__ int8_t *codes(size_t bh) const { return reinterpret_cast<int8_t *>(head(bh) + HB_CODES); }
+  __device__ __forceinline__ float *col_scale(size_t bh) const { return reinterpret_cast<float *>(head(bh) + HB_COL_SCALE); }
+  __device__ __forceinline__ float *row_smooth(size_t bh) const { return reinterpret_cast<float *>(head(bh) + HB_ROW_SMOOTH); }
+  __device__ __forceinline__ uint16_t *comp_k(size_t bh) const { return reinterpret_cast<uint16_t *>(head(bh) + HB_COMP_K); }
+  __device__ __forceinline__ uint16_t *comp_u(size_t bh) const { return reinterpret_cast<uint16_t *>(head(bh) + hb_comp_u(r)); }
+  // row of record j of head bh; `diag` selects the row length
+  __device__ __forceinline__ float *record(size_t bh, int j, bool diag) const {
+    return records + (bh * W + j) * (size_t)record_floats(diag);
+  }
 };
 
 __device__ __forceinline__ float bf16_bits(uint16_t h) { return __uint_as_float(static_cast<uint32_t>(h) << 16); }

@@ -1,15 +1,23 @@
-// Decode: one token for one (sequence, value head), done by ONE WARP.
+// Decode: one token for one (sequence, value head), done by a CTA of two warps with different roles.
 //
 // Eq. 10 (readout of the smoothed, compensated window representation) evaluated for x = alpha.k and
 // x = alpha.q in one pass over the 8-bit codes:
 //   S_{l-1}^T (alpha.x) = (B/127) Z^T (C Gamma_{1:l} x) + Uc (Kc^T Gamma_{1:l} x) + sum_j u_j (kt_j^T Gamma_{j+1:l} x)
 // then u = v - S_{l-1}^T(alpha.k) (Eq. 3), o = S_{l-1}^T(alpha.q) + u (kt^T q), and the record is appended.
 //
-// Data movement: everything a head needs (16 KiB of codes, the two scale vectors, the compensators and the
-// n buffered records) is brought into the warp's own shared-memory slot by TMA bulk copies that complete on
-// an mbarrier; the warp loads the token's vectors meanwhile, waits once, and computes out of shared memory.
-// A warp therefore keeps a whole head (about 27 KB at W = 16) in flight, and nothing in the kernel needs a
-// CTA-wide barrier: warps are independent workers that walk over the heads with a grid stride.
+// Data movement: a head's block (16 KiB of codes, the two scale vectors, the compensators: 19 KiB) and
+// its n buffered record rows are each contiguous in memory and are brought into the CTA's shared-memory slot
+// by TWO TMA bulk copies that complete on an mbarrier: a few large bulk requests keep the memory system busy
+// where thousands of 16-byte loads could not (plain loads are limited per warp), and about 64 KB in flight
+// per SM saturate HBM.  The slot is small enough for six CTAs per SM.  CTAs are persistent and walk over
+// the heads with a grid stride.  No load sits on a head's critical path (with the memory system kept full a
+// load takes several microseconds to return): the token's vectors are fetched two heads ahead into
+// registers, the per-head scalars (window position, beta, scalar alpha) for 32 heads at a time, one per lane.
+//
+// Roles: the STREAM warp turns C Gamma x into fixed-point digits, runs the tensor-core pass over the codes
+// and finishes u and o; the DOT warp meanwhile takes the projections onto the buffered records and the
+// compensators, appends the new record and, once the stream warp is done with the slot, requests the next
+// head.  They meet at two named barriers per head.
 //
 // Arithmetic: the first term is a dense int8 contraction, Z^T [128 x 128] against the two vectors.  The
 // vectors are put on a 30-bit block fixed-point grid and split into four signed base-256 digits each, which
@@ -26,25 +34,34 @@ namespace lq {
 // Set when a bounded wait gave up (bit 0: a decode warp's wait for its bulk copies).  Never cleared by kernels.
 __device__ int g_device_error = 0;
 
-// ---- per-warp shared-memory slot ----
+// Phase timing (development aid, compiled in with -DLQ_TIMING only): clock cycles per phase of the decode
+// warps, summed over all heads by lane 0 of each warp (slots 0..15: stream warp, 16..31: dot warp).
+#ifdef LQ_TIMING
+__device__ unsigned long long g_phase_cycles[32];
+#define LQ_TICK(slot)                                                                               \
+  do {                                                                                              \
+    const long long now_ = clock64();                                                               \
+    if (lane == 0) atomicAdd(&g_phase_cycles[16 * role + (slot)], (unsigned long long)(now_ - tick_)); \
+    tick_ = now_;                                                                                   \
+  } while (0)
+#else
+#define LQ_TICK(slot) do { } while (0)
+#endif
+
+// ---- shared-memory slot of one CTA ----
 struct DecodeSlot {
-  // byte offsets inside a slot; every region starts on a 16-byte boundary
-  int zt, cs, bs, ck, cu, bk, bu, ba, digits, y, pk, pq, gs, mbar, bytes;
+  // byte offsets inside the slot; every region starts on a 16-byte boundary
+  int head, rec, bas, digits, y, pk, pq, mbar, bytes;
   __host__ __device__ DecodeSlot(int W, int r, bool diag) {
+    const int rows = W > 1 ? W - 1 : 1;   // a window holds at most W-1 records when a token arrives
     int o = 0;
-    zt = o; o += D * D;                 // codes, Z^T
-    cs = o; o += 4 * D;                 // row_smooth
-    bs = o; o += 4 * D;                 // col_scale
-    ck = o; o += 2 * D * r;             // compensator keys, fp16
-    cu = o; o += 2 * D * r;             // compensator values, fp16
-    bk = o; o += 4 * D * W;             // buffered write keys
-    bu = o; o += 4 * D * W;             // buffered corrections
-    ba = o; o += diag ? 4 * D * W : 0;  // buffered diagonal decays, turned in place into Gamma_{j+1:l}
-    digits = o; o += 8 * D;             // digit planes: plane 4v+d = digit d of vector v (0: k, 1: q)
-    y = o; o += 2 * 4 * D;              // exact integer sums of the state stream, rounded to fp32: [2][128]
-    pk = o; o += 4 * (MAX_W + MAX_R + 16);
-    pq = o; o += 4 * (MAX_W + MAX_R + 16);   // projections; pq[n+r] holds kt^T q
-    gs = o; o += 4 * MAX_W;             // scalar-gate decays Gamma_{j+1:l}
+    head = o; o += head_bytes(r);          // the head block: codes | col_scale | row_smooth | comp_k | comp_u
+    rec = o; o += 4 * record_floats(diag) * rows;   // buffered record rows
+    bas = o; o += diag ? 0 : 2 * 4 * MAX_W;         // scalar gate: the records' decays, one copy per warp
+    digits = o; o += 8 * D;               // digit planes: plane 4v+d = digit d of vector v (0: k, 1: q)
+    y = o; o += 2 * 4 * D;                // exact integer sums of the state stream, rounded to fp32: [2][128]
+    pk = o; o += (4 * (W + r + 1) + 15) / 16 * 16;
+    pq = o; o += (4 * (W + r + 1) + 15) / 16 * 16;   // projections; pq[n+r] holds kt^T q
     mbar = o; o += 16;
     bytes = (o + 127) / 128 * 128;
   }
@@ -114,265 +131,435 @@ __device__ __forceinline__ void widen8_f16(const uint4 w, float (&x)[8]) {
   }
 }
 
-// Persistent kernel of one-warp CTAs: warp `gw` of the grid takes heads gw, gw + nwarps, ...
+// sums of four values over sixteen neighbouring lanes each, the four shuffle chains interleaved
+__device__ __forceinline__ void tree16x4(float (&x)[4]) {
+#pragma unroll
+  for (int s = 1; s <= 8; s <<= 1) {
+#pragma unroll
+    for (int v = 0; v < 4; v++) x[v] = x[v] + __shfl_xor_sync(FULL, x[v], s);
+  }
+}
+
+// Named barriers of the CTA (64 threads each): one side arrives, the other waits.
+//   1: dot warp -> stream warp, "the projections are in shared memory"
+//   2: stream warp -> dot warp, "the slot may be overwritten"
+__device__ __forceinline__ void named_arrive(int id) {
+  __threadfence_block();
+  asm volatile("bar.arrive %0, 64;\n" ::"r"(id) : "memory");
+}
+__device__ __forceinline__ void named_wait(int id) { asm volatile("bar.sync %0, 64;\n" ::"r"(id) : "memory"); }
+
+// The token's vectors as raw bf16 bits, loaded two heads ahead: lane c (and its twin c+16) owns key
+// channels 8c..8c+7, lane l value channels 4l..4l+3.
+struct TokenRaw {
+  uint4 k, q, a;        // a: diagonal-gate alpha
+  uint2 v;
+  float ba_lo, ba_hi;   // scalar gate: decays of buffered records `lane` and `lane + 32` (stale beyond n)
+};
+
 template <int GATE>
-__global__ void __launch_bounds__(32) decode_kernel(const Params p) {
-  extern __shared__ __align__(128) unsigned char lq_smem_raw[];
+__device__ __forceinline__ void load_token(const Params &p, size_t bh, int lane, int role, TokenRaw &tk) {
+  const int b = static_cast<int>(bh / p.heads_v), hv = static_cast<int>(bh % p.heads_v), c = lane & 15;
+  const size_t qk_off = ((size_t)b * p.heads_qk + hv / (p.heads_v / p.heads_qk)) * D;
+  tk.k = *reinterpret_cast<const uint4 *>(p.k + qk_off + 8 * c);
+  tk.q = *reinterpret_cast<const uint4 *>(p.q + qk_off + 8 * c);
+  if (role == 0) tk.v = *reinterpret_cast<const uint2 *>(p.v + bh * D + 4 * lane);
+  if (GATE == LQ_GATE_DIAG) {
+    tk.a = *reinterpret_cast<const uint4 *>(p.alpha + bh * D + 8 * c);
+  } else {
+    if (lane < p.W) tk.ba_lo = p.decays[bh * (size_t)p.W + lane];
+    if (lane + 32 < p.W) tk.ba_hi = p.decays[bh * (size_t)p.W + lane + 32];
+  }
+}
+
+// Persistent kernel of two-warp CTAs: CTA `blockIdx.x` takes heads blockIdx.x, blockIdx.x + gridDim.x, ...
+template <int GATE>
+__global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
+  extern __shared__ __align__(128) unsigned char slot[];
+  constexpr bool DIAG = GATE == LQ_GATE_DIAG;
+  constexpr int RF = record_floats(DIAG);
   const int W = p.W, r = p.r;
-  const DecodeSlot L(W, r, GATE == LQ_GATE_DIAG);
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const DecodeSlot L(W, r, DIAG);
+  const int lane = threadIdx.x & 31, role = threadIdx.x >> 5;      // role 0: stream warp, role 1: dot warp
   const int c = lane & 15, half = lane >> 4, g = lane >> 2, t = lane & 3;
-  unsigned char *slot = lq_smem_raw + (size_t)warp * L.bytes;
-  const int8_t *zt = reinterpret_cast<const int8_t *>(slot + L.zt);
-  const float *cs = reinterpret_cast<const float *>(slot + L.cs), *bs = reinterpret_cast<const float *>(slot + L.bs);
-  const uint16_t *ckh = reinterpret_cast<const uint16_t *>(slot + L.ck), *cuh = reinterpret_cast<const uint16_t *>(slot + L.cu);
-  const float *bk = reinterpret_cast<const float *>(slot + L.bk), *bu = reinterpret_cast<const float *>(slot + L.bu);
-  float *ba = reinterpret_cast<float *>(slot + L.ba);
+  const int8_t *zt = reinterpret_cast<const int8_t *>(slot + L.head + HB_CODES);
+  const float *bs = reinterpret_cast<const float *>(slot + L.head + HB_COL_SCALE);
+  const float *cs = reinterpret_cast<const float *>(slot + L.head + HB_ROW_SMOOTH);
+  const uint16_t *ckh = reinterpret_cast<const uint16_t *>(slot + L.head + HB_COMP_K);
+  const uint16_t *cuh = reinterpret_cast<const uint16_t *>(slot + L.head + hb_comp_u(r));
+  const float *rec = reinterpret_cast<const float *>(slot + L.rec);     // rows of RF floats: kt | u | (alpha)
+  float *bas = reinterpret_cast<float *>(slot + L.bas) + role * MAX_W;   // this warp's copy of the decays
   int8_t *digits = reinterpret_cast<int8_t *>(slot + L.digits);
   float *y = reinterpret_cast<float *>(slot + L.y), *pk = reinterpret_cast<float *>(slot + L.pk);
-  float *pq = reinterpret_cast<float *>(slot + L.pq), *gs = reinterpret_cast<float *>(slot + L.gs);
+  float *pq = reinterpret_cast<float *>(slot + L.pq);
   const uint32_t bar = smem_addr(slot + L.mbar), slot_a = smem_addr(slot);
 
-  if (lane == 0) mbar_init(bar, 1);
-  __syncwarp();
+  if (threadIdx.x == 0) mbar_init(bar, 1);
+  __syncthreads();
   uint32_t parity = 0;
+  const size_t nh = (size_t)p.batch * p.heads_v, G = gridDim.x;
 
-  const size_t nh = (size_t)p.batch * p.heads_v;
-  const size_t nwarps = (size_t)gridDim.x * (blockDim.x >> 5);
-  const int group = p.heads_v / p.heads_qk;
-
-  for (size_t bh = (size_t)blockIdx.x * (blockDim.x >> 5) + warp; bh < nh; bh += nwarps) {
-    const int b = static_cast<int>(bh / p.heads_v), hv = static_cast<int>(bh % p.heads_v);
-    const int n = p.win_pos[b] & 0xFFFF;     // bits 16.. are the arrival counter of this launch
-    if (n >= W) continue;                    // nothing can be appended: the sequence gets no token
-
-    // (1) request the head: bulk copies into the slot, completion counted in bytes on the mbarrier
+  // Requests head bh (n records buffered) into the slot: two bulk copies, issued by two lanes of the dot
+  // warp when nobody reads the slot any more.
+  auto request = [&](size_t bh, int n) {
+    // the slot was last touched through ordinary loads and stores; order them before the async writes
+    asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+    const uint32_t hb = head_bytes(r), rb = 4u * RF * n;
     if (lane == 0) {
-      // the slot was last touched through ordinary loads and stores; order them before the async writes
-      asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
-      const uint32_t rec = 4u * D * n;
-      uint32_t total = D * D + 8u * D + 4u * D * r + 2u * rec + (GATE == LQ_GATE_DIAG ? rec : 0u);
-      mbar_expect_tx(bar, total);
-      bulk_g2s(slot_a + L.zt, p.codes + bh * (size_t)(D * D), D * D, bar);
-      bulk_g2s(slot_a + L.cs, p.row_smooth + bh * D, 4 * D, bar);
-      bulk_g2s(slot_a + L.bs, p.col_scale + bh * D, 4 * D, bar);
-      if (r > 0) {
-        bulk_g2s(slot_a + L.ck, p.comp_k + bh * (size_t)(r * D), 2 * D * r, bar);
-        bulk_g2s(slot_a + L.cu, p.comp_u + bh * (size_t)(r * D), 2 * D * r, bar);
-      }
-      if (n > 0) {
-        bulk_g2s(slot_a + L.bk, p.buf_k + bh * (size_t)(W * D), rec, bar);
-        bulk_g2s(slot_a + L.bu, p.buf_u + bh * (size_t)(W * D), rec, bar);
-        if (GATE == LQ_GATE_DIAG) bulk_g2s(slot_a + L.ba, p.buf_a + bh * (size_t)(W * D), rec, bar);
-      }
+      mbar_expect_tx(bar, hb + rb);
+      bulk_g2s(slot_a + L.head, p.head(bh), hb, bar);
+    }
+    if (lane == 1 && n > 0) bulk_g2s(slot_a + L.rec, p.record(bh, 0, DIAG), rb, bar);
+  };
+
+  // Per-head scalars of this CTA's heads, 32 heads at a time: lane l holds those of the CTA's (32*batch+l)-th head
+  int sc_n = 0;
+  uint32_t sc_beta = 0, sc_alpha = 0;
+  auto load_scalars = [&](size_t first_bh) {
+    const size_t bh = first_bh + (size_t)lane * G;
+    if (bh < nh) {
+      sc_n = p.win_pos[bh / p.heads_v];     // bits 16.. are the arrival counter of this launch: masked at use
+      sc_beta = p.beta[bh];
+      if (!DIAG) sc_alpha = p.alpha[bh];
+    }
+  };
+
+  // Arrival on win_pos (see arrive_and_set) is split: the atomic is issued when a head is done, its return
+  // value is looked at one head later, so that the warp does not sit out the round trip.
+  int pend_old = 0, pend_b = -1, pend_new = 0;
+  auto settle = [&]() {
+    if (pend_b >= 0 && (pend_old >> 16) == p.heads_v - 1) p.win_pos[pend_b] = pend_new;
+    pend_b = -1;
+  };
+
+  // A head whose window is already full (n >= W) gets no token: it is neither requested nor waited for.
+  load_scalars(blockIdx.x);
+  TokenRaw tok0, tok1, tok2;                  // this head's token, the next head's, the one after
+  tok0.ba_lo = tok0.ba_hi = tok1.ba_lo = tok1.ba_hi = tok2.ba_lo = tok2.ba_hi = 1.0f;
+  if (blockIdx.x < nh) load_token<GATE>(p, blockIdx.x, lane, role, tok0);
+  if (blockIdx.x + G < nh) load_token<GATE>(p, blockIdx.x + G, lane, role, tok1);
+  {
+    const int n0 = __shfl_sync(FULL, sc_n, 0) & 0xFFFF;
+    if (role == 1 && blockIdx.x < nh && n0 < W) request(blockIdx.x, n0);
+  }
+#ifdef LQ_TIMING
+  long long tick_ = clock64();
+#endif
+  int idx = 0;                               // position of the head in this CTA's list
+  for (size_t bh = blockIdx.x; bh < nh; bh += G, idx++) {
+    const int n = __shfl_sync(FULL, sc_n, idx & 31) & 0xFFFF;
+    const float beta = __uint_as_float(__shfl_sync(FULL, sc_beta, idx & 31) << 16);
+    const float alpha_s = __uint_as_float(__shfl_sync(FULL, sc_alpha, idx & 31) << 16);
+    // the next head's scalars: from the next batch when this head is the last of its batch
+    const size_t bh_next = bh + G;
+    if ((idx & 31) == 31) load_scalars(bh_next);
+    const int n_next = bh_next < nh ? (__shfl_sync(FULL, sc_n, (idx + 1) & 31) & 0xFFFF) : W;
+    const bool active = n < W, next_active = n_next < W;
+    const int b = static_cast<int>(bh / p.heads_v);
+    if (bh + 2 * G < nh) load_token<GATE>(p, bh + 2 * G, lane, role, tok2);   // used two trips from now
+    const TokenRaw cur = tok0;
+    tok0 = tok1;
+    tok1 = tok2;
+    LQ_TICK(0);
+
+    if (!active) {                           // nothing was requested for this head; keep the pipeline going
+      if (role == 1 && next_active) request(bh_next, n_next);
+      continue;
     }
 
-    // (2) the token, straight into registers.  Lane c (and its twin c+16) owns key channels 8c..8c+7;
-    // lane l owns value channels 4l..4l+3.
-    float k8[8], q8[8], kt8[8], a8[8], v4[4];
-    {
-      const size_t qk_off = ((size_t)b * p.heads_qk + hv / group) * D;
-      widen8_bf16(*reinterpret_cast<const uint4 *>(p.k + qk_off + 8 * c), k8);
-      widen8_bf16(*reinterpret_cast<const uint4 *>(p.q + qk_off + 8 * c), q8);
-      const uint2 vw = *reinterpret_cast<const uint2 *>(p.v + bh * D + 4 * lane);
-      v4[0] = __uint_as_float(vw.x << 16); v4[1] = __uint_as_float(vw.x & 0xFFFF0000u);
-      v4[2] = __uint_as_float(vw.y << 16); v4[3] = __uint_as_float(vw.y & 0xFFFF0000u);
-      const float beta = bf16_bits(p.beta[bh]);
-      if (GATE == LQ_GATE_DIAG) {
-        widen8_bf16(*reinterpret_cast<const uint4 *>(p.alpha + bh * D + 8 * c), a8);
-      } else {
-        const float a = bf16_bits(p.alpha[bh]);
+    // ---- this head's token ----
+    float k8[8], q8[8], a8[8];
+    widen8_bf16(cur.k, k8);
+    widen8_bf16(cur.q, q8);
+    if (DIAG) {
+      widen8_bf16(cur.a, a8);
+    } else {
 #pragma unroll
-        for (int e = 0; e < 8; e++) a8[e] = a;
-      }
-#pragma unroll
-      for (int e = 0; e < 8; e++) kt8[e] = beta * k8[e];
+      for (int e = 0; e < 8; e++) a8[e] = alpha_s;
+      bas[lane] = cur.ba_lo;
+      bas[lane + 32] = cur.ba_hi;
     }
-    float ba_lo = 1.0f, ba_hi = 1.0f;        // scalar gate: decay of record `lane` and of record `lane + 32`
-    if (GATE == LQ_GATE_SCALAR) {
-      if (lane < n) ba_lo = p.buf_a[bh * (size_t)W + lane];
-      if (lane + 32 < n) ba_hi = p.buf_a[bh * (size_t)W + lane + 32];
-    }
+    LQ_TICK(1);
 
-    // (3) wait for the slot (bounded: a copy that never lands must not hang the GPU)
+    // ---- wait for the slot (bounded: a copy that never lands must not hang the GPU) ----
     if (!mbar_wait(bar, parity)) {
-      if (lane == 0) atomicOr(&g_device_error, 1);
+      if (lane == 0) { atomicOr(&g_device_error, 1); settle(); }
       mbar_wait(bar, parity);                // one more bounded wait for the copies in flight, then give up
       return;
     }
     parity ^= 1u;
+    __syncwarp();
+    LQ_TICK(2);
 
-    // (4) cumulative decays from the newest record back (Appendix B.2).  After the loop g8 = Gamma_{1:l}.
-    float g8[8];
+    if (role == 1) {
+      // =========================== DOT WARP ===========================
+      // Projections.  A dot product of 128 terms is taken by sixteen lanes (lane c owns block c of eight
+      // terms); the two halves of the warp work on different vectors, two per half and trip, so that four
+      // shuffle trees overlap.  Both halves make the same number of trips (the shuffles name all 32 lanes);
+      // an index outside the range recomputes a valid item and is not stored.
+      // Records are walked from the newest back, with g8 = Gamma_{j+1:l} kept up on the way (Appendix B.2).
+      float g8[8], kt8[8];
 #pragma unroll
-    for (int e = 0; e < 8; e++) g8[e] = a8[e];
-    if (GATE == LQ_GATE_DIAG) {
-      for (int j = n - 1; j >= 0; j--) {
-        float aj[8];
-        load8(ba + j * D + 8 * c, aj);
-        __syncwarp();                        // both twins have read the decay before one of them replaces it
-        if (half == 0) store8(ba + j * D + 8 * c, g8);   // Gamma_{j+1:l} in place of the record's decay
+      for (int e = 0; e < 8; e++) { g8[e] = a8[e]; kt8[e] = beta * k8[e]; }
+      for (int jt = n - 1; jt >= 0; jt -= 4) {       // records jt, jt-1, jt-2, jt-3
+        float s4[4];
+        int jo[2];
 #pragma unroll
-        for (int e = 0; e < 8; e++) g8[e] = g8[e] * aj[e];
-      }
-    } else {
-      float gsc = a8[0];
-      for (int j = n - 1; j >= 0; j--) {     // every lane runs the same scalar chain
-        if (lane == (j & 31)) gs[j] = gsc;
-        gsc = gsc * __shfl_sync(FULL, j < 32 ? ba_lo : ba_hi, j & 31);
-      }
-#pragma unroll
-      for (int e = 0; e < 8; e++) g8[e] = gsc;
-    }
-    float gk8[8], gq8[8];
-#pragma unroll
-    for (int e = 0; e < 8; e++) { gk8[e] = g8[e] * k8[e]; gq8[e] = g8[e] * q8[e]; }
-
-    // (4b) C Gamma k (lanes 0..15) and C Gamma q (lanes 16..31) on their fixed-point grids, as digit planes
-    float back_own;
-    {
-      float c8[8], x8[8];
-      load8(cs + 8 * c, c8);
-      float m = 0.0f;
-#pragma unroll
-      for (int e = 0; e < 8; e++) {
-        x8[e] = c8[e] * (half ? gq8[e] : gk8[e]);
-        m = fmaxf(m, fabsf(x8[e]));
-      }
-#pragma unroll
-      for (int s = 1; s <= 8; s <<= 1) m = fmaxf(m, __shfl_xor_sync(FULL, m, s));
-      float scale;
-      fixed_point_scales(m, scale, back_own);
-      uint32_t lo[4] = {0u, 0u, 0u, 0u}, hi[4] = {0u, 0u, 0u, 0u};      // [digit]: bytes of elements 0..3 / 4..7
-#pragma unroll
-      for (int e = 0; e < 8; e++) {
-        int X = __float2int_rn(x8[e] * scale);
-#pragma unroll
-        for (int d = 0; d < 4; d++) {       // X = d0 + 256 d1 + 65536 d2 + 2^24 d3, digits in [-128, 127]
-          const int dig = (X << 24) >> 24;
-          const uint32_t byte = static_cast<uint32_t>(dig) & 0xFFu;
-          if (e < 4) lo[d] |= byte << (8 * e); else hi[d] |= byte << (8 * (e - 4));
-          X = (X - dig) >> 8;
-        }
-      }
-#pragma unroll
-      for (int d = 0; d < 4; d++)
-        *reinterpret_cast<uint2 *>(digits + (4 * half + d) * D + 8 * c) = make_uint2(lo[d], hi[d]);
-    }
-    const float back_other = __shfl_xor_sync(FULL, back_own, 16);
-    const float back_k = half ? back_other : back_own, back_q = half ? back_own : back_other;
-    __syncwarp();                            // in-place decays, gs and digit planes are visible to the warp
-
-    // (5) projections: the two halves of the warp take one dot-product pair each per trip (lane c owns block
-    // c of eight terms).  Both halves make the same number of trips: the shuffles name all 32 lanes.
-    {
-      const int total = n + r + 1;
-      for (int jb = 0; jb < total; jb += 2) {
-        const int jown = jb + half;
-        const int j = jown < total ? jown : total - 1;
-        float x8[8], yk8[8], yq8[8];
-        if (j < n) {
-          load8(bk + j * D + 8 * c, x8);
-          if (GATE == LQ_GATE_DIAG) {
-            float gj8[8];
-            load8(ba + j * D + 8 * c, gj8);
-#pragma unroll
-            for (int e = 0; e < 8; e++) { yk8[e] = gj8[e] * k8[e]; yq8[e] = gj8[e] * q8[e]; }
+        for (int u = 0; u < 2; u++) {
+          // the decays of the two records of this pair; the half that owns the older one steps over the newer
+          float gmine[8];
+          const int jn = jt - 2 * u, jold = jn - 1;  // newer, older
+          float an[8], ao[8];
+          if (DIAG) {
+            load8(rec + (jn > 0 ? jn : 0) * RF + REC_A + 8 * c, an);
+            load8(rec + (jold > 0 ? jold : 0) * RF + REC_A + 8 * c, ao);
           } else {
-            const float gj = gs[j];
+            const float x = bas[jn > 0 ? jn : 0], z = bas[jold > 0 ? jold : 0];
 #pragma unroll
-            for (int e = 0; e < 8; e++) { yk8[e] = gj * k8[e]; yq8[e] = gj * q8[e]; }
+            for (int e = 0; e < 8; e++) { an[e] = x; ao[e] = z; }
           }
-        } else if (j < n + r) {
-          widen8_f16(*reinterpret_cast<const uint4 *>(ckh + (j - n) * D + 8 * c), x8);
 #pragma unroll
-          for (int e = 0; e < 8; e++) { yk8[e] = gk8[e]; yq8[e] = gq8[e]; }
-        } else {                             // kt^T q, kept in the pq slot; the pk slot is unused
+          for (int e = 0; e < 8; e++) {
+            const float gn = g8[e], go = gn * an[e];      // Gamma_{jn+1:l}, Gamma_{jold+1:l}
+            gmine[e] = half ? go : gn;
+            g8[e] = go * ao[e];                           // past both records
+          }
+          jo[u] = jn - half;
+          const int j = jo[u] >= 0 ? jo[u] : 0;
+          float x8[8];
+          load8(rec + j * RF + REC_KT + 8 * c, x8);
+          float sk = x8[0] * (gmine[0] * k8[0]), sq = x8[0] * (gmine[0] * q8[0]);
 #pragma unroll
-          for (int e = 0; e < 8; e++) { x8[e] = kt8[e]; yk8[e] = q8[e]; yq8[e] = q8[e]; }
+          for (int e = 1; e < 8; e++) {
+            sk = fmaf(x8[e], gmine[e] * k8[e], sk);
+            sq = fmaf(x8[e], gmine[e] * q8[e], sq);
+          }
+          s4[2 * u] = sk; s4[2 * u + 1] = sq;
         }
-        float sk = x8[0] * yk8[0], sq = x8[0] * yq8[0];
+        tree16x4(s4);
 #pragma unroll
-        for (int e = 1; e < 8; e++) { sk = fmaf(x8[e], yk8[e], sk); sq = fmaf(x8[e], yq8[e], sq); }
-        sk = tree16(sk);
-        sq = tree16(sq);
-        if (c == 0 && jown < total) { pk[j] = sk; pq[j] = sq; }
+        for (int u = 0; u < 2; u++)
+          if (c == 0 && jo[u] >= 0) { pk[jo[u]] = s4[2 * u]; pq[jo[u]] = s4[2 * u + 1]; }
       }
-    }
-
-    // (6) the state stream on the tensor cores: eight 16-row tiles of Z^T, K = 128 as four k-blocks.
-    // A thread's 16 bytes of a row hold key channels 64p+16t..64p+16t+15 and serve two k-blocks; the digit
-    // planes are read with the same permutation of the key index.
-    {
-      uint4 bf[2];
+      LQ_TICK(3);
+      // Compensator keys against Gamma_{1:l} k and Gamma_{1:l} q; item r is kt^T q (kept in pq[n+r]).
+      // g8 may have run past record 0 above: Gamma_{1:l} is rebuilt from the exact chain.
+      {
+        float gam[8];
 #pragma unroll
-      for (int pp = 0; pp < 2; pp++) bf[pp] = *reinterpret_cast<const uint4 *>(digits + g * D + 64 * pp + 16 * t);
+        for (int e = 0; e < 8; e++) gam[e] = a8[e];
+        for (int j = n - 1; j >= 0; j--) {
+          float aj[8];
+          if (DIAG) load8(rec + j * RF + REC_A + 8 * c, aj);
+          else {
+            const float x = bas[j];
+#pragma unroll
+            for (int e = 0; e < 8; e++) aj[e] = x;
+          }
+#pragma unroll
+          for (int e = 0; e < 8; e++) gam[e] = gam[e] * aj[e];
+        }
+        float gk8[8], gq8[8];
+#pragma unroll
+        for (int e = 0; e < 8; e++) { gk8[e] = gam[e] * k8[e]; gq8[e] = gam[e] * q8[e]; }
+        for (int hb = 0; hb < r + 1; hb += 4) {
+          float s4[4];
+          int ho[2];
+#pragma unroll
+          for (int u = 0; u < 2; u++) {
+            ho[u] = hb + 2 * u + half;
+            const int h = ho[u] < r ? ho[u] : (r > 0 ? r - 1 : 0);
+            float x8[8];
+            if (r > 0) widen8_f16(*reinterpret_cast<const uint4 *>(ckh + h * D + 8 * c), x8);
+            const bool is_ktq = ho[u] >= r;
+            float sk, sq;
+            {
+              const float x0 = is_ktq ? kt8[0] : x8[0];
+              sk = x0 * (is_ktq ? q8[0] : gk8[0]);
+              sq = x0 * (is_ktq ? q8[0] : gq8[0]);
+            }
+#pragma unroll
+            for (int e = 1; e < 8; e++) {
+              const float xe = is_ktq ? kt8[e] : x8[e];
+              sk = fmaf(xe, is_ktq ? q8[e] : gk8[e], sk);
+              sq = fmaf(xe, is_ktq ? q8[e] : gq8[e], sq);
+            }
+            s4[2 * u] = sk; s4[2 * u + 1] = sq;
+          }
+          tree16x4(s4);
+#pragma unroll
+          for (int u = 0; u < 2; u++)
+            if (c == 0 && ho[u] <= r) { pk[n + ho[u]] = s4[2 * u]; pq[n + ho[u]] = s4[2 * u + 1]; }
+        }
+      }
+      __syncwarp();
+      LQ_TICK(4);
+      named_arrive(1);                       // the projections are in shared memory
+      // append the key side of the record (and its decay)
+      {
+        float *row = p.record(bh, n, DIAG);
+        if (half == 0) {
+          store8(row + REC_KT + 8 * c, kt8);
+          if (DIAG) store8(row + REC_A + 8 * c, a8);
+          else if (lane == 0) p.decays[bh * (size_t)W + n] = a8[0];
+        }
+      }
+      LQ_TICK(5);
+      named_wait(2);                         // the stream warp has read all it needs from the slot
+      LQ_TICK(6);
+      if (next_active) request(bh_next, n_next);
+      LQ_TICK(7);
+    } else {
+      // =========================== STREAM WARP ===========================
+      // Gamma_{1:l}: the chain of decays from the newest record back (Appendix B.2)
+      float gam[8];
+#pragma unroll
+      for (int e = 0; e < 8; e++) gam[e] = a8[e];
+      if (DIAG) {
 #pragma unroll 2
-      for (int mt = 0; mt < 8; mt++) {
-        int c4[4] = {0, 0, 0, 0};
-        const int j = 16 * mt + g;
+        for (int j = n - 1; j >= 0; j--) {
+          float aj[8];
+          load8(rec + j * RF + REC_A + 8 * c, aj);
 #pragma unroll
-        for (int pp = 0; pp < 2; pp++) {
-          const uint4 zlo = *reinterpret_cast<const uint4 *>(zt + j * D + 64 * pp + 16 * t);
-          const uint4 zhi = *reinterpret_cast<const uint4 *>(zt + (j + 8) * D + 64 * pp + 16 * t);
-          mma_s8(c4, zlo.x, zhi.x, zlo.y, zhi.y, bf[pp].x, bf[pp].y);
-          mma_s8(c4, zlo.z, zhi.z, zlo.w, zhi.w, bf[pp].z, bf[pp].w);
+          for (int e = 0; e < 8; e++) gam[e] = gam[e] * aj[e];
         }
-        // c4[0], c4[1]: row g, planes 2t, 2t+1;  c4[2], c4[3]: row g+8.  Planes 4v..4v+3 are the digits of
-        // vector v: lanes t = 0, 1 carry the k sums and t = 2, 3 the q sums, even t the low digit pair.
-        long long lo = static_cast<long long>(c4[0]) + (static_cast<long long>(c4[1]) << 8);
-        long long hi = static_cast<long long>(c4[2]) + (static_cast<long long>(c4[3]) << 8);
-        if (t & 1) { lo <<= 16; hi <<= 16; }
-        lo += __shfl_xor_sync(FULL, lo, 1);
-        hi += __shfl_xor_sync(FULL, hi, 1);
-        if (!(t & 1)) {
-          float *dst = y + (t >> 1) * D;
-          dst[j] = __ll2float_rn(lo);
-          dst[j + 8] = __ll2float_rn(hi);
+      } else {
+        float gsc = a8[0];
+#pragma unroll 4
+        for (int j = n - 1; j >= 0; j--) gsc = gsc * bas[j];
+#pragma unroll
+        for (int e = 0; e < 8; e++) gam[e] = gsc;
+      }
+      LQ_TICK(3);
+      // C Gamma k (lanes 0..15) and C Gamma q (lanes 16..31) on their fixed-point grids, as digit planes
+      float back_own;
+      {
+        float c8[8], x8[8];
+        load8(cs + 8 * c, c8);
+        float m = 0.0f;
+#pragma unroll
+        for (int e = 0; e < 8; e++) {
+          x8[e] = c8[e] * (gam[e] * (half ? q8[e] : k8[e]));
+          m = fmaxf(m, fabsf(x8[e]));
+        }
+#pragma unroll
+        for (int s = 1; s <= 8; s <<= 1) m = fmaxf(m, __shfl_xor_sync(FULL, m, s));
+        float scale;
+        fixed_point_scales(m, scale, back_own);
+        // X = d0 + 256 d1 + 65536 d2 + 2^24 d3 with digits in [-128, 127]: the digit is the low byte read as
+        // signed, and taking it off is (X + 128) >> 8.  The bytes of the four stages of an element are the
+        // four digits; prmt gathers the same digit of four elements into one word.
+        uint32_t st[8][4];
+#pragma unroll
+        for (int e = 0; e < 8; e++) {
+          int X = __float2int_rn(x8[e] * scale);
+#pragma unroll
+          for (int d = 0; d < 4; d++) { st[e][d] = static_cast<uint32_t>(X); X = (X + 128) >> 8; }
+        }
+#pragma unroll
+        for (int d = 0; d < 4; d++) {
+          const uint32_t lo = __byte_perm(__byte_perm(st[0][d], st[1][d], 0x0040), __byte_perm(st[2][d], st[3][d], 0x0040), 0x5410);
+          const uint32_t hi = __byte_perm(__byte_perm(st[4][d], st[5][d], 0x0040), __byte_perm(st[6][d], st[7][d], 0x0040), 0x5410);
+          *reinterpret_cast<uint2 *>(digits + (4 * half + d) * D + 8 * c) = make_uint2(lo, hi);
         }
       }
-    }
-    __syncwarp();
+      const float back_other = __shfl_xor_sync(FULL, back_own, 16);
+      const float back_k = half ? back_other : back_own, back_q = half ? back_own : back_other;
+      __syncwarp();                          // the digit planes are visible to the warp
+      LQ_TICK(4);
 
-    // (7) per value channel (lane l: channels 4l..4l+3): scale the sums, add compensator and record terms
-    {
-      const float4 yk4 = *reinterpret_cast<const float4 *>(y + 4 * lane);
-      const float4 yq4 = *reinterpret_cast<const float4 *>(y + D + 4 * lane);
-      const float4 b4 = *reinterpret_cast<const float4 *>(bs + 4 * lane);
-      const float s4[4] = {b4.x / 127.0f, b4.y / 127.0f, b4.z / 127.0f, b4.w / 127.0f};
-      float rk[4] = {s4[0] * (yk4.x * back_k), s4[1] * (yk4.y * back_k), s4[2] * (yk4.z * back_k), s4[3] * (yk4.w * back_k)};
-      float rq[4] = {s4[0] * (yq4.x * back_q), s4[1] * (yq4.y * back_q), s4[2] * (yq4.z * back_q), s4[3] * (yq4.w * back_q)};
-      for (int h = 0; h < r; h++) {
-        const uint2 w = *reinterpret_cast<const uint2 *>(cuh + h * D + 4 * lane);
-        const float2 f01 = __half22float2(*reinterpret_cast<const __half2 *>(&w.x));
-        const float2 f23 = __half22float2(*reinterpret_cast<const __half2 *>(&w.y));
-        const float uc[4] = {f01.x, f01.y, f23.x, f23.y};
-        const float pkh = pk[n + h], pqh = pq[n + h];
+      // The state stream on the tensor cores: eight 16-row tiles of Z^T, K = 128 as four k-blocks.  A
+      // thread's 16 bytes of a row hold key channels 64p+16t..64p+16t+15 and serve two k-blocks; the digit
+      // planes are read with the same permutation of the key index.  The two 64-channel halves of a tile
+      // accumulate separately (exact integers: any split gives the same sum), which halves the dependent
+      // chain of MMAs.  Digit pairs are recombined in int32 (|sum| < 2^30), the two pairs in binary64, which
+      // holds the 47-bit total exactly, and one rounding takes it to fp32.
+      {
+        uint4 bf[2];
 #pragma unroll
-        for (int e = 0; e < 4; e++) { rk[e] = fmaf(uc[e], pkh, rk[e]); rq[e] = fmaf(uc[e], pqh, rq[e]); }
-      }
-      for (int jj = 0; jj < n; jj++) {
-        const float4 u4 = *reinterpret_cast<const float4 *>(bu + jj * D + 4 * lane);
-        const float uj[4] = {u4.x, u4.y, u4.z, u4.w};
-        const float pkj = pk[jj], pqj = pq[jj];
+        for (int pp = 0; pp < 2; pp++) bf[pp] = *reinterpret_cast<const uint4 *>(digits + g * D + 64 * pp + 16 * t);
 #pragma unroll
-        for (int e = 0; e < 4; e++) { rk[e] = fmaf(uj[e], pkj, rk[e]); rq[e] = fmaf(uj[e], pqj, rq[e]); }
+        for (int mt = 0; mt < 8; mt++) {
+          int ca[4] = {0, 0, 0, 0}, cb[4] = {0, 0, 0, 0};
+          const int j = 16 * mt + g;
+          {
+            const uint4 zlo = *reinterpret_cast<const uint4 *>(zt + j * D + 16 * t);
+            const uint4 zhi = *reinterpret_cast<const uint4 *>(zt + (j + 8) * D + 16 * t);
+            mma_s8(ca, zlo.x, zhi.x, zlo.y, zhi.y, bf[0].x, bf[0].y);
+            mma_s8(ca, zlo.z, zhi.z, zlo.w, zhi.w, bf[0].z, bf[0].w);
+          }
+          {
+            const uint4 zlo = *reinterpret_cast<const uint4 *>(zt + j * D + 64 + 16 * t);
+            const uint4 zhi = *reinterpret_cast<const uint4 *>(zt + (j + 8) * D + 64 + 16 * t);
+            mma_s8(cb, zlo.x, zhi.x, zlo.y, zhi.y, bf[1].x, bf[1].y);
+            mma_s8(cb, zlo.z, zhi.z, zlo.w, zhi.w, bf[1].z, bf[1].w);
+          }
+          // c[0], c[1]: row g, planes 2t, 2t+1;  c[2], c[3]: row g+8.  Planes 4v..4v+3 are the digits of
+          // vector v: lanes t = 0, 1 carry the k sums and t = 2, 3 the q sums, even t the low digit pair.
+          const int pair_g = (ca[0] + cb[0]) + ((ca[1] + cb[1]) << 8);
+          const int pair_g8 = (ca[2] + cb[2]) + ((ca[3] + cb[3]) << 8);
+          const int other_g = __shfl_xor_sync(FULL, pair_g, 1), other_g8 = __shfl_xor_sync(FULL, pair_g8, 1);
+          if (!(t & 1)) {                    // this lane has the low pair, its neighbour sent the high pair
+            float *dst = y + (t >> 1) * D;
+            dst[j] = __double2float_rn(fma(static_cast<double>(other_g), 65536.0, static_cast<double>(pair_g)));
+            dst[j + 8] = __double2float_rn(fma(static_cast<double>(other_g8), 65536.0, static_cast<double>(pair_g8)));
+          }
+        }
       }
-      const float ktq = pq[n + r];
-      float u[4], o[4];
+      __syncwarp();
+      LQ_TICK(5);
+
+      // Per value channel (lane l: channels 4l..4l+3): scale the sums, then add the compensator and record
+      // terms with the projections of the dot warp
+      {
+        const float4 yk4 = *reinterpret_cast<const float4 *>(y + 4 * lane);
+        const float4 yq4 = *reinterpret_cast<const float4 *>(y + D + 4 * lane);
+        const float4 s4 = *reinterpret_cast<const float4 *>(bs + 4 * lane);      // code steps B_j / 127
+        float rk[4] = {s4.x * (yk4.x * back_k), s4.y * (yk4.y * back_k), s4.z * (yk4.z * back_k), s4.w * (yk4.w * back_k)};
+        float rq[4] = {s4.x * (yq4.x * back_q), s4.y * (yq4.y * back_q), s4.z * (yq4.z * back_q), s4.w * (yq4.w * back_q)};
+        const float v4[4] = {__uint_as_float(cur.v.x << 16), __uint_as_float(cur.v.x & 0xFFFF0000u),
+                             __uint_as_float(cur.v.y << 16), __uint_as_float(cur.v.y & 0xFFFF0000u)};
+        LQ_TICK(6);
+        named_wait(1);                       // pk, pq are complete
+        LQ_TICK(7);
+#pragma unroll 2
+        for (int h = 0; h < r; h++) {
+          const uint2 w = *reinterpret_cast<const uint2 *>(cuh + h * D + 4 * lane);
+          const float2 f01 = __half22float2(*reinterpret_cast<const __half2 *>(&w.x));
+          const float2 f23 = __half22float2(*reinterpret_cast<const __half2 *>(&w.y));
+          const float uc[4] = {f01.x, f01.y, f23.x, f23.y};
+          const float pkh = pk[n + h], pqh = pq[n + h];
 #pragma unroll
-      for (int e = 0; e < 4; e++) { u[e] = v4[e] - rk[e]; o[e] = fmaf(u[e], ktq, rq[e]); }
-      *reinterpret_cast<float4 *>(p.o + bh * D + 4 * lane) = make_float4(o[0], o[1], o[2], o[3]);
-      *reinterpret_cast<float4 *>(p.buf_u + (bh * W + n) * (size_t)D + 4 * lane) = make_float4(u[0], u[1], u[2], u[3]);
-      if (half == 0) {
-        store8(p.buf_k + (bh * W + n) * (size_t)D + 8 * c, kt8);
-        if (GATE == LQ_GATE_DIAG) store8(p.buf_a + (bh * W + n) * (size_t)D + 8 * c, a8);
-        else if (lane == 0) p.buf_a[bh * W + n] = a8[0];
+          for (int e = 0; e < 4; e++) { rk[e] = fmaf(uc[e], pkh, rk[e]); rq[e] = fmaf(uc[e], pqh, rq[e]); }
+        }
+#pragma unroll 4
+        for (int jj = 0; jj < n; jj++) {
+          const float4 u4 = *reinterpret_cast<const float4 *>(rec + jj * RF + REC_U + 4 * lane);
+          const float uj[4] = {u4.x, u4.y, u4.z, u4.w};
+          const float pkj = pk[jj], pqj = pq[jj];
+#pragma unroll
+          for (int e = 0; e < 4; e++) { rk[e] = fmaf(uj[e], pkj, rk[e]); rq[e] = fmaf(uj[e], pqj, rq[e]); }
+        }
+        const float ktq = pq[n + r];
+        float u[4], o[4];
+#pragma unroll
+        for (int e = 0; e < 4; e++) { u[e] = v4[e] - rk[e]; o[e] = fmaf(u[e], ktq, rq[e]); }
+        __syncwarp();                        // every lane is done reading the slot
+        LQ_TICK(8);
+        named_arrive(2);
+        *reinterpret_cast<float4 *>(p.o + bh * D + 4 * lane) = make_float4(o[0], o[1], o[2], o[3]);
+        *reinterpret_cast<float4 *>(p.record(bh, n, DIAG) + REC_U + 4 * lane) = make_float4(u[0], u[1], u[2], u[3]);
       }
+      if (lane == 0) {
+        settle();
+        pend_old = atomicAdd(p.win_pos + b, 0x10000);
+        pend_b = b;
+        pend_new = n + 1;
+      }
+      LQ_TICK(9);
     }
-    __syncwarp();
-    if (lane == 0) arrive_and_set(p.win_pos, b, p.heads_v, n + 1);
   }
+  if (role == 0 && lane == 0) settle();
 }
 
 }  // namespace lq

@@ -19,7 +19,8 @@ GATE_DIAG = 1
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "liblq.so")
 _lib = None
 
-EXPORTS = ["lq_decode_step", "lq_decode_step_host", "lq_decode_stage_bytes", "lq_window_flush",
+EXPORTS = ["lq_decode_step", "lq_decode_step_host", "lq_decode_stage_bytes", "lq_head_bytes", "lq_record_floats",
+           "lq_window_flush",
            "lq_quantize_state", "lq_dequantize_state", "lq_ref_decode_step_f32", "lq_ref_decode_step_bf16",
            "lq_decode_launches", "lq_check_device", "lq_status_string", "lq_version"]
 
@@ -34,8 +35,7 @@ class _Shape(C.Structure):
 
 
 class _State(C.Structure):
-    _fields_ = [(n, C.c_void_p) for n in
-                ("codes", "col_scale", "row_smooth", "comp_k", "comp_u", "buf_k", "buf_u", "buf_a", "win_pos")]
+    _fields_ = [(n, C.c_void_p) for n in ("heads", "records", "decays", "win_pos")]
 
 
 def lib() -> C.CDLL:
@@ -50,6 +50,9 @@ def lib() -> C.CDLL:
         L.lq_version.restype = C.c_int
         L.lq_decode_stage_bytes.restype = C.c_uint64
         L.lq_decode_stage_bytes.argtypes = [C.c_void_p]
+        for name in ("lq_head_bytes", "lq_record_floats"):
+            getattr(L, name).restype = C.c_uint64
+            getattr(L, name).argtypes = [C.c_void_p]
         L.lq_decode_launches.restype = C.c_int
         L.lq_decode_launches.argtypes = [C.c_void_p]
         for name in ("lq_decode_step", "lq_decode_step_host", "lq_check_device", "lq_window_flush", "lq_quantize_state",
@@ -77,37 +80,52 @@ class Shape:
                       self.gate, self.smooth)
 
 
+def head_bytes(sh: Shape) -> int:
+    s = sh.c()
+    return int(lib().lq_head_bytes(C.byref(s)))
+
+
+def record_floats(sh: Shape) -> int:
+    s = sh.c()
+    return int(lib().lq_record_floats(C.byref(s)))
+
+
 class State:
-    """Device tensors of the window representation of B x Hv heads (layouts as in ``lq_state``)."""
+    """Device tensors of the window representation of B x Hv heads, in the layout of ``lq_state``:
+    ``heads`` (one contiguous byte block per head), ``records`` (one fp32 row per buffered record),
+    ``decays`` (scalar gate) and ``win_pos``.  The named pieces (codes, col_scale, row_smooth, comp_k,
+    comp_u, buf_k, buf_u, buf_a) are strided views into those tensors."""
 
     def __init__(self, sh: Shape, device="cuda"):
         B, H, K, V, W, r = sh.batch, sh.heads_v, sh.d_k, sh.d_v, sh.W, sh.r
-        z = lambda shape, dt: torch.zeros(shape, dtype=dt, device=device)
         self.shape = sh
-        self.codes = z((B, H, K, V), torch.int8)
-        self.col_scale = z((B, H, V), torch.float32)
-        self.row_smooth = torch.ones((B, H, K), dtype=torch.float32, device=device)
-        self.comp_k = z((B, H, max(r, 1), K), torch.float16)
-        self.comp_u = z((B, H, max(r, 1), V), torch.float16)
-        self.buf_k = z((B, H, W, K), torch.float32)
-        self.buf_u = z((B, H, W, V), torch.float32)
-        self.buf_a = z((B, H, W, K) if sh.gate == GATE_DIAG else (B, H, W), torch.float32)
-        self.win_pos = z((B,), torch.int32)
+        hb, rf = head_bytes(sh), record_floats(sh)
+        assert hb > 0 and rf > 0, "shape not supported by the library"
+        self.heads = torch.zeros((B, H, hb), dtype=torch.uint8, device=device)
+        self.records = torch.zeros((B, H, W, rf), dtype=torch.float32, device=device)
+        self.decays = torch.zeros((B, H, W), dtype=torch.float32, device=device)
+        self.win_pos = torch.zeros((B,), dtype=torch.int32, device=device)
+        o = 0
+        self.codes = self.heads[..., o:o + K * V].view(torch.int8).unflatten(-1, (V, K)); o += K * V   # Z^T
+        self.col_scale = self.heads[..., o:o + 4 * V].view(torch.float32); o += 4 * V
+        self.row_smooth = self.heads[..., o:o + 4 * K].view(torch.float32); o += 4 * K
+        self.comp_k = self.heads[..., o:o + 2 * r * K].view(torch.float16).unflatten(-1, (r, K)); o += 2 * r * K
+        self.comp_u = self.heads[..., o:o + 2 * r * V].view(torch.float16).unflatten(-1, (r, V)); o += 2 * r * V
+        assert o == hb
+        self.row_smooth.fill_(1.0)
+        self.buf_k = self.records[..., 0:K]
+        self.buf_u = self.records[..., K:K + V]
+        self.buf_a = self.records[..., K + V:K + V + K] if sh.gate == GATE_DIAG else self.decays
 
     def tensors(self):
-        return (self.codes, self.col_scale, self.row_smooth, self.comp_k, self.comp_u, self.buf_k, self.buf_u,
-                self.buf_a, self.win_pos)
+        return (self.heads, self.records, self.decays, self.win_pos)
 
     def c(self, b0: int = 0) -> _State:
         """ctypes view; ``b0`` offsets every array to sequence b0 (sub-batches are addressed by pointer)."""
-        return _State(*[t.data_ptr() + b0 * (t.stride(0) * t.element_size() if t.dim() > 0 else 0)
-                        for t in self.tensors()])
+        return _State(*[t.data_ptr() + b0 * t.stride(0) * t.element_size() for t in self.tensors()])
 
     def nbytes_quantized(self) -> int:
-        r = self.shape.r
-        per_head = (self.shape.d_k * self.shape.d_v + 4 * self.shape.d_v + 4 * self.shape.d_k
-                    + 2 * r * (self.shape.d_k + self.shape.d_v))
-        return per_head * self.shape.batch * self.shape.heads_v
+        return self.heads.numel()
 
 
 def _stream(stream) -> C.c_void_p:

@@ -20,7 +20,7 @@ def dev(a: np.ndarray) -> torch.Tensor:
 
 
 def host(t: torch.Tensor) -> np.ndarray:
-    a = t.detach().cpu()
+    a = t.detach().cpu().contiguous()
     if a.dtype == torch.float16:
         return a.view(torch.int16).numpy().view(np.uint16)
     if a.dtype == torch.int16:

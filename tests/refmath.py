@@ -45,9 +45,9 @@ def general_step(S, q, k, v, beta, alpha, gate):
 
 
 def dequant_plain(codes, col_scale, row_smooth, comp_k16, comp_u16):
-    """C (Z/127) B + Kc Uc^T for one head, in float64 (Appendix B.3, Eq. 6)."""
+    """C (Z/127) B + Kc Uc^T for one head, in float64 (Appendix B.3, Eq. 6); col_scale holds B/127."""
     Z = codes.astype(np.float64)
-    S = row_smooth.astype(np.float64)[:, None] * (Z / 127.0) * col_scale.astype(np.float64)[None, :]
+    S = row_smooth.astype(np.float64)[:, None] * Z * col_scale.astype(np.float64)[None, :]
     kc = comp_k16.view(np.float16).astype(np.float64)
     uc = comp_u16.view(np.float16).astype(np.float64)
     return S + kc.T @ uc

@@ -36,7 +36,7 @@ def test_argument_errors_are_reported_before_any_launch(L):
     sh = lq.Shape(2, 4, 2)
     s = sh.c()
     null = C.c_void_p(None)
-    st = lq._State(*([None] * 9))
+    st = lq._State(*([None] * 4))
     # null shape / null state / null pointers inside the state
     assert L.lq_decode_step(null, C.byref(st), null, null, null, null, null, null, null) == 1
     assert L.lq_decode_step(C.byref(s), null, null, null, null, null, null, null, null) == 1
@@ -54,15 +54,17 @@ def test_argument_errors_are_reported_before_any_launch(L):
                 lq.Shape(2, 4, 2, r=17)):
         u = uns.c()
         assert L.lq_window_flush(C.byref(u), C.byref(st), 0, null) == 4, uns
-        assert L.lq_decode_stage_bytes(C.byref(u)) == 0
+        assert L.lq_decode_stage_bytes(C.byref(u)) == 0 and L.lq_head_bytes(C.byref(u)) == 0
     # misaligned pointer (fake non-null addresses: nothing is dereferenced on the host)
-    fake = [0x1000 * (i + 1) for i in range(9)]
+    fake = [0x1000 * (i + 1) for i in range(4)]
     st_ok = lq._State(*fake)
     fake[0] += 8
     st_bad = lq._State(*fake)
     assert L.lq_quantize_state(C.byref(s), C.c_void_p(0x100000), C.byref(st_bad), null) == 3
     assert L.lq_quantize_state(C.byref(s), C.c_void_p(0x100004), C.byref(st_ok), null) == 3
     assert lq.decode_stage_bytes(sh) > 0 and lq.decode_launches(sh) >= 1
+    assert lq.head_bytes(sh) == 19456 and lq.record_floats(sh) == 256
+    assert lq.record_floats(lq.Shape(2, 4, 2, gate=lq.GATE_DIAG)) == 384
 
 
 def test_binding_fails_loudly_without_the_library(monkeypatch):

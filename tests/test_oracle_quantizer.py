@@ -26,15 +26,15 @@ def test_plain_code_is_the_nearest_of_255_levels(oracle):
     sh, st = _quant(oracle, S, r=0, smooth=0)
     assert np.array_equal(st.row_smooth, np.ones_like(st.row_smooth))
     S64 = S.astype(np.float64)
-    assert np.array_equal(st.col_scale, np.abs(S).max(axis=2))          # scale = column absmax
+    assert np.array_equal(st.col_scale, np.abs(S).max(axis=2) / np.float32(127.0))   # step = column absmax / 127
     levels = np.arange(-127, 128, dtype=np.float64)
     for h in range(3):
-        grid = levels[None, None, :] / 127.0 * st.col_scale[0, h].astype(np.float64)[None, :, None]
+        grid = levels[None, None, :] * st.col_scale[0, h].astype(np.float64)[None, :, None]
         best = levels[np.argmin(np.abs(S64[0, h][:, :, None] - grid), axis=2)]
         assert np.array_equal(st.codes[0, h].astype(np.float64), best)
         err = np.abs(rm.dequant_plain(st.codes[0, h], st.col_scale[0, h], st.row_smooth[0, h],
                                       st.comp_k[0, h], st.comp_u[0, h]) - S64[0, h])
-        assert np.all(err <= st.col_scale[0, h][None, :] / 254.0 * (1 + 1e-6))
+        assert np.all(err <= st.col_scale[0, h][None, :] / 2.0 * (1 + 1e-6))
     # the column's largest entry maps to +-127 and the code range is symmetric
     assert np.all(np.abs(st.codes).max(axis=2) == 127) and st.codes.min() >= -127
     # dequantize is the same formula
@@ -72,10 +72,10 @@ def test_smoothing_scale_is_sqrt_of_row_mean_abs_and_is_invertible(oracle):
     # after smoothing every row's mean magnitude is the square root of what it was
     assert np.allclose(np.abs(X).mean(axis=3), want_c, rtol=1e-12)
     # the value-channel scale is taken on the smoothed residual
-    assert np.allclose(st.col_scale, np.abs(X).max(axis=2), rtol=1e-6)
+    assert np.allclose(st.col_scale, np.abs(X).max(axis=2) / 127.0, rtol=1e-6)
     # elementwise error bound of the whole chain: half a code step in the original coordinates
     D = oracle.dequantize_state(sh, st).astype(np.float64)
-    bound = st.row_smooth[..., None].astype(np.float64) * st.col_scale[:, :, None, :] / 254.0
+    bound = st.row_smooth[..., None].astype(np.float64) * st.col_scale[:, :, None, :] / 2.0
     assert np.all(np.abs(D - S) <= bound * (1 + 1e-5) + 1e-12)
     # smoothing must help on rows of very different magnitude: compare with the unsmoothed code
     sh0, st0 = _quant(oracle, S, r=0, smooth=0)
@@ -122,8 +122,8 @@ def test_compensators_are_the_best_rank_r_fit(oracle, r):
         assert abs(np.linalg.norm(uc[h]) - s[h]) < 2e-3 * s[h]
     # Eq. 6: dequant(R_hat) + K U^T differs from S only by the quantization of the residual
     D = oracle.dequantize_state(sh, st)[0, 0].astype(np.float64)
-    assert np.all(np.abs(D - M) <= st.col_scale[0, 0][None, :] / 254.0 * (1 + 1e-5) + 1e-9)
-    assert np.allclose(st.col_scale[0, 0], np.abs(resid).max(axis=0), rtol=1e-5)
+    assert np.all(np.abs(D - M) <= st.col_scale[0, 0][None, :] / 2.0 * (1 + 1e-5) + 1e-9)
+    assert np.allclose(st.col_scale[0, 0], np.abs(resid).max(axis=0) / 127.0, rtol=1e-5)
 
 
 def test_default_iteration_count_already_captures_the_energy(oracle):

@@ -189,7 +189,7 @@ def test_boundary_term_is_exact_up_to_the_fixed_point_grid(oracle):
             q, k, v, beta, alpha = rm.widen(tok, wl, b, h)
             c = st.row_smooth[b, h].astype(np.float64)
             x = (c.astype(np.float32) * (np.float32(alpha) * k.astype(np.float32))).astype(np.float64)
-            s = (st.col_scale[b, h] / np.float32(127.0)).astype(np.float64)
+            s = st.col_scale[b, h].astype(np.float64)
             Z = st.codes[b, h].astype(np.float64)
             exact = s * (Z.T @ x)
             got = v - st.buf_u[b, h, 0].astype(np.float64)
