@@ -26,10 +26,13 @@
  * Summation order.  The paper never says in which order a sum is taken, yet
  * the 8-bit codes and the fp16 compensators are step functions of fp32
  * values, so the order has to be part of the definition.  Every reduction in
- * this file goes through csum_dot()/csum_abs(): consecutive blocks of eight
- * terms are accumulated left to right (first product rounded, the others
- * folded in with fmaf), and the block results are then added as a balanced
- * binary tree over the block index (neighbours first).  Building the file
+ * this file goes through csum_dot()/csum_abs(): the terms are taken in
+ * consecutive blocks of eight; inside a block the even-numbered and the
+ * odd-numbered terms are accumulated separately, left to right (first product
+ * rounded, the others folded in with fmaf), and the two halves are added; the
+ * block results are then added as a balanced binary tree over the block index
+ * (neighbours first).  (Two interleaved chains per block are what a two-wide
+ * fp32 fused multiply-add gives.)  Building the file
  * with -DLQO_WIDE replaces this by a plain left-to-right sum in binary64,
  * rounded once; comparing the two builds measures how much of any
  * disagreement is attributable to fp32 summation order.
@@ -157,8 +160,13 @@ float lqo_csum_dot(const float *a, const float *b, int n) {
     float acc = 0.0f;
     if (c < nblk) {
       int lo = 8 * c, hi = lo + 8 < n ? lo + 8 : n;
-      acc = a[lo] * b[lo];
-      for (int i = lo + 1; i < hi; i++) acc = fmaf(a[i], b[i], acc);
+      float even = a[lo] * b[lo], odd = 0.0f;
+      for (int i = lo + 2; i < hi; i += 2) even = fmaf(a[i], b[i], even);
+      if (lo + 1 < hi) {
+        odd = a[lo + 1] * b[lo + 1];
+        for (int i = lo + 3; i < hi; i += 2) odd = fmaf(a[i], b[i], odd);
+      }
+      acc = even + odd;
     }
     part[c] = acc;
   }
@@ -185,8 +193,10 @@ float lqo_csum_abs(const float *x, int n) {
     float acc = 0.0f;
     if (c < nblk) {
       int lo = 8 * c, hi = lo + 8 < n ? lo + 8 : n;
-      acc = fabsf(x[lo]);
-      for (int i = lo + 1; i < hi; i++) acc = acc + fabsf(x[i]);
+      float even = fabsf(x[lo]), odd = 0.0f;
+      for (int i = lo + 2; i < hi; i += 2) even = even + fabsf(x[i]);
+      for (int i = lo + 1; i < hi; i += 2) odd = odd + fabsf(x[i]);
+      acc = even + odd;
     }
     part[c] = acc;
   }

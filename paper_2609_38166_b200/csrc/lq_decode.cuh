@@ -11,8 +11,9 @@
 // where thousands of 16-byte loads could not (plain loads are limited per warp), and about 64 KB in flight
 // per SM saturate HBM.  The slot is small enough for six CTAs per SM.  CTAs are persistent and walk over
 // the heads with a grid stride.  No load sits on a head's critical path (with the memory system kept full a
-// load takes several microseconds to return): the token's vectors are fetched two heads ahead into
-// registers, the per-head scalars (window position, beta, scalar alpha) for 32 heads at a time, one per lane.
+// load from DRAM takes several microseconds to return): the token's vectors are asked into the L2 three heads
+// ahead and loaded into registers one head ahead, the per-head scalars (window position, beta, scalar alpha)
+// are loaded for 32 heads at a time, one per lane.
 //
 // Roles: the STREAM warp turns C Gamma x into fixed-point digits, runs the tensor-core pass over the codes
 // and finishes u and o; the DOT warp meanwhile takes the projections onto the buffered records and the
@@ -38,11 +39,13 @@ __device__ int g_device_error = 0;
 // warps, summed over all heads by lane 0 of each warp (slots 0..15: stream warp, 16..31: dot warp).
 #ifdef LQ_TIMING
 __device__ unsigned long long g_phase_cycles[32];
-#define LQ_TICK(slot)                                                                               \
-  do {                                                                                              \
-    const long long now_ = clock64();                                                               \
-    if (lane == 0) atomicAdd(&g_phase_cycles[16 * role + (slot)], (unsigned long long)(now_ - tick_)); \
-    tick_ = now_;                                                                                   \
+// cycles are summed in registers and flushed once per warp at the end of the kernel, so that the probe
+// itself puts no traffic on the memory system while the kernel runs
+#define LQ_TICK(slot)                                     \
+  do {                                                    \
+    const long long now_ = clock64();                     \
+    acc_[slot] += static_cast<unsigned>(now_ - tick_);    \
+    tick_ = now_;                                         \
   } while (0)
 #else
 #define LQ_TICK(slot) do { } while (0)
@@ -70,7 +73,7 @@ struct DecodeSlot {
 // D(16x8, s32) += A(16x32, s8, row-major) * B(32x8, s8, column-major)
 __device__ __forceinline__ void mma_s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                        uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+  asm("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
                : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
                : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
@@ -149,7 +152,7 @@ __device__ __forceinline__ void named_arrive(int id) {
 }
 __device__ __forceinline__ void named_wait(int id) { asm volatile("bar.sync %0, 64;\n" ::"r"(id) : "memory"); }
 
-// The token's vectors as raw bf16 bits, loaded two heads ahead: lane c (and its twin c+16) owns key
+// The token's vectors as raw bf16 bits, loaded one head ahead (and asked into the L2 three heads ahead): lane c (and its twin c+16) owns key
 // channels 8c..8c+7, lane l value channels 4l..4l+3.
 struct TokenRaw {
   uint4 k, q, a;        // a: diagonal-gate alpha
@@ -157,10 +160,20 @@ struct TokenRaw {
   float ba_lo, ba_hi;   // scalar gate: decays of buffered records `lane` and `lane + 32` (stale beyond n)
 };
 
+// A head index with its sequence and value-head parts, stepped without divisions.
+struct HeadIdx {
+  unsigned bh, b, hv;
+  __device__ __forceinline__ void step(unsigned dbh, unsigned db, unsigned dhv, unsigned heads_v) {
+    bh += dbh; b += db; hv += dhv;
+    if (hv >= heads_v) { hv -= heads_v; b += 1; }
+  }
+};
+
 template <int GATE>
-__device__ __forceinline__ void load_token(const Params &p, size_t bh, int lane, int role, TokenRaw &tk) {
-  const int b = static_cast<int>(bh / p.heads_v), hv = static_cast<int>(bh % p.heads_v), c = lane & 15;
-  const size_t qk_off = ((size_t)b * p.heads_qk + hv / (p.heads_v / p.heads_qk)) * D;
+__device__ __forceinline__ void load_token(const Params &p, const HeadIdx h, int group, int lane, int role, TokenRaw &tk) {
+  const int c = lane & 15;
+  const size_t bh = h.bh;
+  const size_t qk_off = ((size_t)h.b * p.heads_qk + h.hv / group) * D;
   tk.k = *reinterpret_cast<const uint4 *>(p.k + qk_off + 8 * c);
   tk.q = *reinterpret_cast<const uint4 *>(p.q + qk_off + 8 * c);
   if (role == 0) tk.v = *reinterpret_cast<const uint2 *>(p.v + bh * D + 4 * lane);
@@ -170,6 +183,22 @@ __device__ __forceinline__ void load_token(const Params &p, size_t bh, int lane,
     if (lane < p.W) tk.ba_lo = p.decays[bh * (size_t)p.W + lane];
     if (lane + 32 < p.W) tk.ba_hi = p.decays[bh * (size_t)p.W + lane + 32];
   }
+}
+
+// Asks the L2 for a later head's token lines (no register is written, so nothing waits for it): when the
+// token is loaded one head ahead it then comes from the L2 instead of queueing behind the bulk traffic.
+template <int GATE>
+__device__ __forceinline__ void prefetch_token_l2(const Params &p, const HeadIdx h, int group, int lane, int role) {
+  const size_t bh = h.bh;
+  const size_t qk_off = ((size_t)h.b * p.heads_qk + h.hv / group) * D;
+  const void *addr = nullptr;     // 256-byte vectors: two 128-byte lines each
+  if (lane < 2) addr = p.k + qk_off + 64 * lane;
+  else if (lane < 4) addr = p.q + qk_off + 64 * (lane - 2);
+  else if (lane < 6 && role == 0) addr = p.v + bh * D + 64 * (lane - 4);
+  else if (GATE == LQ_GATE_DIAG && lane >= 6 && lane < 8) addr = p.alpha + bh * D + 64 * (lane - 6);
+  else if (GATE == LQ_GATE_SCALAR && lane >= 6 && lane < 8 && 32 * (lane - 6) < p.W)
+    addr = p.decays + bh * (size_t)p.W + 32 * (lane - 6);
+  if (addr) asm volatile("prefetch.global.L2 [%0];\n" ::"l"(addr));
 }
 
 // Persistent kernel of two-warp CTAs: CTA `blockIdx.x` takes heads blockIdx.x, blockIdx.x + gridDim.x, ...
@@ -197,13 +226,21 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
   if (threadIdx.x == 0) mbar_init(bar, 1);
   __syncthreads();
   uint32_t parity = 0;
-  const size_t nh = (size_t)p.batch * p.heads_v, G = gridDim.x;
+  const unsigned nh = static_cast<unsigned>(p.batch) * p.heads_v, G = gridDim.x, Hv = p.heads_v;
+  const unsigned G_b = G / Hv, G_hv = G % Hv;       // one grid stride in (sequence, head) steps
+  const int group = p.heads_v / p.heads_qk;
 
+#ifdef LQ_TIMING
+  long long tick_ = clock64();
+  unsigned acc_[12] = {0};
+#endif
   // Requests head bh (n records buffered) into the slot: two bulk copies, issued by two lanes of the dot
   // warp when nobody reads the slot any more.
-  auto request = [&](size_t bh, int n) {
-    // the slot was last touched through ordinary loads and stores; order them before the async writes
-    asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+  auto request = [&](unsigned bh, int n) {
+    // The regions the copies overwrite were only READ through ordinary loads, whose values have been used
+    // before the barrier that precedes this call; the warps write only their scratch regions.  So nothing
+    // written by the generic proxy is at stake and no cross-proxy fence is needed (it costs over a
+    // thousand cycles here).
     const uint32_t hb = head_bytes(r), rb = 4u * RF * n;
     if (lane == 0) {
       mbar_expect_tx(bar, hb + rb);
@@ -215,10 +252,10 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
   // Per-head scalars of this CTA's heads, 32 heads at a time: lane l holds those of the CTA's (32*batch+l)-th head
   int sc_n = 0;
   uint32_t sc_beta = 0, sc_alpha = 0;
-  auto load_scalars = [&](size_t first_bh) {
-    const size_t bh = first_bh + (size_t)lane * G;
+  auto load_scalars = [&](unsigned first_bh) {
+    const unsigned bh = first_bh + lane * G;  // (once per 32 heads: a division is fine here)
     if (bh < nh) {
-      sc_n = p.win_pos[bh / p.heads_v];     // bits 16.. are the arrival counter of this launch: masked at use
+      sc_n = p.win_pos[bh / Hv];            // bits 16.. are the arrival counter of this launch: masked at use
       sc_beta = p.beta[bh];
       if (!DIAG) sc_alpha = p.alpha[bh];
     }
@@ -234,51 +271,60 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
 
   // A head whose window is already full (n >= W) gets no token: it is neither requested nor waited for.
   load_scalars(blockIdx.x);
-  TokenRaw tok0, tok1, tok2;                  // this head's token, the next head's, the one after
-  tok0.ba_lo = tok0.ba_hi = tok1.ba_lo = tok1.ba_hi = tok2.ba_lo = tok2.ba_hi = 1.0f;
-  if (blockIdx.x < nh) load_token<GATE>(p, blockIdx.x, lane, role, tok0);
-  if (blockIdx.x + G < nh) load_token<GATE>(p, blockIdx.x + G, lane, role, tok1);
+  TokenRaw nxt;                               // the token of the head about to start
+  nxt.ba_lo = nxt.ba_hi = 1.0f;
+  HeadIdx hd{blockIdx.x, blockIdx.x / Hv, blockIdx.x % Hv};      // this head, the next one, and three ahead
+  HeadIdx hd1 = hd, hd3;
+  hd1.step(G, G_b, G_hv, Hv);
+  hd3 = hd1;
+  if (hd.bh < nh) load_token<GATE>(p, hd, group, lane, role, nxt);
+  if (hd3.bh < nh) prefetch_token_l2<GATE>(p, hd3, group, lane, role);
+  hd3.step(G, G_b, G_hv, Hv);
+  if (hd3.bh < nh) prefetch_token_l2<GATE>(p, hd3, group, lane, role);
+  hd3.step(G, G_b, G_hv, Hv);
   {
     const int n0 = __shfl_sync(FULL, sc_n, 0) & 0xFFFF;
     if (role == 1 && blockIdx.x < nh && n0 < W) request(blockIdx.x, n0);
   }
 #ifdef LQ_TIMING
-  long long tick_ = clock64();
+  tick_ = clock64();
 #endif
   int idx = 0;                               // position of the head in this CTA's list
-  for (size_t bh = blockIdx.x; bh < nh; bh += G, idx++) {
+  for (; hd.bh < nh; hd = hd1, hd1.step(G, G_b, G_hv, Hv), hd3.step(G, G_b, G_hv, Hv), idx++) {
+    const size_t bh = hd.bh;
     const int n = __shfl_sync(FULL, sc_n, idx & 31) & 0xFFFF;
     const float beta = __uint_as_float(__shfl_sync(FULL, sc_beta, idx & 31) << 16);
     const float alpha_s = __uint_as_float(__shfl_sync(FULL, sc_alpha, idx & 31) << 16);
     // the next head's scalars: from the next batch when this head is the last of its batch
-    const size_t bh_next = bh + G;
+    const unsigned bh_next = hd1.bh;
     if ((idx & 31) == 31) load_scalars(bh_next);
     const int n_next = bh_next < nh ? (__shfl_sync(FULL, sc_n, (idx + 1) & 31) & 0xFFFF) : W;
     const bool active = n < W, next_active = n_next < W;
-    const int b = static_cast<int>(bh / p.heads_v);
-    if (bh + 2 * G < nh) load_token<GATE>(p, bh + 2 * G, lane, role, tok2);   // used two trips from now
-    const TokenRaw cur = tok0;
-    tok0 = tok1;
-    tok1 = tok2;
+    const int b = static_cast<int>(hd.b);
+    if (hd3.bh < nh) prefetch_token_l2<GATE>(p, hd3, group, lane, role);
     LQ_TICK(0);
 
     if (!active) {                           // nothing was requested for this head; keep the pipeline going
+      if (bh_next < nh) load_token<GATE>(p, hd1, group, lane, role, nxt);
       if (role == 1 && next_active) request(bh_next, n_next);
       continue;
     }
 
-    // ---- this head's token ----
+    // ---- this head's token (loaded while the previous head was being worked on); once it is unpacked
+    // the registers are free for the next head's, whose load is then issued ----
     float k8[8], q8[8], a8[8];
-    widen8_bf16(cur.k, k8);
-    widen8_bf16(cur.q, q8);
+    widen8_bf16(nxt.k, k8);
+    widen8_bf16(nxt.q, q8);
+    const uint2 v_raw = nxt.v;
     if (DIAG) {
-      widen8_bf16(cur.a, a8);
+      widen8_bf16(nxt.a, a8);
     } else {
 #pragma unroll
       for (int e = 0; e < 8; e++) a8[e] = alpha_s;
-      bas[lane] = cur.ba_lo;
-      bas[lane + 32] = cur.ba_hi;
+      bas[lane] = nxt.ba_lo;
+      bas[lane + 32] = nxt.ba_hi;
     }
+    if (bh_next < nh) load_token<GATE>(p, hd1, group, lane, role, nxt);       // used one trip from now
     LQ_TICK(1);
 
     // ---- wait for the slot (bounded: a copy that never lands must not hang the GPU) ----
@@ -395,6 +441,11 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
       __syncwarp();
       LQ_TICK(4);
       named_arrive(1);                       // the projections are in shared memory
+      LQ_TICK(5);
+      named_wait(2);                         // the stream warp has read all it needs from the slot
+      LQ_TICK(6);
+      // the request goes out before this warp's global stores: the proxy fence in it would wait for them
+      if (next_active) request(bh_next, n_next);
       // append the key side of the record (and its decay)
       {
         float *row = p.record(bh, n, DIAG);
@@ -404,10 +455,6 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
           else if (lane == 0) p.decays[bh * (size_t)W + n] = a8[0];
         }
       }
-      LQ_TICK(5);
-      named_wait(2);                         // the stream warp has read all it needs from the slot
-      LQ_TICK(6);
-      if (next_active) request(bh_next, n_next);
       LQ_TICK(7);
     } else {
       // =========================== STREAM WARP ===========================
@@ -475,34 +522,40 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
       // chain of MMAs.  Digit pairs are recombined in int32 (|sum| < 2^30), the two pairs in binary64, which
       // holds the 47-bit total exactly, and one rounding takes it to fp32.
       {
-        uint4 bf[2];
-#pragma unroll
-        for (int pp = 0; pp < 2; pp++) bf[pp] = *reinterpret_cast<const uint4 *>(digits + g * D + 64 * pp + 16 * t);
+        constexpr int h0 = 0, h1 = 64;         // the two 64-channel halves (the same split for every lane)
+        const uint4 bfa = *reinterpret_cast<const uint4 *>(digits + g * D + h0 + 16 * t);
+        const uint4 bfb = *reinterpret_cast<const uint4 *>(digits + g * D + h1 + 16 * t);
+        int pair_lo[8], pair_hi[8];            // digit-pair sums of rows g and g+8 of each tile
 #pragma unroll
         for (int mt = 0; mt < 8; mt++) {
           int ca[4] = {0, 0, 0, 0}, cb[4] = {0, 0, 0, 0};
           const int j = 16 * mt + g;
-          {
-            const uint4 zlo = *reinterpret_cast<const uint4 *>(zt + j * D + 16 * t);
-            const uint4 zhi = *reinterpret_cast<const uint4 *>(zt + (j + 8) * D + 16 * t);
-            mma_s8(ca, zlo.x, zhi.x, zlo.y, zhi.y, bf[0].x, bf[0].y);
-            mma_s8(ca, zlo.z, zhi.z, zlo.w, zhi.w, bf[0].z, bf[0].w);
-          }
-          {
-            const uint4 zlo = *reinterpret_cast<const uint4 *>(zt + j * D + 64 + 16 * t);
-            const uint4 zhi = *reinterpret_cast<const uint4 *>(zt + (j + 8) * D + 64 + 16 * t);
-            mma_s8(cb, zlo.x, zhi.x, zlo.y, zhi.y, bf[1].x, bf[1].y);
-            mma_s8(cb, zlo.z, zhi.z, zlo.w, zhi.w, bf[1].z, bf[1].w);
-          }
+          const uint4 alo = *reinterpret_cast<const uint4 *>(zt + j * D + h0 + 16 * t);
+          const uint4 ahi = *reinterpret_cast<const uint4 *>(zt + (j + 8) * D + h0 + 16 * t);
+          const uint4 blo = *reinterpret_cast<const uint4 *>(zt + j * D + h1 + 16 * t);
+          const uint4 bhi = *reinterpret_cast<const uint4 *>(zt + (j + 8) * D + h1 + 16 * t);
+          mma_s8(ca, alo.x, ahi.x, alo.y, ahi.y, bfa.x, bfa.y);
+          mma_s8(cb, blo.x, bhi.x, blo.y, bhi.y, bfb.x, bfb.y);
+          mma_s8(ca, alo.z, ahi.z, alo.w, ahi.w, bfa.z, bfa.w);
+          mma_s8(cb, blo.z, bhi.z, blo.w, bhi.w, bfb.z, bfb.w);
           // c[0], c[1]: row g, planes 2t, 2t+1;  c[2], c[3]: row g+8.  Planes 4v..4v+3 are the digits of
           // vector v: lanes t = 0, 1 carry the k sums and t = 2, 3 the q sums, even t the low digit pair.
-          const int pair_g = (ca[0] + cb[0]) + ((ca[1] + cb[1]) << 8);
-          const int pair_g8 = (ca[2] + cb[2]) + ((ca[3] + cb[3]) << 8);
-          const int other_g = __shfl_xor_sync(FULL, pair_g, 1), other_g8 = __shfl_xor_sync(FULL, pair_g8, 1);
-          if (!(t & 1)) {                    // this lane has the low pair, its neighbour sent the high pair
-            float *dst = y + (t >> 1) * D;
-            dst[j] = __double2float_rn(fma(static_cast<double>(other_g), 65536.0, static_cast<double>(pair_g)));
-            dst[j + 8] = __double2float_rn(fma(static_cast<double>(other_g8), 65536.0, static_cast<double>(pair_g8)));
+          pair_lo[mt] = (ca[0] + cb[0]) + ((ca[1] + cb[1]) << 8);
+          pair_hi[mt] = (ca[2] + cb[2]) + ((ca[3] + cb[3]) << 8);
+        }
+        LQ_TICK(10);
+        int oth_lo[8], oth_hi[8];
+#pragma unroll
+        for (int mt = 0; mt < 8; mt++) {
+          oth_lo[mt] = __shfl_xor_sync(FULL, pair_lo[mt], 1);
+          oth_hi[mt] = __shfl_xor_sync(FULL, pair_hi[mt], 1);
+        }
+        if (!(t & 1)) {                      // this lane has the low pairs, its neighbour sent the high pairs
+          float *dst = y + (t >> 1) * D + g;
+#pragma unroll
+          for (int mt = 0; mt < 8; mt++) {
+            dst[16 * mt] = __double2float_rn(fma(static_cast<double>(oth_lo[mt]), 65536.0, static_cast<double>(pair_lo[mt])));
+            dst[16 * mt + 8] = __double2float_rn(fma(static_cast<double>(oth_hi[mt]), 65536.0, static_cast<double>(pair_hi[mt])));
           }
         }
       }
@@ -517,8 +570,8 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
         const float4 s4 = *reinterpret_cast<const float4 *>(bs + 4 * lane);      // code steps B_j / 127
         float rk[4] = {s4.x * (yk4.x * back_k), s4.y * (yk4.y * back_k), s4.z * (yk4.z * back_k), s4.w * (yk4.w * back_k)};
         float rq[4] = {s4.x * (yq4.x * back_q), s4.y * (yq4.y * back_q), s4.z * (yq4.z * back_q), s4.w * (yq4.w * back_q)};
-        const float v4[4] = {__uint_as_float(cur.v.x << 16), __uint_as_float(cur.v.x & 0xFFFF0000u),
-                             __uint_as_float(cur.v.y << 16), __uint_as_float(cur.v.y & 0xFFFF0000u)};
+        const float v4[4] = {__uint_as_float(v_raw.x << 16), __uint_as_float(v_raw.x & 0xFFFF0000u),
+                             __uint_as_float(v_raw.y << 16), __uint_as_float(v_raw.y & 0xFFFF0000u)};
         LQ_TICK(6);
         named_wait(1);                       // pk, pq are complete
         LQ_TICK(7);
@@ -560,6 +613,10 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
     }
   }
   if (role == 0 && lane == 0) settle();
+#ifdef LQ_TIMING
+  if (lane == 0)
+    for (int i = 0; i < 12; i++) atomicAdd(&g_phase_cycles[16 * role + i], (unsigned long long)acc_[i]);
+#endif
 }
 
 }  // namespace lq

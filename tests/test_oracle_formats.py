@@ -77,15 +77,17 @@ def test_csum_close_to_binary64_sum(oracle, oracle_wide):
 
 
 def test_csum_order_is_blocks_of_eight_then_neighbour_tree(oracle):
-    """Terms chosen so that only the stated order reproduces the result:
-    a huge value, its negation and small values placed where a left-to-right sum loses them."""
-    n = 32
-    a = np.ones(n, np.float32)
-    b = np.zeros(n, np.float32)
-    b[0] = 2.0 ** 30; b[1:8] = 1.0           # block 0: the ones vanish next to 2^30 (spacing 128)
-    b[8] = -(2.0 ** 30); b[9:16] = 1.0       # block 1: the same with the other sign
+    """Terms chosen so that only the stated order reproduces the result: inside a block of eight the even
+    and the odd terms are summed separately and then added; blocks are combined neighbours first."""
+    a = np.ones(32, np.float32)
+    b = np.zeros(32, np.float32)
+    # block 0: even terms 2^30, 1, 1, 1 (the ones vanish next to 2^30, spacing 128); odd terms -2^30, 1, 1, 1
+    b[0] = 2.0 ** 30; b[1] = -(2.0 ** 30); b[2:8] = 1.0
+    b[8:16] = 1.0                            # block 1: 4 + 4
     b[16:32] = 1.0                           # blocks 2, 3: 8 each
-    # blocks: [2^30, -2^30, 8, 8] -> tree: (2^30 + -2^30) + (8 + 8) = 16
-    assert oracle.csum_dot(a, b) == 16.0
-    # a left-to-right sum would give 2^30 - 2^30 + ... = 7 + 16 = 23; a fully pairwise one 30
+    # blocks: [2^30 + (-2^30) = 0, 8, 8, 8] -> tree: (0 + 8) + (8 + 8) = 24
+    assert oracle.csum_dot(a, b) == 24.0
+    # even terms 2^24, 1, 1, 1 stay 2^24 (ties to even); odd terms 1+1+1+1 = 4 survive
+    assert oracle.csum_abs(np.array([2.0 ** 24, 1, 1, 1, 1, 1, 1, 1], np.float32)) == float(2.0 ** 24 + 4)
+    # a left-to-right sum would give 2^30 - 2^30 + 6 + 24 = 30, which is also the exact value
     assert float(np.sum(b.astype(np.float64))) == 30.0
