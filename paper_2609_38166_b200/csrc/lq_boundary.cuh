@@ -192,11 +192,11 @@ __device__ __forceinline__ void quantize_tile(const Params &p, const BoundarySme
   if (p.smooth) {
     float pr[8];
 #pragma unroll
-    for (int a = 0; a < 8; a++) {
-      float s = fabsf(M[a][0]);
+    for (int a = 0; a < 8; a++) {                             // even and odd columns as two chains
+      float even = fabsf(M[a][0]), odd = fabsf(M[a][1]);
 #pragma unroll
-      for (int b = 1; b < 8; b++) s = s + fabsf(M[a][b]);
-      pr[a] = s;
+      for (int b = 2; b < 8; b += 2) { even = even + fabsf(M[a][b]); odd = odd + fabsf(M[a][b + 1]); }
+      pr[a] = even + odd;
     }
     int sel;
     const float tot = row_tree(pr, t.lane, sel);

@@ -2,11 +2,13 @@
 //
 // Everything is compiled with -fmad=false: a product is fused with an addition only where fmaf() is
 // written, so that every value is reproducible bit for bit.  Sums over a channel index follow one
-// fixed order: blocks of eight consecutive terms accumulated left to right (first product rounded, the
-// rest folded in with fmaf), block results added as a balanced binary tree over the block index.
-// The thread mappings below are chosen so that this order is the natural one: a thread owns one block
-// of eight, neighbouring lanes own neighbouring blocks, and butterfly exchanges with lane masks
-// 1, 2, 4, ... walk up the tree.
+// fixed order: the terms are taken in blocks of eight; inside a block the even- and the odd-numbered
+// terms form two chains, each accumulated left to right (first product rounded, the rest folded in with
+// fmaf), and the two chains are added; block results are added as a balanced binary tree over the block
+// index.  The thread mappings below are chosen so that this order is the natural one: a thread owns one
+// block of eight (where registers allow, as four float2 pairs, so that one packed fused multiply-add,
+// FFMA2 on sm_100, advances both chains); neighbouring lanes own neighbouring blocks, and butterfly
+// exchanges with lane masks 1, 2, 4, ... walk up the tree.
 #pragma once
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
@@ -86,15 +88,34 @@ __device__ __forceinline__ float tree16(float x) {
   return x;
 }
 
+__device__ __forceinline__ float2 pair(float x) { return make_float2(x, x); }
+
+// Block result of eight products a[e]*b[e] given as four pairs: the .x components are the even-numbered
+// terms, the .y components the odd-numbered ones; each chain runs left to right, then the two are added.
+__device__ __forceinline__ float block8(const float2 (&a)[4], const float2 (&b)[4]) {
+  float2 acc = __fmul2_rn(a[0], b[0]);
+#pragma unroll
+  for (int c = 1; c < 4; c++) acc = __ffma2_rn(a[c], b[c], acc);
+  return acc.x + acc.y;
+}
+
+__device__ __forceinline__ void load8p(const float *src, float2 (&x)[4]) {
+  const float4 lo = *reinterpret_cast<const float4 *>(src), hi = *reinterpret_cast<const float4 *>(src + 4);
+  x[0] = make_float2(lo.x, lo.y); x[1] = make_float2(lo.z, lo.w);
+  x[2] = make_float2(hi.x, hi.y); x[3] = make_float2(hi.z, hi.w);
+}
+__device__ __forceinline__ void store8p(float *dst, const float2 (&x)[4]) {
+  *reinterpret_cast<float4 *>(dst) = make_float4(x[0].x, x[0].y, x[1].x, x[1].y);
+  *reinterpret_cast<float4 *>(dst + 4) = make_float4(x[2].x, x[2].y, x[3].x, x[3].y);
+}
+
 // Dot product of two 128-vectors in shared memory, computed by sixteen neighbouring lanes
 // (lane c = lane & 15 owns block c); every one of the sixteen lanes returns the sum.
 __device__ __forceinline__ float dot128_shared(const float *a, const float *b, int c) {
-  const float4 a0 = *reinterpret_cast<const float4 *>(a + 8 * c), a1 = *reinterpret_cast<const float4 *>(a + 8 * c + 4);
-  const float4 b0 = *reinterpret_cast<const float4 *>(b + 8 * c), b1 = *reinterpret_cast<const float4 *>(b + 8 * c + 4);
-  float s = a0.x * b0.x;
-  s = fmaf(a0.y, b0.y, s); s = fmaf(a0.z, b0.z, s); s = fmaf(a0.w, b0.w, s);
-  s = fmaf(a1.x, b1.x, s); s = fmaf(a1.y, b1.y, s); s = fmaf(a1.z, b1.z, s); s = fmaf(a1.w, b1.w, s);
-  return tree16(s);
+  float2 a2[4], b2[4];
+  load8p(a + 8 * c, a2);
+  load8p(b + 8 * c, b2);
+  return tree16(block8(a2, b2));
 }
 
 // =====================================================================================
@@ -166,24 +187,32 @@ __device__ __forceinline__ void col_tree(const float (&p)[8], float *part, float
   load8(out + 8 * t.tx, w);
 }
 
-// p[b] = block result over this thread's eight rows of  sum_a M[a][b] * x[a]
+// p[b] = block result over this thread's eight rows of  sum_a M[a][b] * x[a]: rows 0,2,4,6 and rows
+// 1,3,5,7 are the two chains of the block.  (Scalar operations: a packed one would need the per-row
+// multiplier duplicated into a register pair, and the 64-register tile leaves no room for that.)
 __device__ __forceinline__ void col_blocks(const float (&M)[8][8], const float (&x)[8], float (&p)[8]) {
 #pragma unroll
   for (int b = 0; b < 8; b++) {
-    float s = M[0][b] * x[0];
+    float even = M[0][b] * x[0], odd = M[1][b] * x[1];
 #pragma unroll
-    for (int a = 1; a < 8; a++) s = fmaf(M[a][b], x[a], s);
-    p[b] = s;
+    for (int a = 2; a < 8; a += 2) {
+      even = fmaf(M[a][b], x[a], even);
+      odd = fmaf(M[a + 1][b], x[a + 1], odd);
+    }
+    p[b] = even + odd;
   }
 }
 // p[a] = block result over this thread's eight columns of  sum_b M[a][b] * x[b]
 __device__ __forceinline__ void row_blocks(const float (&M)[8][8], const float (&x)[8], float (&p)[8]) {
 #pragma unroll
   for (int a = 0; a < 8; a++) {
-    float s = M[a][0] * x[0];
+    float even = M[a][0] * x[0], odd = M[a][1] * x[1];
 #pragma unroll
-    for (int b = 1; b < 8; b++) s = fmaf(M[a][b], x[b], s);
-    p[a] = s;
+    for (int b = 2; b < 8; b += 2) {
+      even = fmaf(M[a][b], x[b], even);
+      odd = fmaf(M[a][b + 1], x[b + 1], odd);
+    }
+    p[a] = even + odd;
   }
 }
 

@@ -344,43 +344,45 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
       // shuffle trees overlap.  Both halves make the same number of trips (the shuffles name all 32 lanes);
       // an index outside the range recomputes a valid item and is not stored.
       // Records are walked from the newest back, with g8 = Gamma_{j+1:l} kept up on the way (Appendix B.2).
-      float g8[8], kt8[8];
+      float2 k2[4], q2[4], a2[4], g2[4], kt2[4];
 #pragma unroll
-      for (int e = 0; e < 8; e++) { g8[e] = a8[e]; kt8[e] = beta * k8[e]; }
+      for (int cc = 0; cc < 4; cc++) {
+        k2[cc] = make_float2(k8[2 * cc], k8[2 * cc + 1]);
+        q2[cc] = make_float2(q8[2 * cc], q8[2 * cc + 1]);
+        a2[cc] = make_float2(a8[2 * cc], a8[2 * cc + 1]);
+        g2[cc] = a2[cc];
+        kt2[cc] = __fmul2_rn(pair(beta), k2[cc]);
+      }
       for (int jt = n - 1; jt >= 0; jt -= 4) {       // records jt, jt-1, jt-2, jt-3
         float s4[4];
         int jo[2];
 #pragma unroll
         for (int u = 0; u < 2; u++) {
           // the decays of the two records of this pair; the half that owns the older one steps over the newer
-          float gmine[8];
           const int jn = jt - 2 * u, jold = jn - 1;  // newer, older
-          float an[8], ao[8];
+          float2 an[4], ao[4], gmine[4];
           if (DIAG) {
-            load8(rec + (jn > 0 ? jn : 0) * RF + REC_A + 8 * c, an);
-            load8(rec + (jold > 0 ? jold : 0) * RF + REC_A + 8 * c, ao);
+            load8p(rec + (jn > 0 ? jn : 0) * RF + REC_A + 8 * c, an);
+            load8p(rec + (jold > 0 ? jold : 0) * RF + REC_A + 8 * c, ao);
           } else {
-            const float x = bas[jn > 0 ? jn : 0], z = bas[jold > 0 ? jold : 0];
+            const float2 x = pair(bas[jn > 0 ? jn : 0]), z = pair(bas[jold > 0 ? jold : 0]);
 #pragma unroll
-            for (int e = 0; e < 8; e++) { an[e] = x; ao[e] = z; }
+            for (int cc = 0; cc < 4; cc++) { an[cc] = x; ao[cc] = z; }
           }
 #pragma unroll
-          for (int e = 0; e < 8; e++) {
-            const float gn = g8[e], go = gn * an[e];      // Gamma_{jn+1:l}, Gamma_{jold+1:l}
-            gmine[e] = half ? go : gn;
-            g8[e] = go * ao[e];                           // past both records
+          for (int cc = 0; cc < 4; cc++) {
+            const float2 gn = g2[cc], go = __fmul2_rn(gn, an[cc]);   // Gamma_{jn+1:l}, Gamma_{jold+1:l}
+            gmine[cc] = half ? go : gn;
+            g2[cc] = __fmul2_rn(go, ao[cc]);                          // past both records
           }
           jo[u] = jn - half;
           const int j = jo[u] >= 0 ? jo[u] : 0;
-          float x8[8];
-          load8(rec + j * RF + REC_KT + 8 * c, x8);
-          float sk = x8[0] * (gmine[0] * k8[0]), sq = x8[0] * (gmine[0] * q8[0]);
+          float2 x2[4], yk2[4], yq2[4];
+          load8p(rec + j * RF + REC_KT + 8 * c, x2);
 #pragma unroll
-          for (int e = 1; e < 8; e++) {
-            sk = fmaf(x8[e], gmine[e] * k8[e], sk);
-            sq = fmaf(x8[e], gmine[e] * q8[e], sq);
-          }
-          s4[2 * u] = sk; s4[2 * u + 1] = sq;
+          for (int cc = 0; cc < 4; cc++) { yk2[cc] = __fmul2_rn(gmine[cc], k2[cc]); yq2[cc] = __fmul2_rn(gmine[cc], q2[cc]); }
+          s4[2 * u] = block8(x2, yk2);
+          s4[2 * u + 1] = block8(x2, yq2);
         }
         tree16x4(s4);
 #pragma unroll
@@ -389,25 +391,25 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
       }
       LQ_TICK(3);
       // Compensator keys against Gamma_{1:l} k and Gamma_{1:l} q; item r is kt^T q (kept in pq[n+r]).
-      // g8 may have run past record 0 above: Gamma_{1:l} is rebuilt from the exact chain.
+      // g2 may have run past record 0 above: Gamma_{1:l} is rebuilt from the exact chain.
       {
-        float gam[8];
+        float2 gam[4];
 #pragma unroll
-        for (int e = 0; e < 8; e++) gam[e] = a8[e];
+        for (int cc = 0; cc < 4; cc++) gam[cc] = a2[cc];
         for (int j = n - 1; j >= 0; j--) {
-          float aj[8];
-          if (DIAG) load8(rec + j * RF + REC_A + 8 * c, aj);
+          float2 aj[4];
+          if (DIAG) load8p(rec + j * RF + REC_A + 8 * c, aj);
           else {
-            const float x = bas[j];
+            const float2 x = pair(bas[j]);
 #pragma unroll
-            for (int e = 0; e < 8; e++) aj[e] = x;
+            for (int cc = 0; cc < 4; cc++) aj[cc] = x;
           }
 #pragma unroll
-          for (int e = 0; e < 8; e++) gam[e] = gam[e] * aj[e];
+          for (int cc = 0; cc < 4; cc++) gam[cc] = __fmul2_rn(gam[cc], aj[cc]);
         }
-        float gk8[8], gq8[8];
+        float2 gk2[4], gq2[4];
 #pragma unroll
-        for (int e = 0; e < 8; e++) { gk8[e] = gam[e] * k8[e]; gq8[e] = gam[e] * q8[e]; }
+        for (int cc = 0; cc < 4; cc++) { gk2[cc] = __fmul2_rn(gam[cc], k2[cc]); gq2[cc] = __fmul2_rn(gam[cc], q2[cc]); }
         for (int hb = 0; hb < r + 1; hb += 4) {
           float s4[4];
           int ho[2];
@@ -418,19 +420,15 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
             float x8[8];
             if (r > 0) widen8_f16(*reinterpret_cast<const uint4 *>(ckh + h * D + 8 * c), x8);
             const bool is_ktq = ho[u] >= r;
-            float sk, sq;
-            {
-              const float x0 = is_ktq ? kt8[0] : x8[0];
-              sk = x0 * (is_ktq ? q8[0] : gk8[0]);
-              sq = x0 * (is_ktq ? q8[0] : gq8[0]);
-            }
+            float2 x2[4], yk2[4], yq2[4];
 #pragma unroll
-            for (int e = 1; e < 8; e++) {
-              const float xe = is_ktq ? kt8[e] : x8[e];
-              sk = fmaf(xe, is_ktq ? q8[e] : gk8[e], sk);
-              sq = fmaf(xe, is_ktq ? q8[e] : gq8[e], sq);
+            for (int cc = 0; cc < 4; cc++) {
+              x2[cc] = is_ktq ? kt2[cc] : make_float2(x8[2 * cc], x8[2 * cc + 1]);
+              yk2[cc] = is_ktq ? q2[cc] : gk2[cc];
+              yq2[cc] = is_ktq ? q2[cc] : gq2[cc];
             }
-            s4[2 * u] = sk; s4[2 * u + 1] = sq;
+            s4[2 * u] = block8(x2, yk2);
+            s4[2 * u + 1] = block8(x2, yq2);
           }
           tree16x4(s4);
 #pragma unroll
@@ -450,7 +448,7 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
       {
         float *row = p.record(bh, n, DIAG);
         if (half == 0) {
-          store8(row + REC_KT + 8 * c, kt8);
+          store8p(row + REC_KT + 8 * c, kt2);
           if (DIAG) store8(row + REC_A + 8 * c, a8);
           else if (lane == 0) p.decays[bh * (size_t)W + n] = a8[0];
         }
