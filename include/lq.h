@@ -46,7 +46,8 @@ typedef enum {
   LQ_ERR_SHAPE = 2,       /* a dimension is non-positive or inconsistent        */
   LQ_ERR_ALIGN = 3,       /* a pointer is not 16-byte aligned                   */
   LQ_ERR_UNSUPPORTED = 4, /* valid request outside the supported shapes         */
-  LQ_ERR_CUDA = 5         /* the CUDA runtime reported an error on launch/copy  */
+  LQ_ERR_CUDA = 5,        /* the CUDA runtime reported an error on launch/copy  */
+  LQ_ERR_TOO_LARGE = 6    /* the request does not fit the library's built-in scratch buffer */
 } lq_status;
 
 typedef enum {
@@ -131,6 +132,34 @@ lq_status lq_decode_step_host(const lq_shape *shape, const lq_state *state, cons
                               const uint16_t *alpha_h, float *o_h, void *stage, lq_stream stream);
 /* Bytes of device staging lq_decode_step_host needs for `shape` (0 if the shape is invalid). */
 uint64_t lq_decode_stage_bytes(const lq_shape *shape);
+
+/*
+ * lq_decode_step_host for callers that cannot hand over a staging buffer because they cannot allocate one.
+ * (The paper has no counterpart: this is a convenience of the library.)
+ *
+ * Who this is for: a serving process that gave all of the device's memory to its own pools when it started
+ * has nothing left for cudaMalloc to return, and a decode loop that must never stall cannot afford
+ * cudaMalloc/cudaFree either, since both may synchronise the whole device.  Such a caller still owns the
+ * host arrays and the lq_state, but has nowhere to put the few megabytes of staging that the host-buffer
+ * path needs.  Here the staging lives inside the library, in a fixed device array of
+ * LQ_STATIC_STAGE_BYTES bytes that every GPU that loads the library keeps reserved until the process
+ * exits.  The call itself allocates and frees nothing, on the device or through any library.
+ *
+ * Same arguments and behaviour as lq_decode_step_host without `stage`, with these differences:
+ *  - lq_decode_stage_bytes(shape) must not exceed LQ_STATIC_STAGE_BYTES, otherwise LQ_ERR_TOO_LARGE is
+ *    returned and nothing is enqueued (16 MiB covers 256 sequences x 32 heads, the benchmark batch).
+ *  - The first call on each device looks up the device address of the built-in array (with that device
+ *    current).  Make that first call outside any stream capture.
+ *  - The array is shared by all calls and keeps what the previous call left in it.  The output staging is
+ *    therefore cleared at the start of every call: rows of o_h that belong to sequences which get no token
+ *    (win_pos >= W on entry) come back as zeros.
+ *  - Because the array is shared, two calls whose work overlaps on the GPU (different streams, or different
+ *    host threads) race on it.  Order them on one stream, or use lq_decode_step_host with separate buffers.
+ */
+#define LQ_STATIC_STAGE_BYTES (16u << 20)
+lq_status lq_decode_step_host_static(const lq_shape *shape, const lq_state *state, const uint16_t *q_h,
+                                     const uint16_t *k_h, const uint16_t *v_h, const uint16_t *beta_h,
+                                     const uint16_t *alpha_h, float *o_h, lq_stream stream);
 
 /*
  * Window boundary (Secs. 3.2-3.4): for every sequence with win_pos == W, or, when force != 0, with

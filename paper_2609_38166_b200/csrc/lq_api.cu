@@ -1,6 +1,7 @@
 // C boundary of the library: argument checks, launch configuration, and the kernels that wrap the
 // device routines of lq_decode.cuh and lq_boundary.cuh.  Declarations and contracts: include/lq.h.
 #include <algorithm>
+#include <atomic>
 #include <cstdio>
 
 #include "lq_boundary.cuh"
@@ -306,6 +307,57 @@ lq_status lq_decode_step_host(const lq_shape *shape, const lq_state *state, cons
   return LQ_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Host-buffer decode step without a caller-supplied staging buffer: the staging is this array.
+// It is a device object of the library: every GPU that loads the library carries it until exit.  In host
+// code the name below is only a handle; the device address comes from cudaGetSymbolAddress, looked up once
+// per device and cached.
+// ---------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_stage[LQ_STATIC_STAGE_BYTES];
+
+static lq_status static_stage_address(void **out) {
+  constexpr int MAX_DEVICES = 64;
+  static std::atomic<void *> cached[MAX_DEVICES];
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) {
+    cudaGetLastError();
+    return LQ_ERR_CUDA;
+  }
+  void *ptr = cached[dev].load(std::memory_order_acquire);
+  if (!ptr) {                                 // first call on this device (it is the current device)
+    if (cudaGetSymbolAddress(&ptr, g_static_stage) != cudaSuccess || !ptr) {
+      cudaGetLastError();
+      return LQ_ERR_CUDA;
+    }
+    cached[dev].store(ptr, std::memory_order_release);   // two racing first calls store the same address
+  }
+  *out = ptr;
+  return LQ_OK;
+}
+
+lq_status lq_decode_step_host_static(const lq_shape *shape, const lq_state *state, const uint16_t *q_h,
+                                     const uint16_t *k_h, const uint16_t *v_h, const uint16_t *beta_h,
+                                     const uint16_t *alpha_h, float *o_h, lq_stream stream) {
+  lq_status rc = check_shape(shape);
+  if (rc != LQ_OK) return rc;
+  const uint64_t need = lq_decode_stage_bytes(shape);
+  if (need > LQ_STATIC_STAGE_BYTES) return LQ_ERR_TOO_LARGE;
+  if (!q_h || !k_h || !v_h || !beta_h || !alpha_h || !o_h) return LQ_ERR_NULL;
+  void *stage = nullptr;
+  if ((rc = static_stage_address(&stage)) != LQ_OK) return rc;
+  if (shape->batch == 0) return LQ_OK;
+  // The array still holds the previous call's staging.  The inputs are overwritten in full by this call's
+  // copies; the output region is cleared, so that rows no kernel writes (sequences with a full window on
+  // entry) do not leak an earlier call's results into o_h.  The output region is the last one in the buffer.
+  const uint64_t out_bytes = 4ull * shape->batch * shape->heads_v * shape->d_v;
+  unsigned char *out_region = static_cast<unsigned char *>(stage) + (need - (out_bytes + 255) / 256 * 256);
+  if (cudaMemsetAsync(out_region, 0, out_bytes, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) {
+    cudaGetLastError();
+    return LQ_ERR_CUDA;
+  }
+  return lq_decode_step_host(shape, state, q_h, k_h, v_h, beta_h, alpha_h, o_h, stage, stream);
+}
+
 lq_status lq_window_flush(const lq_shape *shape, const lq_state *state, int force, lq_stream stream) {
   lq_status rc = check_shape(shape);
   if (rc != LQ_OK) return rc;
@@ -401,6 +453,7 @@ const char *lq_status_string(lq_status status) {
     case LQ_ERR_ALIGN: return "pointer not 16-byte aligned";
     case LQ_ERR_UNSUPPORTED: return "shape not supported";
     case LQ_ERR_CUDA: return "CUDA runtime error";
+    case LQ_ERR_TOO_LARGE: return "request exceeds the built-in scratch buffer";
   }
   return "unknown status";
 }
