@@ -35,9 +35,9 @@ WARM_TOKENS = 512
 STATE_BYTES = 128 * 128 + 4 * 128 + 4 * 128 + 2 * 4 * (128 + 128)       # 19456 per head at r = 4
 METRIC = "GDN decode state-GB/s at bs256 (8-bit per-window state, W=16, r=4)"
 
-# DRAM bytes per launch of the dominant kernel from the ncu capture summarised under profiles/
-# (dram__bytes_read.sum + dram__bytes_write.sum; scaled to the full batch by heads processed), or None.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+# DRAM bytes per launch from the ncu captures summarised under profiles/ (dram__bytes_read.sum +
+# dram__bytes_write.sum of one full-batch launch of the gdn_b256 workload, W = 16), or None when not captured.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"decode_kernel": None, "boundary_kernel": None}
 
 
 def algorithmic_bytes_per_head_step(W: int, r: int, diag: bool, group: int, launches_fused: bool) -> float:
@@ -50,6 +50,38 @@ def algorithmic_bytes_per_head_step(W: int, r: int, diag: bool, group: int, laun
     inputs = 512 / group + 256 + 2 + 2 * g
     flush = state + (0 if launches_fused else state + W * rec)      # write back (+ re-read when a second kernel does it)
     return state + buf_read + inputs + rec + 512 + flush / W
+
+
+def config_dict(wl, world: int, warm_tokens: int) -> dict:
+    heads = wl.batch * wl.heads_v
+    return {"workload": wl.name, "batch": wl.batch, "heads_v": wl.heads_v, "heads_qk": wl.heads_qk,
+            "d_k": wl.d_k, "d_v": wl.d_v, "W": wl.W, "r": wl.r, "n_iter": wl.n_iter,
+            "gate": "scalar (GDN)" if wl.gate == synth.GATE_SCALAR else "diagonal (KDA)",
+            "state_dtype": "int8 + fp32 scales + fp16 compensators", "record_buffer_dtype": "f32",
+            "inputs_dtype": "bf16", "warmup_tokens": warm_tokens, "window_offsets": "uniform over [0,W)",
+            "l2": "working set %.0f MB per step exceeds the 126 MB L2; no flush needed" %
+                  (heads * (STATE_BYTES + wl.W * 1028) / 1e6),
+            "parallelism": "dp%d (independent batches, no collective)" % world}
+
+
+def shard_workload(wl, rank: int):
+    """Every rank owns its own batch of the same shape (weak scaling): only the seed differs."""
+    return wl.with_(seed=wl.seed + 1000 * rank)
+
+
+def max_over_ranks(value_ms: float, dist_mod=None, device=None) -> float:
+    """Slowest rank's time; `dist_mod` is torch.distributed when a process group is up, else None."""
+    if dist_mod is None or not dist_mod.is_initialized() or dist_mod.get_world_size() == 1:
+        return value_ms
+    import torch
+    t = torch.tensor([value_ms], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist_mod.all_reduce(t, op=dist_mod.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(heads_per_rank: int, world: int, steps: int, ms: float) -> float:
+    """state-GB/s of the whole job: all ranks' head-steps over the slowest rank's time."""
+    return world * heads_per_rank * steps / (ms / 1e3) * STATE_BYTES / 1e9
 
 
 def peaks():
@@ -168,8 +200,7 @@ def run_reference(args, wl):
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": s_per_step * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "tokens_heads_per_s": hs,
-            "config": {"workload": wl.name, "batch": wl.batch, "heads_v": wl.heads_v, "heads_qk": wl.heads_qk,
-                       "d_k": wl.d_k, "d_v": wl.d_v, "W": wl.W, "r": wl.r, "gate": "scalar (GDN)"},
+            "config": config_dict(wl, args.gpus, 0),
             "cpu_baseline": {"value": value, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
@@ -232,7 +263,7 @@ def run_cuda(args, wl):
         dist.barrier()
     lq.lib()                                             # raises if the CUDA library is missing
 
-    wl = wl.with_(seed=wl.seed + 1000 * rank)            # every rank owns its own batch (weak scaling, no exchange)
+    wl = shard_workload(wl, rank)                        # every rank owns its own batch (weak scaling, no exchange)
     sh, st, o = prepare_state(wl, lq, torch, log, args.warm_tokens)
     WARM_TOKENS = args.warm_tokens
     toks = [to_dev(synth.token_inputs(wl, WARM_TOKENS + t), torch) for t in range(wl.W)]
@@ -272,10 +303,7 @@ def run_cuda(args, wl):
         torch.cuda.synchronize()
         sampler.stop()
         clock_source = "identical loop run right after the timed region (timed region shorter than the sampling period)"
-    if world > 1:
-        tmax = torch.tensor([ms], device="cuda")
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        ms = float(tmax.item())
+    ms = max_over_ranks(ms, dist if world > 1 else None, "cuda")
 
     # the same step captured in a CUDA graph (one graph = W steps), for the launch-overhead-free figure
     graph_ms = None
@@ -328,17 +356,34 @@ def run_cuda(args, wl):
         e1.record(stream)
         barrier()
         e2e_ms = e0.elapsed_time(e1)
-        if world > 1:
-            tm = torch.tensor([e2e_ms], device="cuda")
-            dist.all_reduce(tm, op=dist.ReduceOp.MAX)
-            e2e_ms = float(tm.item())
+        e2e_ms = max_over_ranks(e2e_ms, dist if world > 1 else None, "cuda")
         h2d = sum(v.numel() * v.element_size() for v in pin[0].values())
-        e2e = {"value": world * wl.batch * wl.heads_v * n_e2e / (e2e_ms / 1e3) * STATE_BYTES / 1e9, "unit": "GB/s",
+        e2e = {"value": whole_job_value(wl.batch * wl.heads_v, world, n_e2e, e2e_ms), "unit": "GB/s",
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": o_h.numel() * 4, "steps": n_e2e,
                "ms_per_step": e2e_ms / n_e2e,
                "api": "lq_decode_step_host (pinned host q,k,v,beta,alpha in; o out), one call per step"}
     except Exception as exc:
         log(f"end-to-end timing failed: {exc!r}")
+
+    # The two kernels of a step timed separately: a second loop, with an event between the kernels
+    kern = None
+    try:
+        n_k = min(args.steps, 256)
+        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(n_k)]
+        for trio in evs:
+            for e in trio:
+                e.record(stream)               # materialises the CUDA handles
+        torch.cuda.synchronize()
+        for t in range(n_k):
+            d = toks[t % wl.W]
+            evs[t][0].record(stream)
+            lq.decode_step_profiled(sh, st, d["q"], d["k"], d["v"], d["beta"], d["alpha"], o, evs[t][1], stream)
+            evs[t][2].record(stream)
+        torch.cuda.synchronize()
+        kern = {"decode_ms": statistics.mean(e[0].elapsed_time(e[1]) for e in evs),
+                "boundary_ms": statistics.mean(e[1].elapsed_time(e[2]) for e in evs), "steps": n_k}
+    except Exception as exc:
+        log(f"per-kernel timing failed: {exc!r}")
 
     if rank != 0:
         if world > 1:
@@ -353,11 +398,32 @@ def run_cuda(args, wl):
     group = wl.heads_v // wl.heads_qk
     bytes_hs = algorithmic_bytes_per_head_step(wl.W, wl.r, wl.gate == synth.GATE_DIAG, group, launches == 1)
     achieved = heads * bytes_hs / (ms_per_step / 1e3) / 1e9
+    g = 128 if wl.gate == synth.GATE_DIAG else 1
+    rec = 4 * (256 + g)
+    # what each kernel has to move per launch: the decode kernel everything but the boundary; the boundary
+    # kernel, for the 1/W of the heads whose window is full, the window representation in and the head block out
+    decode_bytes = heads * (bytes_hs - (2 * STATE_BYTES + wl.W * rec) / wl.W)
+    boundary_bytes = heads / wl.W * (2 * STATE_BYTES + wl.W * rec)
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "peak_source": peak_src,
-                "kernel": "lq_decode_step = decode_kernel + boundary_kernel, timed together (CUDA events, one step)",
+                "traffic": None, "peak_source": peak_src,
+                "kernel": "one step = decode_kernel + boundary_kernel (algorithmic bytes of both over the step time "
+                          "of the timed region; the decode kernel carries 93 % of the bytes)",
                 "algorithmic_bytes_per_head_step": bytes_hs, "algorithmic_bytes_per_step": heads * bytes_hs,
                 "frac_of_nominal_8TBps": achieved / 8000.0}
+    if kern:
+        dk, bk = kern["decode_ms"], kern["boundary_ms"]
+        roofline["kernels"] = {
+            "decode_kernel": {"ms": dk, "algorithmic_bytes": decode_bytes, "achieved": decode_bytes / dk / 1e6,
+                              "frac": decode_bytes / dk / 1e6 / peak, "bound": "hbm",
+                              "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH["decode_kernel"]},
+            "boundary_kernel": {"ms": bk, "algorithmic_bytes": boundary_bytes, "achieved": boundary_bytes / bk / 1e6,
+                                "frac": boundary_bytes / bk / 1e6 / peak,
+                                "bound": "fp32 issue/latency (see DESIGN.md 6.2), not hbm",
+                                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH["boundary_kernel"]},
+            "how": "CUDA events on the launching stream around each kernel, mean of %d steps in a second loop" %
+                   kern["steps"]}
+        t_d, t_b = NCU_TRAFFIC_BYTES_PER_LAUNCH["decode_kernel"], NCU_TRAFFIC_BYTES_PER_LAUNCH["boundary_kernel"]
+        roofline["traffic"] = (t_d + t_b) if (t_d and t_b) else None
 
     # speed baselines in the same run: dense fp32 / bf16 state, read and written every token
     base = {}
@@ -389,21 +455,14 @@ def run_cuda(args, wl):
 
     cpu = None
     if not args.only_timed:
-        hs_cpu, cores, sample, _ = time_oracle(wl.with_(seed=wl.seed), steps=4 * wl.W, warmup=2, budget_s=25.0)
+        hs_cpu, cores, sample, _ = time_oracle(wl.with_(seed=wl.seed), steps=8 * wl.W, warmup=2, budget_s=25.0)
         cpu = {"value": hs_cpu * STATE_BYTES / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
                "sample": sample, "tokens_heads_per_s": hs_cpu}
 
     line = {"metric": METRIC, "value": hs * STATE_BYTES / 1e9, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": wl.name, "batch": wl.batch, "heads_v": wl.heads_v, "heads_qk": wl.heads_qk,
-                       "d_k": wl.d_k, "d_v": wl.d_v, "W": wl.W, "r": wl.r, "n_iter": wl.n_iter,
-                       "gate": "scalar (GDN)", "state_dtype": "int8 + fp32 scales + fp16 compensators",
-                       "record_buffer_dtype": "f32", "inputs_dtype": "bf16", "warmup_tokens": args.warm_tokens,
-                       "window_offsets": "uniform over [0,W)",
-                       "l2": "working set %.0f MB per step exceeds the 126 MB L2; no flush needed" %
-                             (heads * (STATE_BYTES + wl.W * 1028) / 1e6),
-                       "parallelism": "dp%d (independent batches, no collective)" % world},
+            "config": config_dict(wl, world, args.warm_tokens),
             "tokens_heads_per_s": hs, "pct_hbm_peak_measured": 100 * achieved / peak,
             "pct_hbm_peak_nominal_8TBps": 100 * achieved / 8000.0,
             "cuda_graph_ms_per_step": graph_ms, "gpu_launches": launches * args.steps,

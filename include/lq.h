@@ -121,6 +121,15 @@ lq_status lq_decode_step(const lq_shape *shape, const lq_state *state, const uin
                          const uint16_t *v, const uint16_t *beta, const uint16_t *alpha, float *o, lq_stream stream);
 
 /*
+ * lq_decode_step for a measuring harness: identical work, and in addition the CUDA event `event_between`
+ * (a cudaEvent_t created by the caller; may be null) is recorded on `stream` between the decode kernel and
+ * the window-boundary kernel, so that the two can be timed separately.
+ */
+lq_status lq_decode_step_profiled(const lq_shape *shape, const lq_state *state, const uint16_t *q, const uint16_t *k,
+                                  const uint16_t *v, const uint16_t *beta, const uint16_t *alpha, float *o,
+                                  lq_stream stream, void *event_between);
+
+/*
  * Same as lq_decode_step, but the token's inputs and the output live in HOST memory (pinned memory makes
  * the copies asynchronous): q_h, k_h, v_h, beta_h, alpha_h are copied into the device staging buffer
  * `stage` on `stream`, the step runs, and `o` is copied to o_h.  `stage` is a device buffer of at least

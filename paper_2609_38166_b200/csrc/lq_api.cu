@@ -235,8 +235,9 @@ using namespace lq;
 
 extern "C" {
 
-lq_status lq_decode_step(const lq_shape *shape, const lq_state *state, const uint16_t *q, const uint16_t *k,
-                         const uint16_t *v, const uint16_t *beta, const uint16_t *alpha, float *o, lq_stream stream) {
+static lq_status decode_step_impl(const lq_shape *shape, const lq_state *state, const uint16_t *q, const uint16_t *k,
+                                  const uint16_t *v, const uint16_t *beta, const uint16_t *alpha, float *o,
+                                  lq_stream stream, cudaEvent_t between) {
   lq_status rc = check_shape(shape);
   if (rc != LQ_OK) return rc;
   if ((rc = check_state(shape, state, true)) != LQ_OK) return rc;
@@ -253,7 +254,22 @@ lq_status lq_decode_step(const lq_shape *shape, const lq_state *state, const uin
   rc = diag ? launch_persistent(decode_kernel<LQ_GATE_DIAG>, nh, 64, smem, st, p)
             : launch_persistent(decode_kernel<LQ_GATE_SCALAR>, nh, 64, smem, st, p);
   if (rc != LQ_OK) return rc;
+  if (between && cudaEventRecord(between, st) != cudaSuccess) {
+    cudaGetLastError();
+    return LQ_ERR_CUDA;
+  }
   return launch_boundary<0>(shape, p, st);     // sequences whose window just became full
+}
+
+lq_status lq_decode_step(const lq_shape *shape, const lq_state *state, const uint16_t *q, const uint16_t *k,
+                         const uint16_t *v, const uint16_t *beta, const uint16_t *alpha, float *o, lq_stream stream) {
+  return decode_step_impl(shape, state, q, k, v, beta, alpha, o, stream, nullptr);
+}
+
+lq_status lq_decode_step_profiled(const lq_shape *shape, const lq_state *state, const uint16_t *q, const uint16_t *k,
+                                  const uint16_t *v, const uint16_t *beta, const uint16_t *alpha, float *o,
+                                  lq_stream stream, void *event_between) {
+  return decode_step_impl(shape, state, q, k, v, beta, alpha, o, stream, static_cast<cudaEvent_t>(event_between));
 }
 
 uint64_t lq_head_bytes(const lq_shape *s) { return check_shape(s) == LQ_OK ? (uint64_t)head_bytes(s->r) : 0; }

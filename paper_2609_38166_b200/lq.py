@@ -19,7 +19,7 @@ GATE_DIAG = 1
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "liblq.so")
 _lib = None
 
-EXPORTS = ["lq_decode_step", "lq_decode_step_host", "lq_decode_step_host_static", "lq_decode_stage_bytes", "lq_head_bytes", "lq_record_floats",
+EXPORTS = ["lq_decode_step", "lq_decode_step_profiled", "lq_decode_step_host", "lq_decode_step_host_static", "lq_decode_stage_bytes", "lq_head_bytes", "lq_record_floats",
            "lq_window_flush",
            "lq_quantize_state", "lq_dequantize_state", "lq_ref_decode_step_f32", "lq_ref_decode_step_bf16",
            "lq_decode_launches", "lq_check_device", "lq_status_string", "lq_version"]
@@ -55,7 +55,7 @@ def lib() -> C.CDLL:
             getattr(L, name).argtypes = [C.c_void_p]
         L.lq_decode_launches.restype = C.c_int
         L.lq_decode_launches.argtypes = [C.c_void_p]
-        for name in ("lq_decode_step", "lq_decode_step_host", "lq_decode_step_host_static", "lq_check_device", "lq_window_flush", "lq_quantize_state",
+        for name in ("lq_decode_step", "lq_decode_step_profiled", "lq_decode_step_host", "lq_decode_step_host_static", "lq_check_device", "lq_window_flush", "lq_quantize_state",
                      "lq_dequantize_state", "lq_ref_decode_step_f32", "lq_ref_decode_step_bf16"):
             getattr(L, name).restype = C.c_int
         _lib = L
@@ -157,6 +157,16 @@ def decode_step(sh: Shape, st: State, q, k, v, beta, alpha, o, stream=None, b0: 
     cs = st.c(b0)
     _check(lib().lq_decode_step(C.byref(s), C.byref(cs), _ptr(q, b0), _ptr(k, b0), _ptr(v, b0), _ptr(beta, b0),
                                 _ptr(alpha, b0), _ptr(o, b0), _stream(stream)), "lq_decode_step")
+
+
+def decode_step_profiled(sh: Shape, st: State, q, k, v, beta, alpha, o, event_between, stream=None):
+    """lq_decode_step_profiled: ``event_between`` is a torch.cuda.Event that has been recorded once before
+    (so that its CUDA handle exists); it is re-recorded between the two kernels of the step."""
+    s = sh.c()
+    cs = st.c()
+    _check(lib().lq_decode_step_profiled(C.byref(s), C.byref(cs), _ptr(q), _ptr(k), _ptr(v), _ptr(beta),
+                                         _ptr(alpha), _ptr(o), _stream(stream), C.c_void_p(event_between.cuda_event)),
+           "lq_decode_step_profiled")
 
 
 def decode_stage_bytes(sh: Shape) -> int:

@@ -1,0 +1,94 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times: the whole batch runs on
+the GPU (through bench.prepare_state, i.e. fp32-state warm-up, group-by-group quantization, staggered window
+offsets), and sampled sequences are recomputed one by one by the CPU oracle from the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+import bench
+from oracle.lq_oracle import Shape as OShape, State as OState
+from paper_2609_38166_b200 import lq, synth
+from tests import gpu_util as gu
+
+pytestmark = pytest.mark.gpu
+
+
+def _oracle_sequence(oracle, wl, b, toks, warm, steps):
+    """What bench.prepare_state + `steps` decode steps do to sequence b, on the oracle (batch of one)."""
+    per = max(wl.batch // wl.W, 1)
+    groups = (wl.batch + per - 1) // per
+    g = min(b // per, groups - 1)                       # sequence b is quantized after warm - g tokens
+    one = wl.with_(batch=1)
+    sh = OShape(1, wl.heads_v, wl.heads_qk, wl.d_k, wl.d_v, wl.W, wl.r, wl.n_iter, wl.gate, wl.smooth)
+    cut = lambda tok: {k: np.ascontiguousarray(v[b:b + 1]) for k, v in tok.items()}
+    S = np.zeros((1, wl.heads_v, wl.d_k, wl.d_v), np.float32)
+    st = OState(sh)
+    outs = []
+    for t in range(warm + steps):
+        if t == warm - g:
+            oracle.quantize_state(sh, S, st)
+        if t < warm - g:
+            oracle.ref_step_f32(sh, S, **cut(toks[t]))
+        else:
+            o = oracle.decode_step(sh, st, **cut(toks[t]))
+            if t >= warm:
+                outs.append(o[0])
+    return st, outs
+
+
+@pytest.mark.parametrize("name,W,warm,steps", [("gdn_b256", 16, 24, 20), ("gdn_b256", 8, 12, 10),
+                                               ("kda_b128_outlier", 16, 20, 18)])
+def test_full_batch_against_sampled_oracle_sequences(oracle, name, W, warm, steps):
+    wl = synth.config(name).with_(W=W)
+    toks = [synth.token_inputs(wl, t) for t in range(warm + steps)]
+    sh, st, o = bench.prepare_state(wl, lq, torch, lambda m: None, warm)
+    sample = sorted({0, 1, wl.batch // W, wl.batch // 2 + 3, wl.batch - wl.batch // W - 1, wl.batch - 1})
+    got = {b: [] for b in sample}
+    for t in range(steps):
+        d = bench.to_dev(toks[warm + t], torch)
+        lq.decode_step(sh, st, d["q"], d["k"], d["v"], d["beta"], d["alpha"], o)
+        oh = o[sample].cpu().numpy()
+        for i, b in enumerate(sample):
+            got[b].append(oh[i])
+    torch.cuda.synchronize()
+    assert lq.check_device() == 0
+    codes = gu.gpu_codes(st)
+    for b in sample:
+        ost, want = _oracle_sequence(oracle, wl, b, toks, warm, steps)
+        for t in range(steps):
+            assert np.allclose(got[b][t], want[t], rtol=1e-3, atol=1e-5), (b, t)
+            assert np.array_equal(got[b][t], want[t]), (b, t)
+        frac, worst = gu.code_mismatch(codes[b], ost.codes[0])
+        assert worst <= 1 and frac <= 1e-4 and frac == 0.0, (b, frac, worst)
+        assert int(st.win_pos[b]) == int(ost.win_pos[0])
+        for name_, g, w in (("col_scale", st.col_scale, ost.col_scale), ("row_smooth", st.row_smooth, ost.row_smooth),
+                            ("buf_u", st.buf_u, ost.buf_u), ("buf_k", st.buf_k, ost.buf_k)):
+            assert np.array_equal(gu.host(g[b]), w[0]), (b, name_)
+        assert np.array_equal(gu.host(st.comp_u[b]), ost.comp_u[0]), b
+
+
+def test_drift_against_the_unquantized_recurrence():
+    """Accuracy figure (reported, not a parity check): relative error of o against the fp32-state kernel fed
+    the same inputs, heavy-tailed values, per block of 64 steps of a 256-step chain."""
+    wl = synth.config("gdn_drift").with_(batch=8, heads_v=8, heads_qk=8)
+    sh = lq.Shape(wl.batch, wl.heads_v, wl.heads_qk, wl.d_k, wl.d_v, wl.W, wl.r, wl.n_iter, wl.gate, wl.smooth)
+    st = lq.State(sh)
+    S = torch.zeros((wl.batch, wl.heads_v, 128, 128), dtype=torch.float32, device="cuda")
+    S16 = torch.zeros((wl.batch, wl.heads_v, 128, 128), dtype=torch.int16, device="cuda")
+    lq.quantize_state(sh, S, st)
+    o = torch.empty((wl.batch, wl.heads_v, 128), dtype=torch.float32, device="cuda")
+    oref, o16 = torch.empty_like(o), torch.empty_like(o)
+    err, err16 = [], []
+    for step in range(256):
+        d = bench.to_dev(synth.token_inputs(wl, step), torch)
+        a = (d["q"], d["k"], d["v"], d["beta"], d["alpha"])
+        lq.decode_step(sh, st, *a, o)
+        lq.ref_decode_step_f32(sh, S, *a, oref)
+        lq.ref_decode_step_bf16(sh, S16, *a, o16)
+        err.append(float((o - oref).norm() / oref.norm()))
+        err16.append(float((o16 - oref).norm() / oref.norm()))
+    blocks = [float(np.mean(err[i:i + 64])) for i in range(0, 256, 64)]
+    blocks16 = [float(np.mean(err16[i:i + 64])) for i in range(0, 256, 64)]
+    print("drift 8-bit per-window:", blocks, " bf16 per-step:", blocks16)
+    assert max(blocks[1:]) < 2e-3                       # stays flat: no accumulation along the chain
+    assert blocks[3] < 3 * blocks[1] + 1e-4
