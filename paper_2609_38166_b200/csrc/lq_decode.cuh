@@ -11,9 +11,8 @@
 // where thousands of 16-byte loads could not (plain loads are limited per warp), and about 64 KB in flight
 // per SM saturate HBM.  The slot is small enough for six CTAs per SM.  CTAs are persistent and walk over
 // the heads with a grid stride.  No load sits on a head's critical path (with the memory system kept full a
-// load from DRAM takes several microseconds to return): the token's vectors are asked into the L2 three heads
-// ahead and loaded into registers one head ahead, the per-head scalars (window position, beta, scalar alpha)
-// are loaded for 32 heads at a time, one per lane.
+// load takes microseconds to return): the token's vectors are loaded into registers one head ahead, the
+// per-head scalars (window position, beta, scalar alpha) for 32 heads at a time, one per lane.
 //
 // Roles: the STREAM warp turns C Gamma x into fixed-point digits, runs the tensor-core pass over the codes
 // and finishes u and o; the DOT warp meanwhile takes the projections onto the buffered records and the
@@ -152,7 +151,7 @@ __device__ __forceinline__ void named_arrive(int id) {
 }
 __device__ __forceinline__ void named_wait(int id) { asm volatile("bar.sync %0, 64;\n" ::"r"(id) : "memory"); }
 
-// The token's vectors as raw bf16 bits, loaded one head ahead (and asked into the L2 three heads ahead): lane c (and its twin c+16) owns key
+// The token's vectors as raw bf16 bits, loaded one head ahead: lane c (and its twin c+16) owns key
 // channels 8c..8c+7, lane l value channels 4l..4l+3.
 struct TokenRaw {
   uint4 k, q, a;        // a: diagonal-gate alpha
@@ -183,22 +182,6 @@ __device__ __forceinline__ void load_token(const Params &p, const HeadIdx h, int
     if (lane < p.W) tk.ba_lo = p.decays[bh * (size_t)p.W + lane];
     if (lane + 32 < p.W) tk.ba_hi = p.decays[bh * (size_t)p.W + lane + 32];
   }
-}
-
-// Asks the L2 for a later head's token lines (no register is written, so nothing waits for it): when the
-// token is loaded one head ahead it then comes from the L2 instead of queueing behind the bulk traffic.
-template <int GATE>
-__device__ __forceinline__ void prefetch_token_l2(const Params &p, const HeadIdx h, int group, int lane, int role) {
-  const size_t bh = h.bh;
-  const size_t qk_off = ((size_t)h.b * p.heads_qk + h.hv / group) * D;
-  const void *addr = nullptr;     // 256-byte vectors: two 128-byte lines each
-  if (lane < 2) addr = p.k + qk_off + 64 * lane;
-  else if (lane < 4) addr = p.q + qk_off + 64 * (lane - 2);
-  else if (lane < 6 && role == 0) addr = p.v + bh * D + 64 * (lane - 4);
-  else if (GATE == LQ_GATE_DIAG && lane >= 6 && lane < 8) addr = p.alpha + bh * D + 64 * (lane - 6);
-  else if (GATE == LQ_GATE_SCALAR && lane >= 6 && lane < 8 && 32 * (lane - 6) < p.W)
-    addr = p.decays + bh * (size_t)p.W + 32 * (lane - 6);
-  if (addr) asm volatile("prefetch.global.L2 [%0];\n" ::"l"(addr));
 }
 
 // Persistent kernel of two-warp CTAs: CTA `blockIdx.x` takes heads blockIdx.x, blockIdx.x + gridDim.x, ...
@@ -273,15 +256,10 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
   load_scalars(blockIdx.x);
   TokenRaw nxt;                               // the token of the head about to start
   nxt.ba_lo = nxt.ba_hi = 1.0f;
-  HeadIdx hd{blockIdx.x, blockIdx.x / Hv, blockIdx.x % Hv};      // this head, the next one, and three ahead
-  HeadIdx hd1 = hd, hd3;
+  HeadIdx hd{blockIdx.x, blockIdx.x / Hv, blockIdx.x % Hv};      // this head and the next one
+  HeadIdx hd1 = hd;
   hd1.step(G, G_b, G_hv, Hv);
-  hd3 = hd1;
   if (hd.bh < nh) load_token<GATE>(p, hd, group, lane, role, nxt);
-  if (hd3.bh < nh) prefetch_token_l2<GATE>(p, hd3, group, lane, role);
-  hd3.step(G, G_b, G_hv, Hv);
-  if (hd3.bh < nh) prefetch_token_l2<GATE>(p, hd3, group, lane, role);
-  hd3.step(G, G_b, G_hv, Hv);
   {
     const int n0 = __shfl_sync(FULL, sc_n, 0) & 0xFFFF;
     if (role == 1 && blockIdx.x < nh && n0 < W) request(blockIdx.x, n0);
@@ -290,7 +268,7 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
   tick_ = clock64();
 #endif
   int idx = 0;                               // position of the head in this CTA's list
-  for (; hd.bh < nh; hd = hd1, hd1.step(G, G_b, G_hv, Hv), hd3.step(G, G_b, G_hv, Hv), idx++) {
+  for (; hd.bh < nh; hd = hd1, hd1.step(G, G_b, G_hv, Hv), idx++) {
     const size_t bh = hd.bh;
     const int n = __shfl_sync(FULL, sc_n, idx & 31) & 0xFFFF;
     const float beta = __uint_as_float(__shfl_sync(FULL, sc_beta, idx & 31) << 16);
@@ -301,7 +279,6 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
     const int n_next = bh_next < nh ? (__shfl_sync(FULL, sc_n, (idx + 1) & 31) & 0xFFFF) : W;
     const bool active = n < W, next_active = n_next < W;
     const int b = static_cast<int>(hd.b);
-    if (hd3.bh < nh) prefetch_token_l2<GATE>(p, hd3, group, lane, role);
     LQ_TICK(0);
 
     if (!active) {                           // nothing was requested for this head; keep the pipeline going
