@@ -200,24 +200,27 @@ __device__ __forceinline__ void quantize_tile(const Params &p, const BoundarySme
     }
     int sel;
     const float tot = row_tree(pr, t.lane, sel);
-    if (t.tx < 8) sm.vec[8 * t.ty + sel] = fmaxf(sqrtf(tot / static_cast<float>(D)), 1e-6f);
+    if (t.tx < 8) {                                           // one thread per row: c_i and 1 / c_i
+      const float ci = fmaxf(sqrtf(tot / static_cast<float>(D)), 1e-6f);
+      sm.vec[8 * t.ty + sel] = ci;
+      sm.colv[8 * t.ty + sel] = 1.0f / ci;
+    }
     __syncthreads();
     load8(sm.vec + 8 * t.ty, c);
+    if (t.tx == 0) store8(p.row_smooth(bh) + 8 * t.ty, c);
+    load8(sm.colv + 8 * t.ty, c);                             // from here on c holds 1 / c_i
+#pragma unroll
+    for (int a = 0; a < 8; a++) {
+#pragma unroll
+      for (int b = 0; b < 8; b++) M[a][b] = M[a][b] * c[a];
+    }
   } else {
 #pragma unroll
-    for (int a = 0; a < 8; a++) c[a] = 1.0f;
+    for (int a = 0; a < 8; a++) c[a] = 1.0f;                  // X = R / 1 = R
+    if (t.tx == 0) store8(p.row_smooth(bh) + 8 * t.ty, c);
   }
-  if (t.tx == 0) store8(p.row_smooth(bh) + 8 * t.ty, c);
-#pragma unroll
-  for (int a = 0; a < 8; a++) {
-    const float inv_c = 1.0f / c[a];
-#pragma unroll
-    for (int b = 0; b < 8; b++) M[a][b] = M[a][b] * inv_c;
-  }
-  // per-value-channel scale: column maximum of |X| (exact in any order)
-  float amax[8];
+  // per-value-channel scale: column maximum of |X| (exact in any order); one thread per column finishes it
   {
-    float4 q;
     float m[8];
 #pragma unroll
     for (int b = 0; b < 8; b++) {
@@ -226,44 +229,30 @@ __device__ __forceinline__ void quantize_tile(const Params &p, const BoundarySme
       for (int a = 1; a < 8; a++) s = fmaxf(s, fabsf(M[a][b]));
       m[b] = fmaxf(s, __shfl_xor_sync(FULL, s, 16));
     }
-    if (t.lane < 16) {
-      q = make_float4(m[0], m[1], m[2], m[3]);
-      *reinterpret_cast<float4 *>(sm.part + t.warp * D + 8 * t.tx) = q;
-      q = make_float4(m[4], m[5], m[6], m[7]);
-      *reinterpret_cast<float4 *>(sm.part + t.warp * D + 8 * t.tx + 4) = q;
+    if (t.lane < 16) store8(sm.part + t.warp * D + 8 * t.tx, m);
+    __syncthreads();
+    const int col = threadIdx.x;
+    if (col < D) {
+      float amax = sm.part[col];
+#pragma unroll
+      for (int wv = 1; wv < 8; wv++) amax = fmaxf(amax, sm.part[wv * D + col]);
+      p.col_scale(bh)[col] = amax / 127.0f;                   // stored as the step of the code, B_j / 127
+      sm.cs[col] = amax > 0.0f ? 127.0f / amax : 0.0f;
     }
     __syncthreads();
-#pragma unroll
-    for (int b = 0; b < 8; b++) amax[b] = 0.0f;
-#pragma unroll
-    for (int wv = 0; wv < 8; wv++) {
-      float x[8];
-      load8(sm.part + wv * D + 8 * t.tx, x);
-#pragma unroll
-      for (int b = 0; b < 8; b++) amax[b] = fmaxf(amax[b], x[b]);
-    }
-  }
-  if (t.ty == 0) {                                            // stored as the step of the code, B_j / 127
-    float step[8];
-#pragma unroll
-    for (int b = 0; b < 8; b++) step[b] = amax[b] / 127.0f;
-    store8(p.col_scale(bh) + 8 * t.tx, step);
   }
   float inv[8];
-#pragma unroll
-  for (int b = 0; b < 8; b++) inv[b] = amax[b] > 0.0f ? 127.0f / amax[b] : 0.0f;
+  load8(sm.cs + 8 * t.tx, inv);
   int8_t *ZT = p.codes(bh);
 #pragma unroll
   for (int b = 0; b < 8; b++) {
-    uint32_t w2[2] = {0u, 0u};
+    // |X * inv| <= 127 (1 + 2^-23), so the nearest integer (ties to even) is already inside [-127, 127]
+    int z[8];
 #pragma unroll
-    for (int a = 0; a < 8; a++) {
-      float zf = rintf(M[a][b] * inv[b]);                     // ties to even
-      zf = fminf(fmaxf(zf, -127.0f), 127.0f);
-      const uint32_t byte = static_cast<uint32_t>(static_cast<int>(zf)) & 0xFFu;
-      w2[a >> 2] |= byte << (8 * (a & 3));
-    }
-    *reinterpret_cast<uint2 *>(ZT + (8 * t.tx + b) * D + 8 * t.ty) = make_uint2(w2[0], w2[1]);
+    for (int a = 0; a < 8; a++) z[a] = __float2int_rn(M[a][b] * inv[b]);
+    const uint32_t lo = __byte_perm(__byte_perm(z[0], z[1], 0x0040), __byte_perm(z[2], z[3], 0x0040), 0x5410);
+    const uint32_t hi = __byte_perm(__byte_perm(z[4], z[5], 0x0040), __byte_perm(z[6], z[7], 0x0040), 0x5410);
+    *reinterpret_cast<uint2 *>(ZT + (8 * t.tx + b) * D + 8 * t.ty) = make_uint2(lo, hi);
   }
 }
 
