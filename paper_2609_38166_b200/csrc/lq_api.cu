@@ -20,35 +20,57 @@ __global__ void __launch_bounds__(256, 2) boundary_kernel(const Params p) {
   const BoundarySmem sm(reinterpret_cast<float *>(lq_smem4), p.W, p.r, GATE == LQ_GATE_DIAG);
   const Tile t;
   const size_t nh = (size_t)p.batch * p.heads_v;
-  for (size_t bh = blockIdx.x; bh < nh; bh += gridDim.x) {
-    const int b = static_cast<int>(bh / p.heads_v);
-    int n = 0;
-    if (MODE != 1) {
-      n = p.win_pos[b] & 0xFFFF;
-      if (MODE == 0 && !(n == p.W || (p.force && n > 0))) continue;
-      if (n > p.W) n = p.W;
+  __shared__ uint32_t todo[2];
+  // The CTA owns heads blockIdx.x + k * gridDim.x.  Warp 0 looks at 32 of them at a time (one load each, all in
+  // flight together) and publishes which ones have work; then the CTA handles those one after the other.
+  for (size_t base = blockIdx.x; base < nh; base += 32 * (size_t)gridDim.x) {
+    int n_mine = 0;
+    if (t.warp == 0) {
+      const size_t cand = base + t.lane * (size_t)gridDim.x;
+      bool want = false;
+      if (cand < nh) {
+        if (MODE != 1) n_mine = p.win_pos[cand / p.heads_v] & 0xFFFF;
+        want = MODE != 0 || n_mine == p.W || (p.force && n_mine > 0);
+      }
+      const uint32_t m = __ballot_sync(FULL, want);
+      if (t.lane == 0) todo[0] = m;
     }
-    float M[8][8];
-    if (MODE == 1) {
-      const float *S = p.S + bh * (size_t)(D * D);
-#pragma unroll
-      for (int a = 0; a < 8; a++) load8(S + (8 * t.ty + a) * D + 8 * t.tx, M[a]);
-    } else {
-      __syncthreads();                       // the previous head's use of shared memory is over
-      reconstruct_tile<GATE>(p, sm, t, bh, n, M);
-    }
-    if (MODE == 2) {
-      float *S = p.S + bh * (size_t)(D * D);
-#pragma unroll
-      for (int a = 0; a < 8; a++) store8(S + (8 * t.ty + a) * D + 8 * t.tx, M[a]);
-      continue;
-    }
-    quantize_tile(p, sm, t, bh, M);
     __syncthreads();
-    if (t.tid == 0) {
-      if (MODE == 0) arrive_and_set(p.win_pos, b, p.heads_v, 0);
-      else p.win_pos[b] = 0;                 // nobody reads win_pos in this mode
+    uint32_t mask = todo[0];
+    while (mask) {
+      const int kbit = __ffs(mask) - 1;
+      mask &= mask - 1;
+      const size_t bh = base + kbit * (size_t)gridDim.x;
+      const int b = static_cast<int>(bh / p.heads_v);
+      int n = 0;
+      if (MODE != 1) {
+        if (t.warp == 0) { n = __shfl_sync(FULL, n_mine, kbit); if (t.lane == 0) todo[1] = n; }
+        __syncthreads();                     // also: the previous head's use of shared memory is over
+        n = todo[1];
+        if (n > p.W) n = p.W;
+      }
+      float M[8][8];
+      if (MODE == 1) {
+        const float *S = p.S + bh * (size_t)(D * D);
+#pragma unroll
+        for (int a = 0; a < 8; a++) load8(S + (8 * t.ty + a) * D + 8 * t.tx, M[a]);
+      } else {
+        reconstruct_tile<GATE>(p, sm, t, bh, n, M);
+      }
+      if (MODE == 2) {
+        float *S = p.S + bh * (size_t)(D * D);
+#pragma unroll
+        for (int a = 0; a < 8; a++) store8(S + (8 * t.ty + a) * D + 8 * t.tx, M[a]);
+        continue;
+      }
+      quantize_tile(p, sm, t, bh, M);
+      __syncthreads();
+      if (t.tid == 0) {
+        if (MODE == 0) arrive_and_set(p.win_pos, b, p.heads_v, 0);
+        else p.win_pos[b] = 0;                 // nobody reads win_pos in this mode
+      }
     }
+    __syncthreads();                         // todo[] is rewritten by the next round
   }
 }
 
