@@ -65,7 +65,10 @@ typedef struct {
   int d_k, d_v; /* state is d_k x d_v                                             */
   int W;        /* window length (the paper's p)                                  */
   int r;        /* Compensator Tokens per state                                   */
-  int n_iter;   /* power-iteration steps per Compensator Token at a boundary      */
+  int n_iter;   /* power-iteration steps per Compensator Token at a boundary (2 is  */
+                /* the default of the binding); compensator h starts from the u of  */
+                /* the (h+1)-th newest buffered record, scaled to unit length, or   */
+                /* from the all-equal unit vector where there is no such record     */
   int gate;     /* lq_gate                                                        */
   int smooth;   /* 1: residual smoothing (Sec. 3.4); 0: c = 1 (ablation)          */
 } lq_shape;

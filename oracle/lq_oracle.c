@@ -360,8 +360,15 @@ static void head_reconstruct(const lqo_shape *sh, const head_view *hv, int n, fl
 /*   that are actually stored (fp16);                                   */
 /*   smoothing scales c, Sec. 3.4 (square root of the row mean |.|);    */
 /*   per-value-channel symmetric 8-bit codes, Appendix B.3.             */
+/* The paper does not say where the power iteration starts.  Here the   */
+/* iteration for component h starts from the value side u of the        */
+/* (h+1)-th newest buffered record, scaled to unit length (the newest   */
+/* records dominate the state that is being fitted); where there is no  */
+/* such record, or it is (numerically) zero, from the vector with all   */
+/* entries equal.  `starts` holds `nstarts` rows of d_v floats, oldest  */
+/* first (the u part of the record buffer), or is NULL.                 */
 /* ------------------------------------------------------------------ */
-static void head_quantize(const lqo_shape *sh, float *M, const head_view *hv) {
+static void head_quantize(const lqo_shape *sh, float *M, const head_view *hv, const float *starts, int nstarts) {
   int K = sh->d_k, V = sh->d_v;
   float *w = (float *)malloc(sizeof(float) * V), *t = (float *)malloc(sizeof(float) * K);
   float *col = (float *)malloc(sizeof(float) * K);
@@ -370,6 +377,14 @@ static void head_quantize(const lqo_shape *sh, float *M, const head_view *hv) {
   for (int h = 0; h < sh->r; h++) {
     int vanished = 0;
     for (int j = 0; j < V; j++) w[j] = 1.0f / sqrtf((float)V);
+    if (starts && h < nstarts) {
+      const float *u = starts + (size_t)(nstarts - 1 - h) * V;
+      float nu0 = lqo_csum_dot(u, u, V);
+      if (nu0 >= 1e-30f) {
+        float s0 = 1.0f / sqrtf(nu0);
+        for (int j = 0; j < V; j++) w[j] = u[j] * s0;
+      }
+    }
     for (int it = 0; it < sh->n_iter; it++) {
       for (int i = 0; i < K; i++) t[i] = lqo_csum_dot(M + (size_t)i * V, w, V);      /* t = M w      */
       float nu = lqo_csum_dot(t, t, K);
@@ -425,7 +440,7 @@ static void head_flush(const lqo_shape *sh, const head_view *hv, int n) {
   float *S = (float *)malloc(sizeof(float) * (size_t)K * V);
   head_reconstruct(sh, hv, n, S);
   if (hv->S0) memcpy(hv->S0, S, sizeof(float) * (size_t)K * V);
-  else head_quantize(sh, S, hv);
+  else head_quantize(sh, S, hv, hv->bu, n);
   free(S);
 }
 
@@ -583,7 +598,7 @@ int lqo_quantize_state(const lqo_shape *sh, const float *S, lqo_state *st) {
     if (hv.S0) { memcpy(hv.S0, S + (size_t)bh * KV, sizeof(float) * KV); continue; }
     float *M = (float *)malloc(sizeof(float) * KV);
     memcpy(M, S + (size_t)bh * KV, sizeof(float) * KV);
-    head_quantize(sh, M, &hv);
+    head_quantize(sh, M, &hv, NULL, 0);
     free(M);
   }
   for (int b = 0; b < sh->batch; b++) st->win_pos[b] = 0;

@@ -54,7 +54,7 @@ class Shape:
     d_v: int
     W: int
     r: int = 4
-    n_iter: int = 3
+    n_iter: int = 2
     gate: int = GATE_SCALAR
     smooth: int = 1
 

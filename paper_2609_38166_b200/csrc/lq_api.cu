@@ -63,7 +63,7 @@ __global__ void __launch_bounds__(256, 2) boundary_kernel(const Params p) {
         for (int a = 0; a < 8; a++) store8(S + (8 * t.ty + a) * D + 8 * t.tx, M[a]);
         continue;
       }
-      quantize_tile(p, sm, t, bh, M);
+      quantize_tile(p, sm, t, bh, MODE == 0 ? n : 0, M);
       __syncthreads();
       if (t.tid == 0) {
         if (MODE == 0) arrive_and_set(p.win_pos, b, p.heads_v, 0);

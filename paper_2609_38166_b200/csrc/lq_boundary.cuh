@@ -122,8 +122,10 @@ __device__ __forceinline__ void reconstruct_tile(const Params &p, const Boundary
 
 // Quantize the dense state held in M (destroyed) and write codes, scales and compensators of head bh.
 // Uses sm.vec and sm.part; begins with a barrier so that it may follow any other use of shared memory.
+// The power iteration of compensator h starts from the value side u of the (h+1)-th newest of the n records in
+// sm.bu, scaled to unit length; from the all-equal unit vector where there is no such record or it is zero.
 __device__ __forceinline__ void quantize_tile(const Params &p, const BoundarySmem &sm, const Tile &t, size_t bh,
-                                              float (&M)[8][8]) {
+                                              int n, float (&M)[8][8]) {
   const int r = p.r;
   __syncthreads();
   int h = 0;
@@ -132,6 +134,16 @@ __device__ __forceinline__ void quantize_tile(const Params &p, const BoundarySme
     const float w0 = 1.0f / sqrtf(static_cast<float>(D));
 #pragma unroll
     for (int b = 0; b < 8; b++) w[b] = w0;
+    if (h < n) {
+      const float *u = sm.bu + (n - 1 - h) * D;
+      const float nu0 = dot128_shared(u, u, t.lane & 15);     // same value in every thread
+      if (nu0 >= 1e-30f) {
+        const float s0 = 1.0f / sqrtf(nu0);
+        load8(u + 8 * t.tx, w);
+#pragma unroll
+        for (int b = 0; b < 8; b++) w[b] = w[b] * s0;
+      }
+    }
     bool vanished = false;
     for (int it = 0; it < p.n_iter; it++) {
       float pr[8];

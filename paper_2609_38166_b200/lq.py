@@ -71,7 +71,7 @@ class Shape:
     d_v: int = 128
     W: int = 16
     r: int = 4
-    n_iter: int = 3
+    n_iter: int = 2
     gate: int = GATE_SCALAR
     smooth: int = 1
 

@@ -43,7 +43,7 @@ class Workload:
     d_v: int = 128
     W: int = 16
     r: int = 4
-    n_iter: int = 3
+    n_iter: int = 2
     gate: int = GATE_SCALAR
     smooth: int = 1
     v_dist: str = "normal"          # "normal" | "student3"

@@ -190,3 +190,57 @@ def test_format_size_matches_the_paper():
     # this build buffers records in fp32; the paper's fp16 figure is half of ours
     rec = st.buf_k.nbytes + st.buf_u.nbytes + st.buf_a.nbytes
     assert rec // 2 == gold["fp16_buffer_bytes_p16_gdn"]
+
+
+@pytest.mark.parametrize("gate", [synth.GATE_SCALAR, synth.GATE_DIAG])
+def test_flush_fit_from_record_start_vectors_reaches_the_optimum(oracle, gate):
+    """At a window boundary the power iteration of compensator h starts from the (h+1)-th newest record's u
+    instead of the all-equal vector.  Whatever the start, with enough steps the fit of Eqs. 5-6 must end at
+    the Eckart-Young optimum of the state that the window representation holds (Eq. 7), here computed by a
+    library SVD of the dequantized pre-flush state."""
+    rng = np.random.default_rng(17)
+    B, H, K, V, W, r = 1, 2, 128, 128, 6, 3
+    sh = Shape(B, H, H, K, V, W, r, 80, gate, 0)
+    st = State(sh)
+    oracle.quantize_state(sh, np.zeros((B, H, K, V), np.float32), st)
+    # six records with well separated weights: the state is their decayed sum, rank 6 with a gapped spectrum
+    wts = np.array([0.6, 4.0, 0.3, 9.0, 1.5, 0.1])[None, None, :, None]
+    qk, _ = np.linalg.qr(rng.standard_normal((H, K, W)))
+    qu, _ = np.linalg.qr(rng.standard_normal((H, V, W)))
+    st.buf_k[...] = (qk.transpose(0, 2, 1)[None] * wts).astype(np.float32)
+    st.buf_u[...] = qu.transpose(0, 2, 1)[None].astype(np.float32)
+    st.buf_a[...] = rng.uniform(0.8, 1.0, st.buf_a.shape).astype(np.float32)
+    st.win_pos[...] = W
+    Sp = oracle.dequantize_state(sh, st).astype(np.float64)
+    oracle.window_flush(sh, st)
+    assert st.win_pos[0] == 0
+    for h in range(H):
+        kc = st.comp_k_f32()[0, h].astype(np.float64)
+        uc = st.comp_u_f32()[0, h].astype(np.float64)
+        sv = np.linalg.svd(Sp[0, h], compute_uv=False)
+        best = np.sqrt((sv[r:] ** 2).sum())
+        resid = np.linalg.norm(Sp[0, h] - kc.T @ uc)
+        assert resid <= best * (1 + 2e-3) + 2.0 ** -10 * np.sqrt((sv[:r] ** 2).sum())
+        assert resid >= best * (1 - 1e-6)
+
+
+def test_record_start_vector_is_what_the_first_step_multiplies(oracle):
+    """One power-iteration step from start vector w gives k = S w / |S w|.  With a single record whose u is
+    orthogonal to everything else in the state, S u_newest is along that record's key: the first compensator
+    key after one step must be that (decayed) key direction, which the all-equal start would not give."""
+    rng = np.random.default_rng(5)
+    B, H, K, V, W = 1, 1, 128, 128, 4
+    sh = Shape(B, H, H, K, V, W, 1, 1, synth.GATE_SCALAR, 0)
+    st = State(sh)
+    oracle.quantize_state(sh, np.zeros((B, H, K, V), np.float32), st)
+    q, _ = np.linalg.qr(rng.standard_normal((V, W)))
+    keys = rng.standard_normal((W, K)); keys /= np.linalg.norm(keys, axis=1, keepdims=True)
+    st.buf_k[0, 0] = keys.astype(np.float32)
+    st.buf_u[0, 0] = (q.T * np.array([5.0, 3.0, 2.0, 0.05])[:, None]).astype(np.float32)   # newest one is small
+    st.buf_a[...] = 1.0
+    st.win_pos[...] = W
+    oracle.window_flush(sh, st)
+    k1 = st.comp_k_f32()[0, 0, 0].astype(np.float64)
+    # S u_3 = sum_j k_j (u_j . u_3) = k_3 |u_3|^2 : the newest record's key, although it is the weakest one
+    assert abs(abs(k1 @ keys[3]) - 1.0) < 2e-3
+    assert abs(k1 @ keys[0]) < 0.5
