@@ -21,6 +21,9 @@ __global__ void __launch_bounds__(256, 2) boundary_kernel(const Params p) {
   const Tile t;
   const size_t nh = (size_t)p.batch * p.heads_v;
   __shared__ uint32_t todo[2];
+#ifdef LQ_TIMING
+  if (threadIdx.x == 0) { for (int i = 0; i < 16; i++) lq_bacc[i] = 0; lq_btick = clock64(); }
+#endif
   // The CTA owns heads blockIdx.x + k * gridDim.x.  Warp 0 looks at 32 of them at a time (one load each, all in
   // flight together) and publishes which ones have work; then the CTA handles those one after the other.
   for (size_t base = blockIdx.x; base < nh; base += 32 * (size_t)gridDim.x) {
@@ -36,6 +39,7 @@ __global__ void __launch_bounds__(256, 2) boundary_kernel(const Params p) {
       if (t.lane == 0) todo[0] = m;
     }
     __syncthreads();
+    LQ_BTICK(0);
     uint32_t mask = todo[0];
     while (mask) {
       const int kbit = __ffs(mask) - 1;
@@ -65,6 +69,7 @@ __global__ void __launch_bounds__(256, 2) boundary_kernel(const Params p) {
       }
       quantize_tile(p, sm, t, bh, MODE == 0 ? n : 0, M);
       __syncthreads();
+      LQ_BTICK(9);
       if (t.tid == 0) {
         if (MODE == 0) arrive_and_set(p.win_pos, b, p.heads_v, 0);
         else p.win_pos[b] = 0;                 // nobody reads win_pos in this mode
@@ -72,6 +77,11 @@ __global__ void __launch_bounds__(256, 2) boundary_kernel(const Params p) {
     }
     __syncthreads();                         // todo[] is rewritten by the next round
   }
+#ifdef LQ_TIMING
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 16; i++) atomicAdd(&g_phase_cycles[32 + i], (unsigned long long)lq_bacc[i]);
+  }
+#endif
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -475,7 +485,7 @@ lq_status lq_check_device(int *flags) {
 #ifdef LQ_TIMING
 // development aid: copies the phase counters to host memory and clears them
 int lq_debug_phase_cycles(unsigned long long *out) {
-  unsigned long long zero[32] = {0};
+  unsigned long long zero[64] = {0};
   if (cudaMemcpyFromSymbol(out, g_phase_cycles, sizeof(zero)) != cudaSuccess) return 1;
   return cudaMemcpyToSymbol(g_phase_cycles, zero, sizeof(zero)) != cudaSuccess;
 }

@@ -70,17 +70,33 @@ __device__ __forceinline__ void reconstruct_tile(const Params &p, const Boundary
     cp_async_wait_all();
   }
   __syncthreads();
+  LQ_BTICK(1);
   // cumulative decays, newest record first (Appendix B.2): kd_j = Gamma_{j+1:n} kt_j, gam = Gamma_{1:n}
   if (t.tid < D) {
     const int i = t.tid;
     float g = 1.0f;
-    for (int j = n - 1; j >= 0; j--) {
+    int j = n - 1;
+    for (; j >= 3; j -= 4) {                                  // four records per trip: the loads go out together
+      float kt[4], a[4];
+#pragma unroll
+      for (int e = 0; e < 4; e++) {
+        kt[e] = sm.kd[(j - e) * D + i];
+        a[e] = GATE == LQ_GATE_DIAG ? sm.ba[(j - e) * D + i] : sm.ba[j - e];
+      }
+#pragma unroll
+      for (int e = 0; e < 4; e++) {
+        sm.kd[(j - e) * D + i] = g * kt[e];
+        g = g * a[e];
+      }
+    }
+    for (; j >= 0; j--) {
       sm.kd[j * D + i] = g * sm.kd[j * D + i];
       g = g * (GATE == LQ_GATE_DIAG ? sm.ba[j * D + i] : sm.ba[j]);
     }
     sm.gam[i] = g;
   }
   __syncthreads();
+  LQ_BTICK(2);
 
   float ci[8], gi[8], sj[8];
   load8(sm.cs + 8 * t.ty, ci);
@@ -118,6 +134,7 @@ __device__ __forceinline__ void reconstruct_tile(const Params &p, const Boundary
 #pragma unroll
       for (int b = 0; b < 8; b++) M[a][b] = fmaf(kj[a], uj[b], M[a][b]);
   }
+  LQ_BTICK(3);
 }
 
 // Quantize the dense state held in M (destroyed) and write codes, scales and compensators of head bh.
@@ -192,6 +209,7 @@ __device__ __forceinline__ void quantize_tile(const Params &p, const BoundarySme
 #pragma unroll
       for (int b = 0; b < 8; b++) M[a][b] = fmaf(-kf[a], uf[b], M[a][b]);
   }
+  LQ_BTICK(4);
   // a vanished component means nothing is left to fit: this and all later compensators are zero
   for (; h < r; h++) {
     if (t.tx == 0) *reinterpret_cast<uint4 *>(p.comp_k(bh) + h * D + 8 * t.ty) = make_uint4(0, 0, 0, 0);
@@ -220,6 +238,7 @@ __device__ __forceinline__ void quantize_tile(const Params &p, const BoundarySme
     __syncthreads();
     load8(sm.vec + 8 * t.ty, c);
     if (t.tx == 0) store8(p.row_smooth(bh) + 8 * t.ty, c);
+    LQ_BTICK(5);
     load8(sm.colv + 8 * t.ty, c);                             // from here on c holds 1 / c_i
 #pragma unroll
     for (int a = 0; a < 8; a++) {
@@ -253,6 +272,7 @@ __device__ __forceinline__ void quantize_tile(const Params &p, const BoundarySme
     }
     __syncthreads();
   }
+  LQ_BTICK(6);
   float inv[8];
   load8(sm.cs + 8 * t.tx, inv);
   int8_t *ZT = p.codes(bh);

@@ -118,6 +118,34 @@ __device__ __forceinline__ float dot128_shared(const float *a, const float *b, i
   return tree16(block8(a2, b2));
 }
 
+// Phase timing (development aid, compiled in with -DLQ_TIMING only): clock cycles per phase of the decode
+// warps, summed over all heads by lane 0 of each warp (slots 0..15: stream warp, 16..31: dot warp; 32..: thread 0 of the boundary kernel's CTAs).
+#ifdef LQ_TIMING
+__device__ unsigned long long g_phase_cycles[64];
+// cycles are summed in registers and flushed once per warp at the end of the kernel, so that the probe
+// itself puts no traffic on the memory system while the kernel runs
+#define LQ_TICK(slot)                                     \
+  do {                                                    \
+    const long long now_ = clock64();                     \
+    acc_[slot] += static_cast<unsigned>(now_ - tick_);    \
+    tick_ = now_;                                         \
+  } while (0)
+// the boundary kernel's variant: thread 0 of the CTA keeps its sums in shared memory
+__shared__ unsigned lq_bacc[16];
+__shared__ long long lq_btick;
+#define LQ_BTICK(slot)                                          \
+  do {                                                          \
+    if (threadIdx.x == 0) {                                     \
+      const long long now_ = clock64();                         \
+      lq_bacc[slot] += static_cast<unsigned>(now_ - lq_btick);  \
+      lq_btick = now_;                                          \
+    }                                                           \
+  } while (0)
+#else
+#define LQ_TICK(slot) do { } while (0)
+#define LQ_BTICK(slot) do { } while (0)
+#endif
+
 // =====================================================================================
 // 8x8 register tiles: a CTA of 256 threads holds one 128x128 state, thread (ty, tx) owning rows
 // 8ty..8ty+7 and columns 8tx..8tx+7, with tx = lane & 15 and ty = 2*warp + (lane >> 4).

@@ -34,22 +34,6 @@ namespace lq {
 // Set when a bounded wait gave up (bit 0: a decode warp's wait for its bulk copies).  Never cleared by kernels.
 __device__ int g_device_error = 0;
 
-// Phase timing (development aid, compiled in with -DLQ_TIMING only): clock cycles per phase of the decode
-// warps, summed over all heads by lane 0 of each warp (slots 0..15: stream warp, 16..31: dot warp).
-#ifdef LQ_TIMING
-__device__ unsigned long long g_phase_cycles[32];
-// cycles are summed in registers and flushed once per warp at the end of the kernel, so that the probe
-// itself puts no traffic on the memory system while the kernel runs
-#define LQ_TICK(slot)                                     \
-  do {                                                    \
-    const long long now_ = clock64();                     \
-    acc_[slot] += static_cast<unsigned>(now_ - tick_);    \
-    tick_ = now_;                                         \
-  } while (0)
-#else
-#define LQ_TICK(slot) do { } while (0)
-#endif
-
 // ---- shared-memory slot of one CTA ----
 struct DecodeSlot {
   // byte offsets inside the slot; every region starts on a 16-byte boundary
