@@ -35,6 +35,19 @@ WARM_TOKENS = 512
 STATE_BYTES = 128 * 128 + 4 * 128 + 4 * 128 + 2 * 4 * (128 + 128)       # 19456 per head at r = 4
 METRIC = "GDN decode state-GB/s at bs256 (8-bit per-window state, W=16, r=4)"
 
+
+def state_bytes(r: int) -> int:
+    """Bytes of the quantized state of one head: codes, two fp32 scale vectors, r fp16 compensator pairs."""
+    return 128 * 128 + 4 * 128 + 4 * 128 + 2 * r * (128 + 128)
+
+
+def metric_name(wl) -> str:
+    """The headline metric's name; other shapes (flags --gate/--batch/--W/--r) are named after themselves."""
+    if wl.gate == synth.GATE_SCALAR and wl.batch == 256 and wl.W == 16 and wl.r == 4:
+        return METRIC
+    return "%s decode state-GB/s at bs%d (8-bit per-window state, W=%d, r=%d)" % (
+        "GDN" if wl.gate == synth.GATE_SCALAR else "KDA", wl.batch, wl.W, wl.r)
+
 # DRAM bytes per launch from the ncu captures summarised under profiles/ (dram__bytes_read.sum +
 # dram__bytes_write.sum of one full-batch launch of the gdn_b256 workload, W = 16), or None when not captured.
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {"decode_kernel": 238.2e6, "boundary_kernel": 18.4e6}
@@ -60,7 +73,7 @@ def config_dict(wl, world: int, warm_tokens: int) -> dict:
             "state_dtype": "int8 + fp32 scales + fp16 compensators", "record_buffer_dtype": "f32",
             "inputs_dtype": "bf16", "warmup_tokens": warm_tokens, "window_offsets": "uniform over [0,W)",
             "l2": "working set %.0f MB per step exceeds the 126 MB L2; no flush needed" %
-                  (heads * (STATE_BYTES + wl.W * 1028) / 1e6),
+                  (heads * (state_bytes(wl.r) + wl.W * (1028 if wl.gate == synth.GATE_SCALAR else 1536)) / 1e6),
             "parallelism": "dp%d (independent batches, no collective)" % world}
 
 
@@ -79,9 +92,9 @@ def max_over_ranks(value_ms: float, dist_mod=None, device=None) -> float:
     return float(t.item())
 
 
-def whole_job_value(heads_per_rank: int, world: int, steps: int, ms: float) -> float:
+def whole_job_value(heads_per_rank: int, world: int, steps: int, ms: float, r: int = 4) -> float:
     """state-GB/s of the whole job: all ranks' head-steps over the slowest rank's time."""
-    return world * heads_per_rank * steps / (ms / 1e3) * STATE_BYTES / 1e9
+    return world * heads_per_rank * steps / (ms / 1e3) * state_bytes(r) / 1e9
 
 
 def peaks():
@@ -195,8 +208,8 @@ def run_reference(args, wl):
     if rank != 0:
         return
     hs, cores, sample, s_per_step = time_oracle(wl, args.steps, args.warmup, budget_s=150.0)
-    value = hs * STATE_BYTES / 1e9
-    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": args.gpus,
+    value = hs * state_bytes(wl.r) / 1e9
+    line = {"impl": "reference", "metric": metric_name(wl), "value": value, "unit": "GB/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": s_per_step * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "tokens_heads_per_s": hs,
@@ -358,7 +371,7 @@ def run_cuda(args, wl):
         e2e_ms = e0.elapsed_time(e1)
         e2e_ms = max_over_ranks(e2e_ms, dist if world > 1 else None, "cuda")
         h2d = sum(v.numel() * v.element_size() for v in pin[0].values())
-        e2e = {"value": whole_job_value(wl.batch * wl.heads_v, world, n_e2e, e2e_ms), "unit": "GB/s",
+        e2e = {"value": whole_job_value(wl.batch * wl.heads_v, world, n_e2e, e2e_ms, wl.r), "unit": "GB/s",
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": o_h.numel() * 4, "steps": n_e2e,
                "ms_per_step": e2e_ms / n_e2e,
                "api": "lq_decode_step_host (pinned host q,k,v,beta,alpha in; o out), one call per step"}
@@ -402,8 +415,8 @@ def run_cuda(args, wl):
     rec = 4 * (256 + g)
     # what each kernel has to move per launch: the decode kernel everything but the boundary; the boundary
     # kernel, for the 1/W of the heads whose window is full, the window representation in and the head block out
-    decode_bytes = heads * (bytes_hs - (2 * STATE_BYTES + wl.W * rec) / wl.W)
-    boundary_bytes = heads / wl.W * (2 * STATE_BYTES + wl.W * rec)
+    decode_bytes = heads * (bytes_hs - (2 * state_bytes(wl.r) + wl.W * rec) / wl.W)
+    boundary_bytes = heads / wl.W * (2 * state_bytes(wl.r) + wl.W * rec)
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": None, "peak_source": peak_src,
                 "kernel": "one step = decode_kernel + boundary_kernel (algorithmic bytes of both over the step time "
@@ -456,10 +469,10 @@ def run_cuda(args, wl):
     cpu = None
     if not args.only_timed:
         hs_cpu, cores, sample, _ = time_oracle(wl.with_(seed=wl.seed), steps=8 * wl.W, warmup=2, budget_s=25.0)
-        cpu = {"value": hs_cpu * STATE_BYTES / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
+        cpu = {"value": hs_cpu * state_bytes(wl.r) / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
                "sample": sample, "tokens_heads_per_s": hs_cpu}
 
-    line = {"metric": METRIC, "value": hs * STATE_BYTES / 1e9, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+    line = {"metric": metric_name(wl), "value": hs * state_bytes(wl.r) / 1e9, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": config_dict(wl, world, args.warm_tokens),
@@ -471,6 +484,117 @@ def run_cuda(args, wl):
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+# --------------------------------------------------------------------------------------------------
+# Throughput sweep: GDN and KDA, batch x W x r, uniform window offsets; one JSON line per point
+# --------------------------------------------------------------------------------------------------
+def run_sweep(args):
+    import torch
+    from paper_2609_38166_b200 import build, lq
+
+    log = lambda m: print(f"[sweep] {m}", file=sys.stderr, flush=True)
+    torch.cuda.set_device(0)
+    build.build()
+    lq.lib()
+    peak, peak_src = peaks()
+    l2 = torch.cuda.get_device_properties(0).L2_cache_size
+    stream = torch.cuda.current_stream()
+    batches = [int(x) for x in args.sweep_batches.split(",")]
+    windows = [int(x) for x in args.sweep_W.split(",")]
+    ranks = [int(x) for x in args.sweep_r.split(",")]
+    gates = [g for g in args.sweep_gates.split(",")]
+    warm = max(windows) + 8
+    rows = []
+    for gate_name in gates:
+        diag = gate_name == "kda"
+        for B in batches:
+            base_wl = synth.Workload(f"sweep_{gate_name}", B, 32, 32 if diag else 16, 128, 128, 16, 4,
+                                     gate=synth.GATE_DIAG if diag else synth.GATE_SCALAR, seed=5)
+            cache = {}
+
+            def tok(t, base_wl=base_wl, cache=cache):
+                if t not in cache:
+                    cache[t] = to_dev(synth.token_inputs(base_wl, t), torch)
+                return cache[t]
+
+            def timed(fn, nrep, cycle):
+                for t in range(cycle + 3):                     # also draws every token of the cycle (CPU work)
+                    fn(t)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                e0.record(stream)
+                for t in range(nrep):
+                    fn(t)
+                e1.record(stream)
+                torch.cuda.synchronize()
+                return e0.elapsed_time(e1) / nrep
+
+            # the two dense-state baselines of this (gate, batch)
+            sh0 = lq.Shape(B, 32, base_wl.heads_qk, 128, 128, 16, 4, 2, base_wl.gate, 1)
+            o = torch.empty((B, 32, 128), dtype=torch.float32, device="cuda")
+            S = torch.zeros((B, 32, 128, 128), dtype=torch.float32, device="cuda")
+            ms32 = timed(lambda t: lq.ref_decode_step_f32(sh0, S, *[tok(t % 16)[k] for k in
+                                                                    ("q", "k", "v", "beta", "alpha")], o), 100, 16)
+            del S
+            S16 = torch.zeros((B, 32, 128, 128), dtype=torch.int16, device="cuda")
+            ms16 = timed(lambda t: lq.ref_decode_step_bf16(sh0, S16, *[tok(t % 16)[k] for k in
+                                                                       ("q", "k", "v", "beta", "alpha")], o), 100, 16)
+            del S16
+            for W in windows:
+                for r in ranks:
+                    wl = base_wl.with_(W=W, r=r)
+                    # same staggering as the headline run, with a short pre-fill (speed does not depend on it)
+                    sh = lq.Shape(B, 32, wl.heads_qk, 128, 128, W, r, wl.n_iter, wl.gate, 1)
+                    st = lq.State(sh)
+                    S = torch.zeros((B, 32, 128, 128), dtype=torch.float32, device="cuda")
+                    per = max(B // W, 1)
+                    groups = (B + per - 1) // per
+                    for t in range(warm + 1):
+                        g = warm - t
+                        b_lq = B
+                        if g < groups:
+                            lo, hi = g * per, (B if g == groups - 1 else (g + 1) * per)
+                            lq.quantize_state(sh, S, st, b0=lo, nb=hi - lo)
+                            b_lq = lo
+                        if t == warm:
+                            break
+                        d = tok(t)
+                        if b_lq > 0:
+                            lq.ref_decode_step_f32(sh, S, d["q"], d["k"], d["v"], d["beta"], d["alpha"], o, b0=0,
+                                                   nb=b_lq)
+                        if b_lq < B:
+                            lq.decode_step(sh, st, d["q"], d["k"], d["v"], d["beta"], d["alpha"], o, b0=b_lq,
+                                           nb=B - b_lq)
+                    del S
+                    nrep = max(args.sweep_steps // W, 1) * W      # every sequence flushes the same number of times
+                    ms = timed(lambda t: lq.decode_step(sh, st, *[tok(warm + t % W)[k] for k in
+                                                                  ("q", "k", "v", "beta", "alpha")], o, stream), nrep, W)
+                    flags = lq.check_device()
+                    heads = B * 32
+                    bytes_hs = algorithmic_bytes_per_head_step(W, r, diag, wl.heads_v // wl.heads_qk, False)
+                    foot = st.heads.numel() + st.records.numel() * 4
+                    state_b = 128 * 128 + 4 * 128 + 4 * 128 + 2 * r * 256
+                    row = {"sweep": True, "gate": gate_name, "batch": B, "W": W, "r": r, "n_iter": wl.n_iter,
+                           "steps": nrep, "ms_per_step": ms, "tokens_heads_per_s": heads / (ms / 1e3),
+                           "state_GBps": heads * state_b / (ms / 1e3) / 1e9,
+                           "total_GBps": heads * bytes_hs / (ms / 1e3) / 1e9,
+                           "pct_hbm_peak_measured": 100 * heads * bytes_hs / (ms / 1e3) / 1e9 / peak,
+                           "speedup_vs_fp32_state": ms32 / ms, "speedup_vs_bf16_state": ms16 / ms,
+                           "fp32_state_ms": ms32, "bf16_state_ms": ms16,
+                           "l2": "L2-resident (window representation %.0f MB < 2 x %.0f MB L2)" % (foot / 1e6, l2 / 1e6)
+                                 if foot < 2 * l2 else "exceeds L2", "device_error_flags": flags}
+                    rows.append(row)
+                    print(json.dumps(row), flush=True)
+                    del st
+            cache.clear()
+            torch.cuda.empty_cache()
+    log("gate  batch   W   r   us/step   state GB/s  total GB/s  %peak   x fp32   x bf16")
+    for x in rows:
+        log(f"{x['gate']:4s} {x['batch']:6d} {x['W']:3d} {x['r']:3d} {1e3 * x['ms_per_step']:9.1f} "
+            f"{x['state_GBps']:11.0f} {x['total_GBps']:11.0f} {x['pct_hbm_peak_measured']:6.1f} "
+            f"{x['speedup_vs_fp32_state']:8.2f} {x['speedup_vs_bf16_state']:8.2f}"
+            f"{'  (L2-resident)' if x['l2'].startswith('L2-res') else ''}")
 
 
 def main():
@@ -485,8 +609,25 @@ def main():
                     help="tokens of the fp32 recurrence that pre-fill the states (512 in the headline workload)")
     ap.add_argument("--only-timed", action="store_true",
                     help="skip the CUDA-graph, end-to-end, baseline-kernel and CPU legs (for profiler runs)")
+    ap.add_argument("--r", type=int, default=4, help="Compensator Tokens per state")
+    ap.add_argument("--n-iter", type=int, default=None, help="power-iteration steps (default: the library's)")
+    ap.add_argument("--gate", default="gdn", choices=["gdn", "kda"])
+    ap.add_argument("--sweep", action="store_true",
+                    help="throughput sweep over gate x batch x W x r (one JSON line per point) instead of the headline run")
+    ap.add_argument("--sweep-batches", default="32,128,256,512,1024")
+    ap.add_argument("--sweep-W", default="8,16,32,64")
+    ap.add_argument("--sweep-r", default="4,8")
+    ap.add_argument("--sweep-gates", default="gdn,kda")
+    ap.add_argument("--sweep-steps", type=int, default=512)
     args = ap.parse_args()
-    wl = synth.config("gdn_b256").with_(W=args.W, batch=args.batch)
+    if args.sweep:
+        run_sweep(args)
+        return
+    wl = synth.config("gdn_b256").with_(W=args.W, batch=args.batch, r=args.r)
+    if args.gate == "kda":
+        wl = wl.with_(name="kda_b%d" % args.batch, gate=synth.GATE_DIAG, heads_qk=wl.heads_v)
+    if args.n_iter is not None:
+        wl = wl.with_(n_iter=args.n_iter)
     if args.impl == "reference":
         run_reference(args, wl)
     else:
