@@ -357,7 +357,7 @@ def run_cuda(args, wl):
 
         def step_host(t):
             d = pin[t % wl.W]
-            lq.decode_step_host(sh, st, d["q"], d["k"], d["v"], d["beta"], d["alpha"], o_h, stage, stream)
+            lq.decode_step_host_pipelined(sh, st, d["q"], d["k"], d["v"], d["beta"], d["alpha"], o_h, stage, stream)
 
         for t in range(5):
             step_host(t)
@@ -368,13 +368,14 @@ def run_cuda(args, wl):
             step_host(t)
         e1.record(stream)
         barrier()
-        e2e_ms = e0.elapsed_time(e1)
-        e2e_ms = max_over_ranks(e2e_ms, dist if world > 1 else None, "cuda")
+        e2e_ms = max_over_ranks(e0.elapsed_time(e1), dist if world > 1 else None, "cuda")
         h2d = sum(v.numel() * v.element_size() for v in pin[0].values())
         e2e = {"value": whole_job_value(wl.batch * wl.heads_v, world, n_e2e, e2e_ms, wl.r), "unit": "GB/s",
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": o_h.numel() * 4, "steps": n_e2e,
                "ms_per_step": e2e_ms / n_e2e,
-               "api": "lq_decode_step_host (pinned host q,k,v,beta,alpha in; o out), one call per step"}
+               "api": "lq_decode_step_host_pipelined, one call per step: pinned host q,k,v,beta,alpha in (read over the "
+                      "bus by a gather launch per half batch), o out to pinned host memory (copied while the "
+                      "window-boundary kernel runs)"}
     except Exception as exc:
         log(f"end-to-end timing failed: {exc!r}")
 

@@ -142,6 +142,28 @@ lq_status lq_decode_step_profiled(const lq_shape *shape, const lq_state *state, 
 lq_status lq_decode_step_host(const lq_shape *shape, const lq_state *state, const uint16_t *q_h,
                               const uint16_t *k_h, const uint16_t *v_h, const uint16_t *beta_h,
                               const uint16_t *alpha_h, float *o_h, void *stage, lq_stream stream);
+/*
+ * lq_decode_step_host with the host<->device transfers overlapped with the kernels.  (The paper's path
+ * starts and ends in device memory; this is a convenience of the library for callers whose tokens arrive in
+ * host memory.)  The batch is cut into two sub-batches of whole sequences.  The inputs of both are brought in
+ * on a copy-in stream, so the second sub-batch arrives while the first is computed; o of a sub-batch is
+ * complete after its decode kernel and is copied out on a copy-out stream while the window-boundary kernel of
+ * that sub-batch and the next sub-batch run.  The two side streams are created per device at the first call
+ * (make that call outside any stream capture) and are tied to `stream` by events on both sides: the call
+ * starts after everything already enqueued on `stream`, and anything enqueued on `stream` afterwards starts
+ * after the last copy.  Same arguments, staging size, results and error codes as lq_decode_step_host; use
+ * pinned host memory, otherwise nothing overlaps.  Batches below sixteen sequences take the unpipelined path.
+ * Calls from several host threads are serialised inside the library while they enqueue.
+ *
+ * Both host-buffer entry points read the inputs with ONE gather launch (per sub-batch) instead of five copies
+ * when all input arrays are pinned, mapped into the device (cudaHostAlloc / cudaHostRegister memory under
+ * unified addressing) and 16-byte aligned with sizes that are multiples of 16 bytes; lq_decode_step_host
+ * then also lets the decode kernel write o straight into the host array.  Otherwise they fall back to
+ * cudaMemcpyAsync.  The results are the same either way.
+ */
+lq_status lq_decode_step_host_pipelined(const lq_shape *shape, const lq_state *state, const uint16_t *q_h,
+                                        const uint16_t *k_h, const uint16_t *v_h, const uint16_t *beta_h,
+                                        const uint16_t *alpha_h, float *o_h, void *stage, lq_stream stream);
 /* Bytes of device staging lq_decode_step_host needs for `shape` (0 if the shape is invalid). */
 uint64_t lq_decode_stage_bytes(const lq_shape *shape);
 

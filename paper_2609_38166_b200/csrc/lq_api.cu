@@ -3,6 +3,7 @@
 #include <algorithm>
 #include <atomic>
 #include <cstdio>
+#include <mutex>
 
 #include "lq_boundary.cuh"
 #include "lq_decode.cuh"
@@ -221,8 +222,8 @@ static int sm_count() {
   return cached;
 }
 
-template <typename K>
-static lq_status launch(K kernel, int grid, int block, size_t smem, cudaStream_t stream, const Params &p) {
+template <typename K, typename P>
+static lq_status launch(K kernel, int grid, int block, size_t smem, cudaStream_t stream, const P &p) {
   if (grid <= 0) return LQ_OK;
   if (smem > 48 * 1024 &&
       cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess) {
@@ -318,9 +319,50 @@ uint64_t lq_decode_stage_bytes(const lq_shape *s) {
   return 2 * up(2 * B * Hqk * K) + up(2 * B * Hv * V) + up(2 * B * Hv) + up(2 * na) + up(4 * B * Hv * V);
 }
 
-lq_status lq_decode_step_host(const lq_shape *shape, const lq_state *state, const uint16_t *q_h, const uint16_t *k_h,
-                              const uint16_t *v_h, const uint16_t *beta_h, const uint16_t *alpha_h, float *o_h,
-                              void *stage, lq_stream stream) {
+}  // extern "C"
+
+// One launch that brings the five input arrays from mapped pinned host memory into the device staging
+// buffer (the alternative, five cudaMemcpyAsync calls, costs about 10 us of latency per copy on top of the
+// transfer itself).  Every segment is a whole number of 16-byte units; both ends are 16-byte aligned.
+namespace {
+struct GatherSegs {
+  const uint4 *src[5];
+  uint4 *dst[5];
+  uint32_t units[5];      // 16-byte units per segment
+};
+__global__ void __launch_bounds__(256) gather_kernel(const GatherSegs g) {
+  const uint32_t stride = gridDim.x * blockDim.x;
+#pragma unroll
+  for (int sgm = 0; sgm < 5; sgm++) {
+    const uint4 *__restrict__ src = g.src[sgm];
+    uint4 *__restrict__ dst = g.dst[sgm];
+    const uint32_t n = g.units[sgm];
+    uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    for (; i + 3 * stride < n; i += 4 * stride) {          // four loads in flight per thread
+      const uint4 a = src[i], b = src[i + stride], c = src[i + 2 * stride], d = src[i + 3 * stride];
+      dst[i] = a; dst[i + stride] = b; dst[i + 2 * stride] = c; dst[i + 3 * stride] = d;
+    }
+    for (; i < n; i += stride) dst[i] = src[i];
+  }
+}
+
+// The device alias of a pinned, mapped host pointer; null if the memory is not mapped into the device.
+template <typename T>
+T *device_alias(T *host) {
+  void *dev = nullptr;
+  if (cudaHostGetDevicePointer(&dev, const_cast<void *>(static_cast<const void *>(host)), 0) != cudaSuccess) {
+    cudaGetLastError();
+    return nullptr;
+  }
+  return static_cast<T *>(dev);
+}
+}  // namespace
+
+extern "C" {
+
+static lq_status host_step_impl(const lq_shape *shape, const lq_state *state, const uint16_t *q_h, const uint16_t *k_h,
+                                const uint16_t *v_h, const uint16_t *beta_h, const uint16_t *alpha_h, float *o_h,
+                                void *stage, lq_stream stream, bool direct_ok) {
   lq_status rc = check_shape(shape);
   if (rc != LQ_OK) return rc;
   if (!q_h || !k_h || !v_h || !beta_h || !alpha_h || !o_h || !stage) return LQ_ERR_NULL;
@@ -338,6 +380,31 @@ lq_status lq_decode_step_host(const lq_shape *shape, const lq_state *state, cons
   float *o_d = reinterpret_cast<float *>(base);
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   if (B == 0) return LQ_OK;
+
+  // Fast path, when all six host arrays are pinned, mapped into the device and 16-byte aligned: one gather
+  // launch reads the inputs over the bus, and the decode kernel writes o straight into the host array (posted
+  // writes that overlap the kernel), so no copy follows the step.
+  const uint16_t *src_h[5] = {q_h, k_h, v_h, beta_h, alpha_h};
+  uint16_t *dst_d[5] = {q_d, k_d, v_d, b_d, a_d};
+  const uint64_t bytes[5] = {nqk, nqk, nv, nb, na};
+  GatherSegs g;
+  bool mapped = direct_ok && aligned16(o_h) && no < (1ull << 35);
+  for (int i = 0; mapped && i < 5; i++) {
+    const uint16_t *alias = (aligned16(src_h[i]) && bytes[i] < (1ull << 35)) ? device_alias(src_h[i]) : nullptr;
+    mapped = alias != nullptr;
+    g.src[i] = reinterpret_cast<const uint4 *>(alias);
+    g.dst[i] = reinterpret_cast<uint4 *>(dst_d[i]);
+    g.units[i] = static_cast<uint32_t>((bytes[i] + 15) / 16);   // the regions of `stage` are padded to 256 bytes;
+  }                                                             // a ragged tail is covered below
+  float *o_alias = mapped ? device_alias(o_h) : nullptr;
+  // a segment that is not a whole number of 16-byte units would read past the end of the host array
+  for (int i = 0; mapped && i < 5; i++) mapped = bytes[i] % 16 == 0;
+  if (mapped && o_alias) {
+    rc = launch(gather_kernel, 2 * sm_count(), 256, 0, st, g);
+    if (rc != LQ_OK) return rc;
+    return lq_decode_step(shape, state, q_d, k_d, v_d, b_d, a_d, o_alias, stream);
+  }
+
   if (cudaMemcpyAsync(q_d, q_h, nqk, cudaMemcpyHostToDevice, st) != cudaSuccess ||
       cudaMemcpyAsync(k_d, k_h, nqk, cudaMemcpyHostToDevice, st) != cudaSuccess ||
       cudaMemcpyAsync(v_d, v_h, nv, cudaMemcpyHostToDevice, st) != cudaSuccess ||
@@ -349,6 +416,154 @@ lq_status lq_decode_step_host(const lq_shape *shape, const lq_state *state, cons
   rc = lq_decode_step(shape, state, q_d, k_d, v_d, b_d, a_d, o_d, stream);
   if (rc != LQ_OK) return rc;
   if (cudaMemcpyAsync(o_h, o_d, no, cudaMemcpyDeviceToHost, st) != cudaSuccess) {
+    cudaGetLastError();
+    return LQ_ERR_CUDA;
+  }
+  return LQ_OK;
+}
+
+lq_status lq_decode_step_host(const lq_shape *shape, const lq_state *state, const uint16_t *q_h, const uint16_t *k_h,
+                              const uint16_t *v_h, const uint16_t *beta_h, const uint16_t *alpha_h, float *o_h,
+                              void *stage, lq_stream stream) {
+  return host_step_impl(shape, state, q_h, k_h, v_h, beta_h, alpha_h, o_h, stage, stream, true);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host-buffer decode step with the copies overlapped with the kernels: the batch is cut into chunks of
+// sequences; chunk c+1 is copied in and chunk c-1 copied out while chunk c is computed.  The copies run on two
+// streams that the library creates per device on first use; events tie them to the caller's stream, so for the
+// caller the call is still one piece of work on `stream`.
+// ---------------------------------------------------------------------------------------------
+namespace {
+constexpr int PIPE_CHUNKS = 2;
+struct HostPipe {
+  bool ready = false;
+  cudaStream_t s_in = nullptr, s_out = nullptr;
+  cudaEvent_t start = nullptr, out = nullptr, in[PIPE_CHUNKS] = {}, done[PIPE_CHUNKS] = {};
+};
+std::mutex g_pipe_mutex;
+HostPipe g_pipes[64];
+
+lq_status host_pipe(HostPipe **out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+    cudaGetLastError();
+    return LQ_ERR_CUDA;
+  }
+  HostPipe &hp = g_pipes[dev];
+  if (!hp.ready) {
+    bool ok = cudaStreamCreateWithFlags(&hp.s_in, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&hp.s_out, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&hp.out, cudaEventDisableTiming) == cudaSuccess;
+    for (int c = 0; ok && c < PIPE_CHUNKS; c++)
+      ok = cudaEventCreateWithFlags(&hp.in[c], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&hp.done[c], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) {
+      cudaGetLastError();
+      return LQ_ERR_CUDA;
+    }
+    hp.ready = true;
+  }
+  *out = &hp;
+  return LQ_OK;
+}
+}  // namespace
+
+lq_status lq_decode_step_host_pipelined(const lq_shape *shape, const lq_state *state, const uint16_t *q_h,
+                                        const uint16_t *k_h, const uint16_t *v_h, const uint16_t *beta_h,
+                                        const uint16_t *alpha_h, float *o_h, void *stage, lq_stream stream) {
+  lq_status rc = check_shape(shape);
+  if (rc != LQ_OK) return rc;
+  if (shape->batch < 8 * PIPE_CHUNKS)          // nothing to overlap
+    return lq_decode_step_host(shape, state, q_h, k_h, v_h, beta_h, alpha_h, o_h, stage, stream);
+  if ((rc = check_state(shape, state, true)) != LQ_OK) return rc;
+  if (!q_h || !k_h || !v_h || !beta_h || !alpha_h || !o_h || !stage) return LQ_ERR_NULL;
+  if (!aligned16(stage)) return LQ_ERR_ALIGN;
+  const uint64_t B = shape->batch, Hv = shape->heads_v, Hqk = shape->heads_qk, K = shape->d_k, V = shape->d_v;
+  const bool diag = shape->gate == LQ_GATE_DIAG;
+  auto up = [](uint64_t x) { return (x + 255) / 256 * 256; };
+  const uint64_t eqk = Hqk * K, ev = Hv * V, eb = Hv, ea = diag ? Hv * K : Hv;   // elements per sequence
+  char *base = static_cast<char *>(stage);
+  uint16_t *q_d = reinterpret_cast<uint16_t *>(base); base += up(2 * B * eqk);
+  uint16_t *k_d = reinterpret_cast<uint16_t *>(base); base += up(2 * B * eqk);
+  uint16_t *v_d = reinterpret_cast<uint16_t *>(base); base += up(2 * B * ev);
+  uint16_t *b_d = reinterpret_cast<uint16_t *>(base); base += up(2 * B * eb);
+  uint16_t *a_d = reinterpret_cast<uint16_t *>(base); base += up(2 * B * ea);
+  float *o_d = reinterpret_cast<float *>(base);
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const uint16_t *src_h[5] = {q_h, k_h, v_h, beta_h, alpha_h};
+  uint16_t *dst_d[5] = {q_d, k_d, v_d, b_d, a_d};
+  const uint64_t per_seq[5] = {eqk, eqk, ev, eb, ea};
+
+  // every sub-batch starts at a multiple of 8 sequences, which keeps all of its pointers 16-byte aligned and
+  // all of its arrays whole numbers of 16-byte units
+  const uint64_t per = (B / PIPE_CHUNKS + 7) / 8 * 8;
+  uint64_t lo[PIPE_CHUNKS + 1];
+  for (int c = 0; c < PIPE_CHUNKS; c++) lo[c] = std::min<uint64_t>(B, c * per);
+  lo[PIPE_CHUNKS] = B;
+
+  // Inputs: when the host arrays are pinned, mapped into the device and aligned, one gather launch per
+  // sub-batch (a few CTAs, which share the device with the kernels of the sub-batch before); otherwise five
+  // copies per sub-batch.
+  const uint16_t *src_a[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+  bool mapped = true;
+  for (int i = 0; mapped && i < 5; i++) {
+    src_a[i] = aligned16(src_h[i]) ? device_alias(src_h[i]) : nullptr;
+    mapped = src_a[i] != nullptr && (2 * B * per_seq[i]) % 16 == 0;
+  }
+
+  std::lock_guard<std::mutex> lock(g_pipe_mutex);   // the events below are shared by all callers on a device
+  HostPipe *hp = nullptr;
+  if ((rc = host_pipe(&hp)) != LQ_OK) return rc;
+  bool ok = cudaEventRecord(hp->start, st) == cudaSuccess &&          // after everything already on `stream`
+            cudaStreamWaitEvent(hp->s_in, hp->start, 0) == cudaSuccess &&
+            cudaStreamWaitEvent(hp->s_out, hp->start, 0) == cudaSuccess;
+  for (int c = 0; ok && c < PIPE_CHUNKS; c++) {
+    const uint64_t b0 = lo[c], nb = lo[c + 1] - lo[c];
+    if (nb == 0) continue;
+    if (mapped) {
+      GatherSegs g;
+      for (int i = 0; i < 5; i++) {
+        g.src[i] = reinterpret_cast<const uint4 *>(src_a[i] + b0 * per_seq[i]);
+        g.dst[i] = reinterpret_cast<uint4 *>(dst_d[i] + b0 * per_seq[i]);
+        g.units[i] = static_cast<uint32_t>((2 * nb * per_seq[i] + 15) / 16);
+      }
+      ok = launch(gather_kernel, sm_count() / 2, 256, 0, hp->s_in, g) == LQ_OK;
+    } else {
+      for (int i = 0; ok && i < 5; i++)
+        ok = cudaMemcpyAsync(dst_d[i] + b0 * per_seq[i], src_h[i] + b0 * per_seq[i], 2 * nb * per_seq[i],
+                             cudaMemcpyHostToDevice, hp->s_in) == cudaSuccess;
+    }
+    ok = ok && cudaEventRecord(hp->in[c], hp->s_in) == cudaSuccess;
+  }
+  // Kernels on `stream`, sub-batch after sub-batch.  o of a sub-batch is complete after its decode kernel, so
+  // its copy to the host starts there, next to the window-boundary kernel, which does not touch o.
+  for (int c = 0; ok && c < PIPE_CHUNKS; c++) {
+    const uint64_t b0 = lo[c], nb = lo[c + 1] - lo[c];
+    if (nb == 0) continue;
+    ok = cudaStreamWaitEvent(st, hp->in[c], 0) == cudaSuccess;
+    if (!ok) break;
+    lq_shape sub = *shape;
+    sub.batch = static_cast<int>(nb);
+    lq_state ss = *state;
+    ss.heads += b0 * Hv * head_bytes(shape->r);
+    ss.records += b0 * Hv * shape->W * record_floats(diag);
+    if (ss.decays) ss.decays += b0 * Hv * shape->W;
+    ss.win_pos += b0;
+    rc = decode_step_impl(&sub, &ss, q_d + b0 * eqk, k_d + b0 * eqk, v_d + b0 * ev, b_d + b0 * eb, a_d + b0 * ea,
+                          o_d + b0 * ev, stream, hp->done[c]);
+    if (rc != LQ_OK) break;
+    ok = cudaStreamWaitEvent(hp->s_out, hp->done[c], 0) == cudaSuccess &&
+         cudaMemcpyAsync(o_h + b0 * ev, o_d + b0 * ev, 4 * nb * ev, cudaMemcpyDeviceToHost, hp->s_out) == cudaSuccess;
+  }
+  // join: whatever was put on the side streams is waited for by `stream`, also after an error above
+  const bool joined = cudaEventRecord(hp->out, hp->s_out) == cudaSuccess &&
+                      cudaStreamWaitEvent(st, hp->out, 0) == cudaSuccess &&
+                      cudaEventRecord(hp->out, hp->s_in) == cudaSuccess &&
+                      cudaStreamWaitEvent(st, hp->out, 0) == cudaSuccess;
+  if (rc != LQ_OK) return rc;
+  if (!ok || !joined) {
     cudaGetLastError();
     return LQ_ERR_CUDA;
   }
@@ -403,7 +618,8 @@ lq_status lq_decode_step_host_static(const lq_shape *shape, const lq_state *stat
     cudaGetLastError();
     return LQ_ERR_CUDA;
   }
-  return lq_decode_step_host(shape, state, q_h, k_h, v_h, beta_h, alpha_h, o_h, stage, stream);
+  // always through the staging buffer, so that the cleared output region is what reaches o_h for such rows
+  return host_step_impl(shape, state, q_h, k_h, v_h, beta_h, alpha_h, o_h, stage, stream, false);
 }
 
 lq_status lq_window_flush(const lq_shape *shape, const lq_state *state, int force, lq_stream stream) {

@@ -19,7 +19,7 @@ GATE_DIAG = 1
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "liblq.so")
 _lib = None
 
-EXPORTS = ["lq_decode_step", "lq_decode_step_profiled", "lq_decode_step_host", "lq_decode_step_host_static", "lq_decode_stage_bytes", "lq_head_bytes", "lq_record_floats",
+EXPORTS = ["lq_decode_step", "lq_decode_step_profiled", "lq_decode_step_host", "lq_decode_step_host_pipelined", "lq_decode_step_host_static", "lq_decode_stage_bytes", "lq_head_bytes", "lq_record_floats",
            "lq_window_flush",
            "lq_quantize_state", "lq_dequantize_state", "lq_ref_decode_step_f32", "lq_ref_decode_step_bf16",
            "lq_decode_launches", "lq_check_device", "lq_status_string", "lq_version"]
@@ -55,7 +55,8 @@ def lib() -> C.CDLL:
             getattr(L, name).argtypes = [C.c_void_p]
         L.lq_decode_launches.restype = C.c_int
         L.lq_decode_launches.argtypes = [C.c_void_p]
-        for name in ("lq_decode_step", "lq_decode_step_profiled", "lq_decode_step_host", "lq_decode_step_host_static", "lq_check_device", "lq_window_flush", "lq_quantize_state",
+        for name in ("lq_decode_step", "lq_decode_step_profiled", "lq_decode_step_host", "lq_decode_step_host_pipelined",
+                     "lq_decode_step_host_static", "lq_check_device", "lq_window_flush", "lq_quantize_state",
                      "lq_dequantize_state", "lq_ref_decode_step_f32", "lq_ref_decode_step_bf16"):
             getattr(L, name).restype = C.c_int
         _lib = L
@@ -187,6 +188,17 @@ def decode_step_host(sh: Shape, st: State, q_h, k_h, v_h, beta_h, alpha_h, o_h, 
     cs = st.c()
     _check(lib().lq_decode_step_host(C.byref(s), C.byref(cs), _ptr(q_h), _ptr(k_h), _ptr(v_h), _ptr(beta_h),
                                      _ptr(alpha_h), _ptr(o_h), _ptr(stage), _stream(stream)), "lq_decode_step_host")
+
+
+def decode_step_host_pipelined(sh: Shape, st: State, q_h, k_h, v_h, beta_h, alpha_h, o_h, stage, stream=None):
+    """lq_decode_step_host_pipelined: same arguments as decode_step_host; copies and kernels overlap."""
+    for t in (q_h, k_h, v_h, beta_h, alpha_h, o_h):
+        assert t.device.type == "cpu" and t.is_contiguous()
+    s = sh.c()
+    cs = st.c()
+    _check(lib().lq_decode_step_host_pipelined(C.byref(s), C.byref(cs), _ptr(q_h), _ptr(k_h), _ptr(v_h), _ptr(beta_h),
+                                               _ptr(alpha_h), _ptr(o_h), _ptr(stage), _stream(stream)),
+           "lq_decode_step_host_pipelined")
 
 
 STATIC_STAGE_BYTES = 16 << 20

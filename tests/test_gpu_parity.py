@@ -210,8 +210,11 @@ def test_empty_batch_is_a_no_op():
     torch.cuda.synchronize()
 
 
-def test_host_buffer_entry_point(oracle):
-    wl = synth.Workload("h", 3, 4, 2, W=4, r=2, seed=700)
+@pytest.mark.parametrize("batch", [3, 8])
+def test_host_buffer_entry_point(oracle, batch):
+    """batch 3: array sizes that are not multiples of 16 bytes (copied with cudaMemcpyAsync); batch 8: the
+    path that gathers the pinned inputs with one launch and writes o straight into the pinned host array."""
+    wl = synth.Workload("h", batch, 4, 2, W=4, r=2, seed=700)
     osh, lsh = gu.shapes(wl)
     ost = OState(osh)
     S0 = synth.dense_states(wl, 9)
@@ -219,7 +222,7 @@ def test_host_buffer_entry_point(oracle):
     st = lq.State(lsh)
     lq.quantize_state(lsh, gu.dev(S0), st)
     stage = torch.empty((lq.decode_stage_bytes(lsh),), dtype=torch.uint8, device="cuda")
-    o_h = torch.empty((3, 4, 128), dtype=torch.float32).pin_memory()
+    o_h = torch.empty((batch, 4, 128), dtype=torch.float32).pin_memory()
     for step in range(6):
         tok = synth.token_inputs(wl, step)
         want = oracle.decode_step(osh, ost, **tok)
@@ -228,3 +231,30 @@ def test_host_buffer_entry_point(oracle):
         torch.cuda.synchronize()
         _close(o_h.numpy(), want, f"host-buffer step {step}")
     gu.assert_state_parity(st, ost, wl.r, "host-buffer chain")
+
+
+@pytest.mark.parametrize("gate,batch", [(synth.GATE_SCALAR, 37), (synth.GATE_DIAG, 16), (synth.GATE_SCALAR, 5)])
+def test_pipelined_host_entry_point(oracle, gate, batch):
+    """Sub-batches with copies on side streams: ragged last sub-batch (37 = 16+16+5+0), an exact split, and a
+    batch below the pipelining threshold; seven tokens with W = 4 cross a window boundary on the way."""
+    wl = synth.Workload("hp", batch, 4, 2, W=4, r=2, gate=gate, seed=710 + batch)
+    osh, lsh = gu.shapes(wl)
+    ost = OState(osh)
+    S0 = synth.dense_states(wl, 11)
+    oracle.quantize_state(osh, S0, ost)
+    st = lq.State(lsh)
+    lq.quantize_state(lsh, gu.dev(S0), st)
+    stage = torch.empty((lq.decode_stage_bytes(lsh),), dtype=torch.uint8, device="cuda")
+    o_h = torch.full((batch, 4, 128), float("nan"), dtype=torch.float32).pin_memory()
+    side = torch.cuda.Stream()
+    for step in range(7):
+        tok = synth.token_inputs(wl, step)
+        want = oracle.decode_step(osh, ost, **tok)
+        pin = {k: torch.from_numpy(v.view(np.int16)).pin_memory() for k, v in tok.items()}
+        with torch.cuda.stream(side):
+            lq.decode_step_host_pipelined(lsh, st, pin["q"], pin["k"], pin["v"], pin["beta"], pin["alpha"], o_h,
+                                          stage, side)
+        side.synchronize()
+        _close(o_h.numpy(), want, f"pipelined host-buffer step {step}")
+    gu.assert_state_parity(st, ost, wl.r, "pipelined host-buffer chain")
+    assert lq.check_device() == 0
