@@ -598,6 +598,105 @@ def run_sweep(args):
             f"{'  (L2-resident)' if x['l2'].startswith('L2-res') else ''}")
 
 
+# --------------------------------------------------------------------------------------------------
+# Ablation ladder (the structure of the paper's component ablation, on synthetic decode inputs): speed of
+# every rung on the benchmark batch, and its error against the fp32 recurrence fed the same tokens.
+# Everything runs on the GPU through the library; no oracle involved.
+# --------------------------------------------------------------------------------------------------
+def run_ladder(args):
+    import torch
+    from paper_2609_38166_b200 import build, lq
+
+    log = lambda m: print(f"[ladder] {m}", file=sys.stderr, flush=True)
+    torch.cuda.set_device(0)
+    build.build()
+    lq.lib()
+    stream = torch.cuda.current_stream()
+    rungs = [("fp32 state, every token", None),
+             ("bf16 state, every token", "bf16"),
+             ("int8 every token (W=1, no compensators, no smoothing)", dict(W=1, r=0, smooth=0)),
+             ("int8 per window (W=16), no compensators, no smoothing", dict(W=16, r=0, smooth=0)),
+             ("+ 4 Compensator Tokens", dict(W=16, r=4, smooth=0)),
+             ("+ residual smoothing (the full method)", dict(W=16, r=4, smooth=1))]
+    rows = []
+    for base_name in ("gdn_b256", "kda_b128_outlier"):
+        base = synth.config(base_name)
+        small = base.with_(batch=16)                     # error: 16 sequences x 32 heads, 64 + 256 tokens
+        n_warm, n_err = 64, 256
+        toks_small = [to_dev(synth.token_inputs(small, t), torch) for t in range(n_warm + n_err)]
+        toks_big = [to_dev(synth.token_inputs(base, 1000 + t), torch) for t in range(16)]
+        keys = ("q", "k", "v", "beta", "alpha")
+        for label, var in rungs:
+            # ---- error against the fp32 recurrence ----
+            wl = small if not isinstance(var, dict) else small.with_(**var)
+            sh = lq.Shape(wl.batch, 32, wl.heads_qk, 128, 128, wl.W, wl.r, wl.n_iter, wl.gate, wl.smooth)
+            S = torch.zeros((wl.batch, 32, 128, 128), dtype=torch.float32, device="cuda")
+            o_ref = torch.empty((wl.batch, 32, 128), dtype=torch.float32, device="cuda")
+            o_var = torch.empty_like(o_ref)
+            for t in range(n_warm):
+                lq.ref_decode_step_f32(sh, S, *[toks_small[t][k] for k in keys], o_ref)
+            st = S16 = None
+            if var == "bf16":
+                S16 = S.to(torch.bfloat16).view(torch.int16).contiguous()
+            elif isinstance(var, dict):
+                st = lq.State(sh)
+                lq.quantize_state(sh, S, st)
+            errs = []
+            for t in range(n_warm, n_warm + n_err):
+                d = [toks_small[t][k] for k in keys]
+                lq.ref_decode_step_f32(sh, S, *d, o_ref)
+                if var is None:
+                    o_var.copy_(o_ref)
+                elif var == "bf16":
+                    lq.ref_decode_step_bf16(sh, S16, *d, o_var)
+                else:
+                    lq.decode_step(sh, st, *d, o_var)
+                num = (o_var - o_ref).flatten(1).norm(dim=1)
+                den = o_ref.flatten(1).norm(dim=1)
+                errs.append((num / den).mean())
+            err = float(torch.stack(errs).mean())
+            del S, S16, st
+            # ---- speed on the full batch, windows staggered as in the headline run ----
+            wlb = base if not isinstance(var, dict) else base.with_(**var)
+            shb = lq.Shape(wlb.batch, 32, wlb.heads_qk, 128, 128, wlb.W, wlb.r, wlb.n_iter, wlb.gate, wlb.smooth)
+            ob = torch.empty((wlb.batch, 32, 128), dtype=torch.float32, device="cuda")
+            if isinstance(var, dict):
+                _, stb, ob = prepare_state(wlb, lq, torch, lambda m: None, 32)
+                fn = lambda t: lq.decode_step(shb, stb, *[toks_big[t % 16][k] for k in keys], ob, stream)
+                state_b = 128 * 128 + 1024 + 2 * wlb.r * 256
+            elif var == "bf16":
+                Sb = torch.zeros((wlb.batch, 32, 128, 128), dtype=torch.int16, device="cuda")
+                fn = lambda t: lq.ref_decode_step_bf16(shb, Sb, *[toks_big[t % 16][k] for k in keys], ob, stream)
+                state_b = 2 * 128 * 128
+            else:
+                Sb = torch.zeros((wlb.batch, 32, 128, 128), dtype=torch.float32, device="cuda")
+                fn = lambda t: lq.ref_decode_step_f32(shb, Sb, *[toks_big[t % 16][k] for k in keys], ob, stream)
+                state_b = 4 * 128 * 128
+            for t in range(48):
+                fn(t)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record(stream)
+            nrep = 512
+            for t in range(nrep):
+                fn(t)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / nrep
+            row = {"ladder": True, "workload": base_name, "rung": label, "ms_per_step": ms,
+                   "state_bytes_per_head": state_b, "rel_err_o_vs_fp32": err,
+                   "error_run": "16 sequences x 32 heads, 64 fp32 warm-up tokens, mean over 256 tokens and heads of |o - o_fp32| / |o_fp32|"}
+            rows.append(row)
+            print(json.dumps(row), flush=True)
+            stb = Sb = None
+            torch.cuda.empty_cache()
+    t32 = {r["workload"]: r["ms_per_step"] for r in rows if r["rung"].startswith("fp32")}
+    log("workload           rung                                                      us/step  x fp32   B/head   rel.err(o)")
+    for r in rows:
+        log(f"{r['workload']:18s} {r['rung']:56s} {1e3 * r['ms_per_step']:8.1f} {t32[r['workload']] / r['ms_per_step']:7.2f} "
+            f"{r['state_bytes_per_head']:8d}   {r['rel_err_o_vs_fp32']:.3e}")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -615,6 +714,9 @@ def main():
     ap.add_argument("--gate", default="gdn", choices=["gdn", "kda"])
     ap.add_argument("--sweep", action="store_true",
                     help="throughput sweep over gate x batch x W x r (one JSON line per point) instead of the headline run")
+    ap.add_argument("--ladder", action="store_true",
+                    help="ablation ladder: fp32 / bf16 / int8 per token / int8 per window / + compensators / + smoothing, "
+                         "speed and error against the fp32 recurrence (one JSON line per rung)")
     ap.add_argument("--sweep-batches", default="32,128,256,512,1024")
     ap.add_argument("--sweep-W", default="8,16,32,64")
     ap.add_argument("--sweep-r", default="4,8")
@@ -623,6 +725,9 @@ def main():
     args = ap.parse_args()
     if args.sweep:
         run_sweep(args)
+        return
+    if args.ladder:
+        run_ladder(args)
         return
     wl = synth.config("gdn_b256").with_(W=args.W, batch=args.batch, r=args.r)
     if args.gate == "kda":
