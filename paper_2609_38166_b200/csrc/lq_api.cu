@@ -22,6 +22,7 @@ __global__ void __launch_bounds__(256, 2) boundary_kernel(const Params p) {
   const Tile t;
   const size_t nh = (size_t)p.batch * p.heads_v;
   __shared__ uint32_t todo[2];
+  grid_dependency_wait();                    // everything the kernel before this one wrote is visible from here on
 #ifdef LQ_TIMING
   if (threadIdx.x == 0) { for (int i = 0; i < 16; i++) lq_bacc[i] = 0; lq_btick = clock64(); }
 #endif
@@ -234,6 +235,35 @@ static lq_status launch(K kernel, int grid, int block, size_t smem, cudaStream_t
   return cudaGetLastError() == cudaSuccess ? LQ_OK : LQ_ERR_CUDA;
 }
 
+// Launch that may begin while the kernel before it on the stream is still draining (programmatic dependent
+// launch): its CTAs become resident as SM resources free up and sit in griddepcontrol.wait until that kernel
+// has completed and its writes are visible.  Only for kernels that execute griddepcontrol.wait before their
+// first access to global memory.
+template <typename K, typename P>
+static lq_status launch_dependent(K kernel, int grid, int block, size_t smem, cudaStream_t stream, const P &p) {
+  if (grid <= 0) return LQ_OK;
+  if (smem > 48 * 1024 &&
+      cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess) {
+    cudaGetLastError();
+    return LQ_ERR_CUDA;
+  }
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(block);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, kernel, p) != cudaSuccess) {
+    cudaGetLastError();
+    return LQ_ERR_CUDA;
+  }
+  return LQ_OK;
+}
+
 // grid = min(work items, CTAs that fit on the device at once), for kernels that stride over their work
 template <typename K>
 static lq_status launch_persistent(K kernel, long items, int block, size_t smem, cudaStream_t stream, const Params &p) {
@@ -249,7 +279,7 @@ static lq_status launch_persistent(K kernel, long items, int block, size_t smem,
     return LQ_ERR_CUDA;
   }
   const long resident = (long)per_sm * sm_count();
-  return launch(kernel, static_cast<int>(items < resident ? items : resident), block, smem, stream, p);
+  return launch_dependent(kernel, static_cast<int>(items < resident ? items : resident), block, smem, stream, p);
 }
 
 template <int MODE>
@@ -258,8 +288,8 @@ static lq_status launch_boundary(const lq_shape *s, const Params &p, cudaStream_
   const size_t smem = BoundarySmem::bytes(s->W, s->r, diag);
   const long nh = (long)s->batch * s->heads_v;
   const int grid = static_cast<int>(nh < 4L * sm_count() ? nh : 4L * sm_count());
-  return diag ? launch(boundary_kernel<LQ_GATE_DIAG, MODE>, grid, 256, smem, stream, p)
-              : launch(boundary_kernel<LQ_GATE_SCALAR, MODE>, grid, 256, smem, stream, p);
+  return diag ? launch_dependent(boundary_kernel<LQ_GATE_DIAG, MODE>, grid, 256, smem, stream, p)
+              : launch_dependent(boundary_kernel<LQ_GATE_SCALAR, MODE>, grid, 256, smem, stream, p);
 }
 
 }  // namespace lq

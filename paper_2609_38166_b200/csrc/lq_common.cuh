@@ -118,6 +118,14 @@ __device__ __forceinline__ float dot128_shared(const float *a, const float *b, i
   return tree16(block8(a2, b2));
 }
 
+// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may become resident
+// before the kernel ahead of it has finished; this is where it waits for that kernel's completion and writes
+// (a no-op for an ordinary launch).  Right after it the kernel allows its own dependents to be scheduled.
+__device__ __forceinline__ void grid_dependency_wait() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // Phase timing (development aid, compiled in with -DLQ_TIMING only): clock cycles per phase of the decode
 // warps, summed over all heads by lane 0 of each warp (slots 0..15: stream warp, 16..31: dot warp; 32..: thread 0 of the boundary kernel's CTAs).
 #ifdef LQ_TIMING

@@ -192,6 +192,7 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
 
   if (threadIdx.x == 0) mbar_init(bar, 1);
   __syncthreads();
+  grid_dependency_wait();                    // no global memory is touched above this line
   uint32_t parity = 0;
   const unsigned nh = static_cast<unsigned>(p.batch) * p.heads_v, G = gridDim.x, Hv = p.heads_v;
   const unsigned G_b = G / Hv, G_hv = G % Hv;       // one grid stride in (sequence, head) steps
