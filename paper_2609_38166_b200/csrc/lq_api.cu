@@ -16,68 +16,88 @@ namespace lq {
 // MODE 1: quantize dense fp32 states         MODE 2: dequantize to dense fp32 states
 // ---------------------------------------------------------------------------------------------
 template <int GATE, int MODE>
-__global__ void __launch_bounds__(256, 2) boundary_kernel(const Params p) {
+__global__ void __launch_bounds__(256, 2) boundary_kernel(const Params p, const int stage_bufs) {
   extern __shared__ float4 lq_smem4[];
-  const BoundarySmem sm(reinterpret_cast<float *>(lq_smem4), p.W, p.r, GATE == LQ_GATE_DIAG);
+  float *smem = reinterpret_cast<float *>(lq_smem4);
+  constexpr bool DIAG = GATE == LQ_GATE_DIAG;
   const Tile t;
   const size_t nh = (size_t)p.batch * p.heads_v;
-  __shared__ uint32_t todo[2];
+  __shared__ uint32_t todo_mask;
+  __shared__ int todo_n[32];
   grid_dependency_wait();                    // everything the kernel before this one wrote is visible from here on
 #ifdef LQ_TIMING
   if (threadIdx.x == 0) { for (int i = 0; i < 16; i++) lq_bacc[i] = 0; lq_btick = clock64(); }
 #endif
   // The CTA owns heads blockIdx.x + k * gridDim.x.  Warp 0 looks at 32 of them at a time (one load each, all in
-  // flight together) and publishes which ones have work; then the CTA handles those one after the other.
+  // flight together) and publishes which ones have work and how many records each holds; then the CTA takes
+  // them one after the other, fetching the next one's data into the other staging buffer meanwhile.
   for (size_t base = blockIdx.x; base < nh; base += 32 * (size_t)gridDim.x) {
-    int n_mine = 0;
     if (t.warp == 0) {
       const size_t cand = base + t.lane * (size_t)gridDim.x;
       bool want = false;
+      int n_mine = 0;
       if (cand < nh) {
         if (MODE != 1) n_mine = p.win_pos[cand / p.heads_v] & 0xFFFF;
         want = MODE != 0 || n_mine == p.W || (p.force && n_mine > 0);
       }
       const uint32_t m = __ballot_sync(FULL, want);
-      if (t.lane == 0) todo[0] = m;
+      todo_n[t.lane] = n_mine > p.W ? p.W : n_mine;
+      if (t.lane == 0) todo_mask = m;
     }
     __syncthreads();
     LQ_BTICK(0);
-    uint32_t mask = todo[0];
+    uint32_t mask = todo_mask;
+    int buf = 0;
+    bool staged = false;                     // the data of the head about to be processed is already on its way
     while (mask) {
       const int kbit = __ffs(mask) - 1;
       mask &= mask - 1;
       const size_t bh = base + kbit * (size_t)gridDim.x;
       const int b = static_cast<int>(bh / p.heads_v);
-      int n = 0;
-      if (MODE != 1) {
-        if (t.warp == 0) { n = __shfl_sync(FULL, n_mine, kbit); if (t.lane == 0) todo[1] = n; }
-        __syncthreads();                     // also: the previous head's use of shared memory is over
-        n = todo[1];
-        if (n > p.W) n = p.W;
-      }
+      const int n = todo_n[kbit];
+      const BoundarySmem sm(smem, p.W, p.r, DIAG, buf);
       float M[8][8];
       if (MODE == 1) {
         const float *S = p.S + bh * (size_t)(D * D);
 #pragma unroll
         for (int a = 0; a < 8; a++) load8(S + (8 * t.ty + a) * D + 8 * t.tx, M[a]);
       } else {
+        // (the barrier that ended the previous head's work also freed both staging buffers for writing)
+        if (!staged) {
+          stage_issue<GATE>(p, sm, t, bh, n);
+          cp_async_commit();
+        }
+        staged = false;
+        if (mask && stage_bufs > 1) {
+          const int knext = __ffs(mask) - 1;
+          const BoundarySmem nx(smem, p.W, p.r, DIAG, buf ^ 1);
+          stage_issue<GATE>(p, nx, t, base + knext * (size_t)gridDim.x, todo_n[knext]);
+          cp_async_commit();
+          staged = true;
+          cp_async_wait_but_one();
+        } else {
+          cp_async_wait_all();
+        }
+        __syncthreads();
+        LQ_BTICK(1);
         reconstruct_tile<GATE>(p, sm, t, bh, n, M);
       }
       if (MODE == 2) {
         float *S = p.S + bh * (size_t)(D * D);
 #pragma unroll
         for (int a = 0; a < 8; a++) store8(S + (8 * t.ty + a) * D + 8 * t.tx, M[a]);
-        continue;
+      } else {
+        quantize_tile(p, sm, t, bh, MODE == 0 ? n : 0, M);
       }
-      quantize_tile(p, sm, t, bh, MODE == 0 ? n : 0, M);
-      __syncthreads();
+      __syncthreads();                       // this head's use of shared memory is over
       LQ_BTICK(9);
-      if (t.tid == 0) {
+      if (MODE != 2 && t.tid == 0) {
         if (MODE == 0) arrive_and_set(p.win_pos, b, p.heads_v, 0);
-        else p.win_pos[b] = 0;                 // nobody reads win_pos in this mode
+        else p.win_pos[b] = 0;               // nobody reads win_pos in this mode
       }
+      if (staged) buf ^= 1;
     }
-    __syncthreads();                         // todo[] is rewritten by the next round
+    __syncthreads();                         // todo_mask / todo_n are rewritten by the next round
   }
 #ifdef LQ_TIMING
   if (threadIdx.x == 0) {
@@ -282,14 +302,42 @@ static lq_status launch_persistent(K kernel, long items, int block, size_t smem,
   return launch_dependent(kernel, static_cast<int>(items < resident ? items : resident), block, smem, stream, p);
 }
 
+// launch with one extra kernel argument (programmatic dependent, like launch_dependent)
+template <typename K>
+static lq_status launch_boundary_kernel(K kernel, int grid, size_t smem, cudaStream_t stream, const Params &p, int bufs) {
+  if (grid <= 0) return LQ_OK;
+  if (smem > 48 * 1024 &&
+      cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess) {
+    cudaGetLastError();
+    return LQ_ERR_CUDA;
+  }
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(256);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, kernel, p, bufs) != cudaSuccess) {
+    cudaGetLastError();
+    return LQ_ERR_CUDA;
+  }
+  return LQ_OK;
+}
+
 template <int MODE>
 static lq_status launch_boundary(const lq_shape *s, const Params &p, cudaStream_t stream) {
   const bool diag = s->gate == LQ_GATE_DIAG;
-  const size_t smem = BoundarySmem::bytes(s->W, s->r, diag);
+  const int bufs = MODE == 1 ? 1 : BoundarySmem::buffers(s->W, s->r, diag);
+  const size_t smem = BoundarySmem::bytes(s->W, s->r, diag, bufs);
   const long nh = (long)s->batch * s->heads_v;
-  const int grid = static_cast<int>(nh < 4L * sm_count() ? nh : 4L * sm_count());
-  return diag ? launch_dependent(boundary_kernel<LQ_GATE_DIAG, MODE>, grid, 256, smem, stream, p)
-              : launch_dependent(boundary_kernel<LQ_GATE_SCALAR, MODE>, grid, 256, smem, stream, p);
+  // persistent: the CTAs that are resident at once (two per SM), each striding over the heads
+  const int grid = static_cast<int>(nh < 2L * sm_count() ? nh : 2L * sm_count());
+  return diag ? launch_boundary_kernel(boundary_kernel<LQ_GATE_DIAG, MODE>, grid, smem, stream, p, bufs)
+              : launch_boundary_kernel(boundary_kernel<LQ_GATE_SCALAR, MODE>, grid, smem, stream, p, bufs);
 }
 
 }  // namespace lq

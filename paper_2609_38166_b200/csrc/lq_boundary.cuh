@@ -7,27 +7,69 @@
 
 namespace lq {
 
-// Shared-memory plan of the boundary kernels (floats).
+// Shared-memory plan of the boundary kernels (in floats).  A fixed part (working vectors of the fit, the
+// compensators widened to fp32) is followed by one or two staging buffers, each holding everything that is read
+// from global memory for one head: with two, the next head of the CTA is fetched while this one is computed.
 struct BoundarySmem {
-  float *kd;     // [W][128]  buffered write keys, turned in place into Gamma_{j+1:n} kt_j
-  float *bu;     // [W][128]  buffered corrections u_j
-  float *ba;     // [W][128]  diagonal-gate decays of the records (diagonal gate only), else [W]
+  // fixed part
   float *ck;     // [r][128]  compensator keys widened to fp32
   float *cu;     // [r][128]  compensator values widened to fp32
   float *vec;    // [128]     row-sum results (t of the power iteration, row mean-abs)
   float *colv;   // [128]     column-sum results
   float *part;   // [8][128]  per-warp column partial sums
   float *gam;    // [128]     Gamma_{1:n}
+  // staging buffer `buf`
+  float *kd;     // [W][128]  buffered write keys, turned in place into Gamma_{j+1:n} kt_j
+  float *bu;     // [W][128]  buffered corrections u_j
+  float *ba;     // [W][128]  diagonal-gate decays of the records (diagonal gate only), else [MAX_W]
   float *cs;     // [128]     smoothing scales c
   float *ss;     // [128]     code steps s_j = B_j / 127
-  __device__ __forceinline__ BoundarySmem(float *base, int W, int r, bool diag) {
-    kd = base; bu = kd + W * D; ba = bu + W * D; ck = ba + (diag ? W * D : MAX_W);
-    cu = ck + r * D; vec = cu + r * D; colv = vec + D; part = colv + D; gam = part + 8 * D; cs = gam + D; ss = cs + D;
+  uint16_t *ckh; // [r][128]  compensator keys as stored (fp16 bits)
+  uint16_t *cuh; // [r][128]  compensator values as stored
+  uint8_t *zt;   // [128][128] codes Z^T, 16-byte chunk q of row v stored at chunk q ^ ((v >> 3) & 7)
+  __host__ __device__ static constexpr int fixed_floats(int r) { return 2 * r * D + 11 * D; }
+  __host__ __device__ static constexpr int stage_floats(int W, int r, bool diag) {
+    return 2 * W * D + (diag ? W * D : MAX_W) + 2 * D + r * D + D * D / 4;
   }
-  static size_t bytes(int W, int r, bool diag) {
-    return sizeof(float) * (size_t)(2 * W * D + (diag ? W * D : MAX_W) + 2 * r * D + 2 * D + 8 * D + 3 * D);
+  __device__ __forceinline__ BoundarySmem(float *base, int W, int r, bool diag, int buf) {
+    ck = base; cu = ck + r * D; vec = cu + r * D; colv = vec + D; part = colv + D; gam = part + 8 * D;
+    kd = base + fixed_floats(r) + buf * stage_floats(W, r, diag);
+    bu = kd + W * D; ba = bu + W * D; cs = ba + (diag ? W * D : MAX_W); ss = cs + D;
+    ckh = reinterpret_cast<uint16_t *>(ss + D); cuh = ckh + r * D;
+    zt = reinterpret_cast<uint8_t *>(cuh + r * D);
   }
+  static size_t bytes(int W, int r, bool diag, int bufs) {
+    return sizeof(float) * (size_t)(fixed_floats(r) + bufs * stage_floats(W, r, diag));
+  }
+  // two staging buffers while two CTAs with two buffers each still fit on an SM
+  static int buffers(int W, int r, bool diag) { return bytes(W, r, diag, 2) <= 110 * 1024 ? 2 : 1; }
 };
+
+// Issue the asynchronous copies that bring head bh (its codes, scales, compensators and n records) into the
+// staging buffer of sm.  The caller commits the group and later waits for it.
+template <int GATE>
+__device__ __forceinline__ void stage_issue(const Params &p, const BoundarySmem &sm, const Tile &t, size_t bh, int n) {
+  constexpr bool DIAG = GATE == LQ_GATE_DIAG;
+  constexpr int RF = record_floats(DIAG);
+  const int r = p.r;
+  const uint8_t *hb = p.head(bh);
+  for (int e = t.tid; e < D * D / 16; e += 256) {             // codes: 1024 chunks of 16 bytes
+    const int v = e >> 3, q = e & 7;
+    cp_async16(sm.zt + v * D + 16 * (q ^ ((v >> 3) & 7)), hb + HB_CODES + 16 * e);
+  }
+  const float *rec = p.record(bh, 0, DIAG);
+  for (int e = t.tid; e < n * (D / 4); e += 256) {
+    const int j = e / (D / 4), q4 = 4 * (e % (D / 4));
+    cp_async16(sm.kd + j * D + q4, rec + j * RF + REC_KT + q4);
+    cp_async16(sm.bu + j * D + q4, rec + j * RF + REC_U + q4);
+    if (DIAG) cp_async16(sm.ba + j * D + q4, rec + j * RF + REC_A + q4);
+  }
+  if (!DIAG && t.tid < n) cp_async4(sm.ba + t.tid, p.decays + bh * (size_t)p.W + t.tid);
+  if (t.tid < D / 4) cp_async16(sm.ss + 4 * t.tid, hb + HB_COL_SCALE + 16 * t.tid);
+  else if (t.tid < D / 2) cp_async16(sm.cs + 4 * (t.tid - D / 4), hb + HB_ROW_SMOOTH + 16 * (t.tid - D / 4));
+  for (int e = t.tid; e < r * D / 4; e += 256)                // 2 r rows of 256 bytes, contiguous in the head block
+    cp_async16(sm.ckh + 8 * e, hb + HB_COMP_K + 16 * e);      // (cuh follows ckh in the buffer as in the block)
+}
 
 // Eq. 7 for the tile of thread t: M = Gamma_{1:n}[C (Z/127) B + Kc Uc^T] + sum_j Gamma_{j+1:n} kt_j u_j^T,
 // evaluated per element as  base = c_i*(Z_ij*s_j) with s_j the stored code step; base = fma(kc_hi, uc_hj, base) for h = 0..r-1;
@@ -36,42 +78,12 @@ struct BoundarySmem {
 template <int GATE>
 __device__ __forceinline__ void reconstruct_tile(const Params &p, const BoundarySmem &sm, const Tile &t, size_t bh,
                                                  int n, float (&M)[8][8]) {
-  const int W = p.W, r = p.r;
+  const int r = p.r;
   constexpr bool DIAG = GATE == LQ_GATE_DIAG;
   constexpr int RF = record_floats(DIAG);
-  // this thread's codes: the layout is value-channel major (Z^T), so a column of the tile is 8 contiguous
-  // bytes; issued first so that they fly while the records are staged
-  uint2 z[8];
-  {
-    const int8_t *ZT = p.codes(bh);
-#pragma unroll
-    for (int b = 0; b < 8; b++) z[b] = *reinterpret_cast<const uint2 *>(ZT + (8 * t.tx + b) * D + 8 * t.ty);
-  }
-  // stage the n records, the compensators and the scales in shared memory
-  {
-    const float *rec = p.record(bh, 0, DIAG);
-    for (int e = t.tid; e < n * (D / 4); e += 256) {
-      const int j = e / (D / 4), q4 = 4 * (e % (D / 4));
-      cp_async16(sm.kd + j * D + q4, rec + j * RF + REC_KT + q4);
-      cp_async16(sm.bu + j * D + q4, rec + j * RF + REC_U + q4);
-      if (DIAG) cp_async16(sm.ba + j * D + q4, rec + j * RF + REC_A + q4);
-    }
-    if (!DIAG && t.tid < n) sm.ba[t.tid] = p.decays[bh * (size_t)W + t.tid];
-    cp_async_commit();
-    const uint16_t *gk = p.comp_k(bh), *gu = p.comp_u(bh);
-    for (int e = t.tid; e < r * D; e += 256) {
-      sm.ck[e] = f16_bits(gk[e]);
-      sm.cu[e] = f16_bits(gu[e]);
-    }
-    if (t.tid < D) {
-      sm.cs[t.tid] = p.row_smooth(bh)[t.tid];
-      sm.ss[t.tid] = p.col_scale(bh)[t.tid];
-    }
-    cp_async_wait_all();
-  }
-  __syncthreads();
-  LQ_BTICK(1);
-  // cumulative decays, newest record first (Appendix B.2): kd_j = Gamma_{j+1:n} kt_j, gam = Gamma_{1:n}
+  // the staging buffer has landed and the CTA has synchronised (the caller did both)
+  // cumulative decays, newest record first (Appendix B.2): kd_j = Gamma_{j+1:n} kt_j, gam = Gamma_{1:n};
+  // the other half of the CTA widens the compensators meanwhile
   if (t.tid < D) {
     const int i = t.tid;
     float g = 1.0f;
@@ -94,6 +106,8 @@ __device__ __forceinline__ void reconstruct_tile(const Params &p, const Boundary
       g = g * (GATE == LQ_GATE_DIAG ? sm.ba[j * D + i] : sm.ba[j]);
     }
     sm.gam[i] = g;
+  } else {
+    for (int e = t.tid - D; e < 2 * r * D; e += 256 - D) sm.ck[e] = f16_bits(sm.ckh[e]);   // ck and cu are adjacent
   }
   __syncthreads();
   LQ_BTICK(2);
@@ -104,7 +118,10 @@ __device__ __forceinline__ void reconstruct_tile(const Params &p, const Boundary
   load8(sm.ss + 8 * t.tx, sj);
 #pragma unroll
   for (int b = 0; b < 8; b++) {
-    const uint32_t lo = z[b].x, hi = z[b].y;
+    // column v = 8 tx + b of the tile: bytes 8 ty .. 8 ty + 7 of row v of Z^T (chunk ty / 2, swizzled by tx)
+    const uint2 zz = *reinterpret_cast<const uint2 *>(sm.zt + (8 * t.tx + b) * D + 16 * ((t.ty >> 1) ^ (t.tx & 7)) +
+                                                      8 * (t.ty & 1));
+    const uint32_t lo = zz.x, hi = zz.y;
 #pragma unroll
     for (int a = 0; a < 8; a++) {
       const uint32_t word = a < 4 ? lo : hi;
