@@ -244,3 +244,40 @@ def test_record_start_vector_is_what_the_first_step_multiplies(oracle):
     # S u_3 = sum_j k_j (u_j . u_3) = k_3 |u_3|^2 : the newest record's key, although it is the weakest one
     assert abs(abs(k1 @ keys[3]) - 1.0) < 2e-3
     assert abs(k1 @ keys[0]) < 0.5
+
+
+@pytest.mark.parametrize("r", [2, 3, 5])
+def test_fitted_keys_are_orthonormal_for_any_count(oracle, r):
+    """Each token is fitted on what the tokens before it left (deflation).  The stored keys must then be unit
+    vectors, mutually orthogonal up to the fp16 rounding of their entries, and R + K U^T must give back the state
+    (Eq. 6) with a residual norm smaller than after r - 1 tokens."""
+    rng = np.random.default_rng(40 + r)
+    M = _gapped(rng, 128, 128, [9.0, 5.0, 3.0, 2.0, 1.2, 0.7])
+    S = M[None, None].astype(np.float32)
+    sh, st = _quant(oracle, S, r=r, n_iter=3, smooth=0)
+    kc = st.comp_k_f32()[0, 0].astype(np.float64)
+    uc = st.comp_u_f32()[0, 0].astype(np.float64)
+    G = kc @ kc.T
+    assert np.allclose(np.diag(G), 1.0, atol=2e-3)
+    assert np.max(np.abs(G - np.diag(np.diag(G)))) < 5e-3
+    resid = M - kc.T @ uc
+    sh2, st2 = _quant(oracle, S, r=r - 1, n_iter=3, smooth=0)
+    resid_fewer = M - st2.comp_k_f32()[0, 0].astype(np.float64).T @ st2.comp_u_f32()[0, 0].astype(np.float64)
+    assert np.linalg.norm(resid) < np.linalg.norm(resid_fewer)
+    # the residual is what the codes hold: dequantized state = Z*step + K U^T, within half a code step of M
+    D = oracle.dequantize_state(sh, st)[0, 0].astype(np.float64)
+    assert np.all(np.abs(D - M) <= st.col_scale[0, 0][None, :] / 2.0 * (1 + 1e-5) + 1e-9)
+
+
+def test_state_without_a_second_direction_stops_after_the_first_token(oracle):
+    """A state that is exactly a multiple of one outer product has no second direction.  With fp16-exact
+    factors the first token removes it exactly, so every later token and every code must be zero."""
+    k = np.zeros(128, np.float32); k[5] = 1.0
+    u = (np.arange(128) % 7 - 3).astype(np.float32) / 8.0
+    S = np.outer(k, u)[None, None].astype(np.float32)
+    sh, st = _quant(oracle, S, r=4, n_iter=2, smooth=1)
+    k0, u0 = st.comp_k_f32()[0, 0, 0], st.comp_u_f32()[0, 0, 0]
+    sign = 1.0 if k0[5] > 0 else -1.0                         # the pair is fixed up to a common sign
+    assert np.array_equal(sign * k0, k) and np.array_equal(sign * u0, u)
+    assert not st.comp_k[0, 0, 1:].any() and not st.comp_u[0, 0, 1:].any()
+    assert not st.codes.any()
