@@ -71,6 +71,11 @@ typedef struct {
                 /* from the all-equal unit vector where there is no such record     */
   int gate;     /* lq_gate                                                        */
   int smooth;   /* 1: residual smoothing (Sec. 3.4); 0: c = 1 (ablation)          */
+  int delta;    /* 1: delta rule, the correction reads the state back with          */
+                /* b = alpha (.) k (DeltaNet, Gated DeltaNet, KDA);                 */
+                /* 0: b = 0, u = v (the other instances of the paper's Table 4:     */
+                /* linear attention, RetNet, Mamba2 with the scalar gate; GLA,      */
+                /* RWKV6, HGRN2 with the diagonal gate; pass beta = 1 for k~ = k)   */
 } lq_shape;
 
 /*

@@ -66,6 +66,8 @@ typedef struct {
   int n_iter;    /* power-iteration steps per compensator (>= 1)            */
   int gate;      /* LQO_GATE_SCALAR (GDN) or LQO_GATE_DIAG (KDA)            */
   int smooth;    /* 1: residual smoothing (Sec. 3.4); 0: c == 1             */
+  int delta;     /* 1: delta rule, read vector b = alpha (.) k (DeltaNet, Gated DeltaNet, KDA);
+                    0: b = 0, so u = v (linear attention, RetNet, Mamba2, GLA, RWKV6, HGRN2: Table 4) */
 } lqo_shape;
 
 typedef struct {
@@ -304,7 +306,7 @@ static void head_ref_step(const lqo_shape *sh, float *S, const token_in *t, floa
   for (int i = 0; i < K; i++) { kt[i] = t->beta * t->k[i]; bv[i] = t->a[i] * t->k[i]; }
   for (int j = 0; j < V; j++) {
     column_of(S, K, V, j, col);
-    u[j] = t->v[j] - lqo_csum_dot(col, bv, K);
+    u[j] = sh->delta ? t->v[j] - lqo_csum_dot(col, bv, K) : t->v[j];   /* b = 0: nothing is read back */
   }
   for (int i = 0; i < K; i++)
     for (int j = 0; j < V; j++) S[(size_t)i * V + j] = fmaf(kt[i], u[j], t->a[i] * S[(size_t)i * V + j]);
@@ -517,7 +519,7 @@ static void head_decode(const lqo_shape *sh, const head_view *hv, int n, const t
       rk = fmaf(hv->bu[(size_t)jj * V + j], pk[jj], rk);
       rq = fmaf(hv->bu[(size_t)jj * V + j], pq[jj], rq);
     }
-    u[j] = t->v[j] - rk;                 /* Eq. 3: u = v - S_{l-1}^T (alpha (.) k) */
+    u[j] = sh->delta ? t->v[j] - rk : t->v[j];   /* Eq. 3: u = v - S_{l-1}^T b, b = alpha (.) k or 0 */
     o[j] = fmaf(u[j], ktq, rq);          /* o = S_{l-1}^T (alpha (.) q) + u (kt^T q) */
   }
 
@@ -538,7 +540,7 @@ static void head_decode(const lqo_shape *sh, const head_view *hv, int n, const t
 static int shape_ok(const lqo_shape *sh) {
   return sh && sh->batch >= 0 && sh->heads_v > 0 && sh->heads_qk > 0 && sh->heads_v % sh->heads_qk == 0 &&
          sh->d_k > 0 && sh->d_v > 0 && sh->W > 0 && sh->r >= 0 && sh->n_iter >= 1 &&
-         (sh->gate == LQO_GATE_SCALAR || sh->gate == LQO_GATE_DIAG);
+         (sh->gate == LQO_GATE_SCALAR || sh->gate == LQO_GATE_DIAG) && (sh->delta == 0 || sh->delta == 1);
 }
 
 int lqo_threads(void) {

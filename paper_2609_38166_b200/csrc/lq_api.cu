@@ -149,7 +149,10 @@ __global__ void __launch_bounds__(256, 2) ref_kernel(const Params p) {
   col_blocks(M, x, pc);
   col_tree(pc, part_s, col_s, t, u);                           // S^T (alpha.k)
 #pragma unroll
-  for (int c = 0; c < 8; c++) u[c] = bf16_bits(p.v[bh * D + 8 * t.tx + c]) - u[c];
+  for (int c = 0; c < 8; c++) {                               // b = 0 (no delta rule): nothing is subtracted
+    const float vc = bf16_bits(p.v[bh * D + 8 * t.tx + c]);
+    u[c] = p.delta ? vc - u[c] : vc;
+  }
   load8(kt_s + 8 * t.ty, kt);
   load8(a_s + 8 * t.ty, ai);
 #pragma unroll
@@ -185,7 +188,8 @@ static bool aligned16(const void *ptr) { return (reinterpret_cast<uintptr_t>(ptr
 static lq_status check_shape(const lq_shape *s) {
   if (!s) return LQ_ERR_NULL;
   if (s->batch < 0 || s->heads_v <= 0 || s->heads_qk <= 0 || s->d_k <= 0 || s->d_v <= 0 || s->W <= 0 || s->r < 0 ||
-      s->n_iter < 1 || s->heads_v % s->heads_qk != 0 || (s->gate != LQ_GATE_SCALAR && s->gate != LQ_GATE_DIAG))
+      s->n_iter < 1 || s->heads_v % s->heads_qk != 0 || (s->gate != LQ_GATE_SCALAR && s->gate != LQ_GATE_DIAG) ||
+      (s->delta != 0 && s->delta != 1))
     return LQ_ERR_SHAPE;
   if (s->d_k != D || s->d_v != D || s->W > MAX_W || s->r > MAX_R) return LQ_ERR_UNSUPPORTED;
   return LQ_OK;
@@ -223,7 +227,7 @@ static lq_status check_state(const lq_shape *s, const lq_state *st, bool need_bu
 static Params make_params(const lq_shape *s, const lq_state *st) {
   Params p{};
   p.batch = s->batch; p.heads_v = s->heads_v; p.heads_qk = s->heads_qk; p.W = s->W; p.r = s->r;
-  p.n_iter = s->n_iter; p.smooth = s->smooth; p.force = 0;
+  p.n_iter = s->n_iter; p.smooth = s->smooth; p.delta = s->delta; p.force = 0;
   if (st) {
     p.heads = st->heads; p.records = st->records; p.decays = st->decays; p.win_pos = st->win_pos;
   }
@@ -800,6 +804,6 @@ const char *lq_status_string(lq_status status) {
   return "unknown status";
 }
 
-int lq_version(void) { return 1; }
+int lq_version(void) { return 2; }
 
 }  // extern "C"

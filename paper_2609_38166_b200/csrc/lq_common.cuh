@@ -35,7 +35,7 @@ constexpr int REC_KT = 0, REC_U = D, REC_A = 2 * D;
 
 // Launch-time description of one call, passed to the kernels by value.
 struct Params {
-  int batch, heads_v, heads_qk, W, r, n_iter, smooth, force;
+  int batch, heads_v, heads_qk, W, r, n_iter, smooth, delta, force;
   uint8_t *heads;    // [B*Hv] head blocks of head_bytes(r)
   float *records;    // [B*Hv][W] record rows of record_floats(gate)
   float *decays;     // scalar gate: [B*Hv][W]

@@ -556,7 +556,7 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
         const float ktq = pq[n + r];
         float u[4], o[4];
 #pragma unroll
-        for (int e = 0; e < 4; e++) { u[e] = v4[e] - rk[e]; o[e] = fmaf(u[e], ktq, rq[e]); }
+        for (int e = 0; e < 4; e++) { u[e] = p.delta ? v4[e] - rk[e] : v4[e]; o[e] = fmaf(u[e], ktq, rq[e]); }
         __syncwarp();                        // every lane is done reading the slot
         LQ_TICK(8);
         named_arrive(2);

@@ -31,7 +31,7 @@ class LqError(RuntimeError):
 
 class _Shape(C.Structure):
     _fields_ = [(n, C.c_int) for n in
-                ("batch", "heads_v", "heads_qk", "d_k", "d_v", "W", "r", "n_iter", "gate", "smooth")]
+                ("batch", "heads_v", "heads_qk", "d_k", "d_v", "W", "r", "n_iter", "gate", "smooth", "delta")]
 
 
 class _State(C.Structure):
@@ -75,10 +75,11 @@ class Shape:
     n_iter: int = 2
     gate: int = GATE_SCALAR
     smooth: int = 1
+    delta: int = 1
 
     def c(self) -> _Shape:
         return _Shape(self.batch, self.heads_v, self.heads_qk, self.d_k, self.d_v, self.W, self.r, self.n_iter,
-                      self.gate, self.smooth)
+                      self.gate, self.smooth, self.delta)
 
 
 def head_bytes(sh: Shape) -> int:
@@ -149,7 +150,7 @@ def _ptr(t: Optional[torch.Tensor], b0: int = 0) -> C.c_void_p:
 
 def _sub(sh: Shape, b0: int, nb: Optional[int]) -> Shape:
     nb = sh.batch - b0 if nb is None else nb
-    return Shape(nb, sh.heads_v, sh.heads_qk, sh.d_k, sh.d_v, sh.W, sh.r, sh.n_iter, sh.gate, sh.smooth)
+    return Shape(nb, sh.heads_v, sh.heads_qk, sh.d_k, sh.d_v, sh.W, sh.r, sh.n_iter, sh.gate, sh.smooth, sh.delta)
 
 
 def decode_step(sh: Shape, st: State, q, k, v, beta, alpha, o, stream=None, b0: int = 0, nb: Optional[int] = None):

@@ -46,6 +46,7 @@ class Workload:
     n_iter: int = 2
     gate: int = GATE_SCALAR
     smooth: int = 1
+    delta: int = 1                  # 1: delta rule (GDN, KDA); 0: no read-back, u = v (Mamba2, GLA, ...)
     v_dist: str = "normal"          # "normal" | "student3"
     outlier_frac: float = 0.0
     outlier_mag: float = 1.0

@@ -120,6 +120,30 @@ def test_staggered_batch_chain(oracle, gate, W, r):
     _run_chain(oracle, wl, 2 * W + 3 if W <= 16 else W + 5, init="dense", stagger=True, check_every=4)
 
 
+@pytest.mark.parametrize("gate", GATES)
+def test_chain_without_the_delta_rule(oracle, gate):
+    """b_t = 0 (Mamba2 / GLA style instances): u = v; decode, boundaries and both baseline kernels against the oracle."""
+    wl = synth.Workload("nd", 5, 4, 2, W=4, r=2, gate=gate, seed=470, delta=0)
+    _run_chain(oracle, wl, 14, init="dense", stagger=True, check_every=3)
+    osh, lsh = gu.shapes(wl)
+    S_o = synth.dense_states(wl, 2)
+    S_d = gu.dev(S_o.copy())
+    S16_o = synth.f32_to_bf16_bits(S_o)
+    S16_d = gu.dev(S16_o.copy())
+    o = torch.empty((wl.batch, wl.heads_v, 128), dtype=torch.float32, device="cuda")
+    for step in range(3):
+        tok = synth.token_inputs(wl, step)
+        td = gu.tok_dev(tok)
+        args = (td["q"], td["k"], td["v"], td["beta"], td["alpha"])
+        want = oracle.ref_step_f32(osh, S_o, **tok)
+        lq.ref_decode_step_f32(lsh, S_d, *args, o)
+        _close(o.cpu().numpy(), want, f"fp32 baseline without the delta rule, step {step}")
+        want16 = oracle.ref_step_bf16(osh, S16_o, **tok)
+        lq.ref_decode_step_bf16(lsh, S16_d, *args, o)
+        _close(o.cpu().numpy(), want16, f"bf16 baseline without the delta rule, step {step}")
+    assert np.array_equal(S_d.cpu().numpy(), S_o)
+
+
 def test_kda_outlier_chain(oracle):
     wl = synth.config("kda_b128_outlier").with_(batch=3, heads_v=4, heads_qk=4)
     _run_chain(oracle, wl, 40, stagger=True, check_every=5)

@@ -10,7 +10,7 @@ from tests import refmath as rm
 
 
 def _shape(wl):
-    return Shape(wl.batch, wl.heads_v, wl.heads_qk, wl.d_k, wl.d_v, wl.W, wl.r, wl.n_iter, wl.gate, wl.smooth)
+    return Shape(wl.batch, wl.heads_v, wl.heads_qk, wl.d_k, wl.d_v, wl.W, wl.r, wl.n_iter, wl.gate, wl.smooth, wl.delta)
 
 
 def _naive_quant64(S):

@@ -12,7 +12,7 @@ GATES = [synth.GATE_SCALAR, synth.GATE_DIAG]
 
 
 def _shape(wl):
-    return Shape(wl.batch, wl.heads_v, wl.heads_qk, wl.d_k, wl.d_v, wl.W, wl.r, wl.n_iter, wl.gate, wl.smooth)
+    return Shape(wl.batch, wl.heads_v, wl.heads_qk, wl.d_k, wl.d_v, wl.W, wl.r, wl.n_iter, wl.gate, wl.smooth, wl.delta)
 
 
 def _rel(a, b):
@@ -195,3 +195,46 @@ def test_boundary_term_is_exact_up_to_the_fixed_point_grid(oracle):
             got = v - st.buf_u[b, h, 0].astype(np.float64)
             grid = 2.0 ** -29 * 2 * np.abs(x).max() * np.abs(Z).sum(axis=0) * s
             assert np.all(np.abs(got - exact) <= grid + 3 * 2.0 ** -24 * (np.abs(exact) + np.abs(v)))
+
+
+@pytest.mark.parametrize("gate", GATES)
+def test_without_the_delta_rule_the_state_is_a_decayed_sum_of_outer_products(oracle, gate):
+    """b_t = 0 (Table 4: linear attention, RetNet, Mamba2 with the scalar gate; GLA, RWKV6, HGRN2 with the diagonal
+    one): nothing is read back, so S_t = sum_i (prod_{i<j<=t} D_j) k~_i v_i^T in closed form and
+    o_t = sum_i <prod D_j k~_i, q_t> v_i.  Checked for the dense reference step and, with a quantized state, for
+    the windowed decode (error within the 8-bit budget) and with the quantizer off (equal up to fp32 rounding)."""
+    wl = synth.Workload("t", 2, 4, 2, 128, 128, W=4, r=2, gate=gate, seed=61, delta=0)
+    sh = _shape(wl)
+    B, H, T = 2, 4, 11
+    toks = [synth.token_inputs(wl, t) for t in range(T)]
+    # closed form in float64
+    o_want = np.zeros((T, B, H, 128))
+    for b in range(B):
+        for h in range(H):
+            w = [rm.widen(tok, wl, b, h) for tok in toks]             # (q, k, v, beta, alpha) in float64
+            for t in range(T):
+                acc = np.zeros(128)
+                for i in range(t + 1):
+                    q_t = w[t][0]
+                    kt = w[i][3] * w[i][1]
+                    for j in range(i + 1, t + 1):
+                        kt = kt * w[j][4]                             # scalar or per-channel decay
+                    acc += (kt @ q_t) * w[i][2]
+                o_want[t, b, h] = acc
+    S = np.zeros((B, H, 128, 128), np.float32)
+    st_off = State(sh, quant=False)
+    st_q = State(sh)
+    oracle.quantize_state(sh, S, st_q)
+    for t in range(T):
+        o_ref = oracle.ref_step_f32(sh, S, **toks[t])
+        o_off = oracle.decode_step(sh, st_off, **toks[t])
+        o_q = oracle.decode_step(sh, st_q, **toks[t])
+        assert np.allclose(o_ref, o_want[t], rtol=1e-5, atol=1e-5)
+        assert np.allclose(o_off, o_want[t], rtol=1e-5, atol=1e-5)
+        assert _rel(o_q, o_want[t]) < 2e-3
+    # and the delta rule really is off: with it on, the same tokens give a different output
+    wl_on = wl.with_(delta=1)
+    S2 = np.zeros((B, H, 128, 128), np.float32)
+    for t in range(T):
+        o_on = oracle.ref_step_f32(_shape(wl_on), S2, **toks[t])
+    assert _rel(o_on, o_want[T - 1]) > 1e-2
