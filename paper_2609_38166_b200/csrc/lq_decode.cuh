@@ -76,8 +76,11 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, int count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
   asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
 }
+// The arrival that announces the bytes of the next copies.  Relaxed: nothing this thread wrote has to be
+// visible to anybody through this barrier (the copies' own completion is what the waiters acquire), and the
+// default release form stalls the warp for about 800 cycles here.
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+  asm volatile("mbarrier.arrive.expect_tx.relaxed.cta.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
 }
 // global -> shared bulk copy; addresses and size are multiples of 16 bytes
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
@@ -202,13 +205,14 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
   long long tick_ = clock64();
   unsigned acc_[12] = {0};
 #endif
-  // Requests head bh (n records buffered) into the slot: two bulk copies, issued by two lanes of the dot
-  // warp when nobody reads the slot any more.
+  // Requests head bh (n records buffered) into the slot: two bulk copies, issued by two lanes of the stream
+  // warp when nobody reads the slot any more.  (Asking for the codes alone right after the tensor-core pass,
+  // as a third copy on the same barrier phase, was measured and changes nothing: the wait is set by the part
+  // that can only be requested last.)
+  // The regions the copies overwrite were only READ through ordinary loads, whose values have been used
+  // before the call; the warps write only their scratch regions.  So nothing written by the generic proxy is
+  // at stake and no cross-proxy fence is needed (it costs over a thousand cycles here).
   auto request = [&](unsigned bh, int n) {
-    // The regions the copies overwrite were only READ through ordinary loads, whose values have been used
-    // before the barrier that precedes this call; the warps write only their scratch regions.  So nothing
-    // written by the generic proxy is at stake and no cross-proxy fence is needed (it costs over a
-    // thousand cycles here).
     const uint32_t hb = head_bytes(r), rb = 4u * RF * n;
     if (lane == 0) {
       mbar_expect_tx(bar, hb + rb);
@@ -247,7 +251,7 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
   if (hd.bh < nh) load_token<GATE>(p, hd, group, lane, role, nxt);
   {
     const int n0 = __shfl_sync(FULL, sc_n, 0) & 0xFFFF;
-    if (role == 1 && blockIdx.x < nh && n0 < W) request(blockIdx.x, n0);
+    if (role == 0 && blockIdx.x < nh && n0 < W) request(blockIdx.x, n0);
   }
 #ifdef LQ_TIMING
   tick_ = clock64();
@@ -268,7 +272,7 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
 
     if (!active) {                           // nothing was requested for this head; keep the pipeline going
       if (bh_next < nh) load_token<GATE>(p, hd1, group, lane, role, nxt);
-      if (role == 1 && next_active) request(bh_next, n_next);
+      if (role == 0 && next_active) request(bh_next, n_next);
       continue;
     }
 
@@ -358,6 +362,7 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
         float2 gam[4];
 #pragma unroll
         for (int cc = 0; cc < 4; cc++) gam[cc] = a2[cc];
+#pragma unroll 4
         for (int j = n - 1; j >= 0; j--) {
           float2 aj[4];
           if (DIAG) load8p(rec + j * RF + REC_A + 8 * c, aj);
@@ -400,12 +405,8 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
       }
       __syncwarp();
       LQ_TICK(4);
-      named_arrive(1);                       // the projections are in shared memory
+      named_arrive(1);                       // the projections are in shared memory; this warp is done with the slot
       LQ_TICK(5);
-      named_wait(2);                         // the stream warp has read all it needs from the slot
-      LQ_TICK(6);
-      // the request goes out before this warp's global stores: the proxy fence in it would wait for them
-      if (next_active) request(bh_next, n_next);
       // append the key side of the record (and its decay)
       {
         float *row = p.record(bh, n, DIAG);
@@ -557,9 +558,9 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
         float u[4], o[4];
 #pragma unroll
         for (int e = 0; e < 4; e++) { u[e] = p.delta ? v4[e] - rk[e] : v4[e]; o[e] = fmaf(u[e], ktq, rq[e]); }
-        __syncwarp();                        // every lane is done reading the slot
-        LQ_TICK(8);
-        named_arrive(2);
+        __syncwarp();                        // every lane is done reading the slot, and so is the dot warp (it
+        LQ_TICK(8);                          // arrived at barrier 1 after its last read): the next head may land
+        if (next_active) request(bh_next, n_next);
         *reinterpret_cast<float4 *>(p.o + bh * D + 4 * lane) = make_float4(o[0], o[1], o[2], o[3]);
         *reinterpret_cast<float4 *>(p.record(bh, n, DIAG) + REC_U + 4 * lane) = make_float4(u[0], u[1], u[2], u[3]);
       }
