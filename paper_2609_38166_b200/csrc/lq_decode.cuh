@@ -233,14 +233,9 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
     }
   };
 
-  // Arrival on win_pos (see arrive_and_set) is split: the atomic is issued when a head is done, its return
-  // value is looked at one head later, so that the warp does not sit out the round trip.
-  int pend_old = 0, pend_b = -1, pend_new = 0;
-  auto settle = [&]() {
-    if (pend_b >= 0 && (pend_old >> 16) == p.heads_v - 1) p.win_pos[pend_b] = pend_new;
-    pend_b = -1;
-  };
-
+  // Arrival on win_pos (see arrive_and_set): the counter says how many heads of the sequence have READ the old
+  // value, which this head did when its scalars were loaded.  The dot warp makes the arrival, at the end of its
+  // work: it has slack, the stream warp (the longer of the two) has none to sit out the atomic's round trip.
   // A head whose window is already full (n >= W) gets no token: it is neither requested nor waited for.
   load_scalars(blockIdx.x);
   TokenRaw nxt;                               // the token of the head about to start
@@ -295,7 +290,7 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
 
     // ---- wait for the slot (bounded: a copy that never lands must not hang the GPU) ----
     if (!mbar_wait(bar, parity)) {
-      if (lane == 0) { atomicOr(&g_device_error, 1); settle(); }
+      if (lane == 0) atomicOr(&g_device_error, 1);
       mbar_wait(bar, parity);                // one more bounded wait for the copies in flight, then give up
       return;
     }
@@ -416,6 +411,7 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
           else if (lane == 0) p.decays[bh * (size_t)W + n] = a8[0];
         }
       }
+      if (lane == 0) arrive_and_set(p.win_pos, b, p.heads_v, n + 1);
       LQ_TICK(7);
     } else {
       // =========================== STREAM WARP ===========================
@@ -564,16 +560,9 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
         *reinterpret_cast<float4 *>(p.o + bh * D + 4 * lane) = make_float4(o[0], o[1], o[2], o[3]);
         *reinterpret_cast<float4 *>(p.record(bh, n, DIAG) + REC_U + 4 * lane) = make_float4(u[0], u[1], u[2], u[3]);
       }
-      if (lane == 0) {
-        settle();
-        pend_old = atomicAdd(p.win_pos + b, 0x10000);
-        pend_b = b;
-        pend_new = n + 1;
-      }
       LQ_TICK(9);
     }
   }
-  if (role == 0 && lane == 0) settle();
 #ifdef LQ_TIMING
   if (lane == 0)
     for (int i = 0; i < 12; i++) atomicAdd(&g_phase_cycles[16 * role + i], (unsigned long long)acc_[i]);
