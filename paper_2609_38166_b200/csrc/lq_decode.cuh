@@ -286,6 +286,14 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
       bas[lane + 32] = nxt.ba_hi;
     }
     if (bh_next < nh) load_token<GATE>(p, hd1, group, lane, role, nxt);       // used one trip from now
+    // scalar gate: Gamma_{1:l}, the chain of decays from the newest record back (Appendix B.2), needs nothing
+    // from the slot, so the stream warp takes it before it waits
+    float gsc = alpha_s;
+    if (!DIAG && role == 0) {
+      __syncwarp();
+#pragma unroll 4
+      for (int j = n - 1; j >= 0; j--) gsc = gsc * bas[j];
+    }
     LQ_TICK(1);
 
     // ---- wait for the slot (bounded: a copy that never lands must not hang the GPU) ----
@@ -428,9 +436,6 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
           for (int e = 0; e < 8; e++) gam[e] = gam[e] * aj[e];
         }
       } else {
-        float gsc = a8[0];
-#pragma unroll 4
-        for (int j = n - 1; j >= 0; j--) gsc = gsc * bas[j];
 #pragma unroll
         for (int e = 0; e < 8; e++) gam[e] = gsc;
       }
@@ -476,8 +481,8 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
       // thread's 16 bytes of a row hold key channels 64p+16t..64p+16t+15 and serve two k-blocks; the digit
       // planes are read with the same permutation of the key index.  The two 64-channel halves of a tile
       // accumulate separately (exact integers: any split gives the same sum), which halves the dependent
-      // chain of MMAs.  Digit pairs are recombined in int32 (|sum| < 2^30), the two pairs in binary64, which
-      // holds the 47-bit total exactly, and one rounding takes it to fp32.
+      // chain of MMAs.  Digit pairs are recombined in int32 (|sum| < 2^30), the two pairs in int64 (the total has
+      // 47 bits), and one rounding takes it to fp32.
       {
         constexpr int h0 = 0, h1 = 64;         // the two 64-channel halves (the same split for every lane)
         const uint4 bfa = *reinterpret_cast<const uint4 *>(digits + g * D + h0 + 16 * t);
@@ -511,8 +516,8 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
           float *dst = y + (t >> 1) * D + g;
 #pragma unroll
           for (int mt = 0; mt < 8; mt++) {
-            dst[16 * mt] = __double2float_rn(fma(static_cast<double>(oth_lo[mt]), 65536.0, static_cast<double>(pair_lo[mt])));
-            dst[16 * mt + 8] = __double2float_rn(fma(static_cast<double>(oth_hi[mt]), 65536.0, static_cast<double>(pair_hi[mt])));
+            dst[16 * mt] = __ll2float_rn(static_cast<long long>(oth_lo[mt]) * 65536 + pair_lo[mt]);
+            dst[16 * mt + 8] = __ll2float_rn(static_cast<long long>(oth_hi[mt]) * 65536 + pair_hi[mt]);
           }
         }
       }
