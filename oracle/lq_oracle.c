@@ -515,10 +515,14 @@ static void head_decode(const lqo_shape *sh, const head_view *hv, int n, const t
         rq = fmaf(uc, ptq[h], rq);
       }
     }
-    for (int jj = 0; jj < n; jj++) {
-      rk = fmaf(hv->bu[(size_t)jj * V + j], pk[jj], rk);
-      rq = fmaf(hv->bu[(size_t)jj * V + j], pq[jj], rq);
+    /* the records' terms: their own sum, from the newest record back, added as one number */
+    float sk = 0.0f, sq = 0.0f;
+    for (int jj = n - 1; jj >= 0; jj--) {
+      sk = fmaf(hv->bu[(size_t)jj * V + j], pk[jj], sk);
+      sq = fmaf(hv->bu[(size_t)jj * V + j], pq[jj], sq);
     }
+    rk = rk + sk;
+    rq = rq + sq;
     u[j] = sh->delta ? t->v[j] - rk : t->v[j];   /* Eq. 3: u = v - S_{l-1}^T b, b = alpha (.) k or 0 */
     o[j] = fmaf(u[j], ktq, rq);          /* o = S_{l-1}^T (alpha (.) q) + u (kt^T q) */
   }

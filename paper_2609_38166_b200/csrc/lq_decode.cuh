@@ -289,10 +289,22 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
     // scalar gate: Gamma_{1:l}, the chain of decays from the newest record back (Appendix B.2), needs nothing
     // from the slot, so the stream warp takes it before it waits
     float gsc = alpha_s;
-    if (!DIAG && role == 0) {
+    if (!DIAG) {
       __syncwarp();
 #pragma unroll 4
       for (int j = n - 1; j >= 0; j--) gsc = gsc * bas[j];
+    }
+    // kt^T q needs only the token: the dot warp takes it before the wait as well.  It goes to one of two places
+    // in turn, because the stream warp may still be reading the previous head's.
+    if (role == 1) {
+      float2 k2p[4], q2p[4];
+#pragma unroll
+      for (int cc = 0; cc < 4; cc++) {
+        k2p[cc] = __fmul2_rn(pair(beta), make_float2(k8[2 * cc], k8[2 * cc + 1]));
+        q2p[cc] = make_float2(q8[2 * cc], q8[2 * cc + 1]);
+      }
+      const float ktq_pre = tree16(block8(k2p, q2p));
+      if (lane == 0) pq[r + (idx & 1)] = ktq_pre;
     }
     LQ_TICK(1);
 
@@ -322,6 +334,7 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
         g2[cc] = a2[cc];
         kt2[cc] = __fmul2_rn(pair(beta), k2[cc]);
       }
+      float rk_rec[4] = {0.0f, 0.0f, 0.0f, 0.0f}, rq_rec[4] = {0.0f, 0.0f, 0.0f, 0.0f};
       for (int jt = n - 1; jt >= 0; jt -= 4) {       // records jt, jt-1, jt-2, jt-3
         float s4[4];
         int jo[2];
@@ -354,61 +367,77 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
           s4[2 * u + 1] = block8(x2, yq2);
         }
         tree16x4(s4);
+        // The record terms sum_j u_j (kt_j^T Gamma k) and the same for q, channels 4 lane .. 4 lane + 3, as one
+        // chain from the newest record back.  Half 0 holds the projections of records jt and jt-2, half 1
+        // those of jt-1 and jt-3: swap them, then take the four records in order.
+        {
+          float oth[4];
 #pragma unroll
-        for (int u = 0; u < 2; u++)
-          if (c == 0 && jo[u] >= 0) { pk[jo[u]] = s4[2 * u]; pq[jo[u]] = s4[2 * u + 1]; }
+          for (int e = 0; e < 4; e++) oth[e] = __shfl_xor_sync(FULL, s4[e], 16);
+#pragma unroll
+          for (int i4 = 0; i4 < 4; i4++) {
+            const int j = jt - i4;
+            if (j < 0) break;                                  // the same for every lane
+            const int u = i4 >> 1;
+            const bool mine = (i4 & 1) == half;
+            const float pkj = mine ? s4[2 * u] : oth[2 * u], pqj = mine ? s4[2 * u + 1] : oth[2 * u + 1];
+            const float4 u4 = *reinterpret_cast<const float4 *>(rec + j * RF + REC_U + 4 * lane);
+            rk_rec[0] = fmaf(u4.x, pkj, rk_rec[0]); rq_rec[0] = fmaf(u4.x, pqj, rq_rec[0]);
+            rk_rec[1] = fmaf(u4.y, pkj, rk_rec[1]); rq_rec[1] = fmaf(u4.y, pqj, rq_rec[1]);
+            rk_rec[2] = fmaf(u4.z, pkj, rk_rec[2]); rq_rec[2] = fmaf(u4.z, pqj, rq_rec[2]);
+            rk_rec[3] = fmaf(u4.w, pkj, rk_rec[3]); rq_rec[3] = fmaf(u4.w, pqj, rq_rec[3]);
+          }
+        }
       }
       LQ_TICK(3);
-      // Compensator keys against Gamma_{1:l} k and Gamma_{1:l} q; item r is kt^T q (kept in pq[n+r]).
-      // g2 may have run past record 0 above: Gamma_{1:l} is rebuilt from the exact chain.
-      {
+      // Compensator keys against Gamma_{1:l} k and Gamma_{1:l} q (the projections go to pk[h], pq[h]).
+      // g2 may have run past record 0 above: Gamma_{1:l} is taken from the exact chain.
+      if (r > 0) {
         float2 gam[4];
+        if (DIAG) {
 #pragma unroll
-        for (int cc = 0; cc < 4; cc++) gam[cc] = a2[cc];
+          for (int cc = 0; cc < 4; cc++) gam[cc] = a2[cc];
 #pragma unroll 4
-        for (int j = n - 1; j >= 0; j--) {
-          float2 aj[4];
-          if (DIAG) load8p(rec + j * RF + REC_A + 8 * c, aj);
-          else {
-            const float2 x = pair(bas[j]);
+          for (int j = n - 1; j >= 0; j--) {
+            float2 aj[4];
+            load8p(rec + j * RF + REC_A + 8 * c, aj);
 #pragma unroll
-            for (int cc = 0; cc < 4; cc++) aj[cc] = x;
+            for (int cc = 0; cc < 4; cc++) gam[cc] = __fmul2_rn(gam[cc], aj[cc]);
           }
+        } else {
 #pragma unroll
-          for (int cc = 0; cc < 4; cc++) gam[cc] = __fmul2_rn(gam[cc], aj[cc]);
+          for (int cc = 0; cc < 4; cc++) gam[cc] = pair(gsc);
         }
         float2 gk2[4], gq2[4];
 #pragma unroll
         for (int cc = 0; cc < 4; cc++) { gk2[cc] = __fmul2_rn(gam[cc], k2[cc]); gq2[cc] = __fmul2_rn(gam[cc], q2[cc]); }
-        for (int hb = 0; hb < r + 1; hb += 4) {
+        for (int hb = 0; hb < r; hb += 4) {
           float s4[4];
           int ho[2];
 #pragma unroll
           for (int u = 0; u < 2; u++) {
             ho[u] = hb + 2 * u + half;
-            const int h = ho[u] < r ? ho[u] : (r > 0 ? r - 1 : 0);
+            const int h = ho[u] < r ? ho[u] : r - 1;
             float x8[8];
-            if (r > 0) widen8_f16(*reinterpret_cast<const uint4 *>(ckh + h * D + 8 * c), x8);
-            const bool is_ktq = ho[u] >= r;
-            float2 x2[4], yk2[4], yq2[4];
+            widen8_f16(*reinterpret_cast<const uint4 *>(ckh + h * D + 8 * c), x8);
+            float2 x2[4];
 #pragma unroll
-            for (int cc = 0; cc < 4; cc++) {
-              x2[cc] = is_ktq ? kt2[cc] : make_float2(x8[2 * cc], x8[2 * cc + 1]);
-              yk2[cc] = is_ktq ? q2[cc] : gk2[cc];
-              yq2[cc] = is_ktq ? q2[cc] : gq2[cc];
-            }
-            s4[2 * u] = block8(x2, yk2);
-            s4[2 * u + 1] = block8(x2, yq2);
+            for (int cc = 0; cc < 4; cc++) x2[cc] = make_float2(x8[2 * cc], x8[2 * cc + 1]);
+            s4[2 * u] = block8(x2, gk2);
+            s4[2 * u + 1] = block8(x2, gq2);
           }
           tree16x4(s4);
 #pragma unroll
           for (int u = 0; u < 2; u++)
-            if (c == 0 && ho[u] <= r) { pk[n + ho[u]] = s4[2 * u]; pq[n + ho[u]] = s4[2 * u + 1]; }
+            if (c == 0 && ho[u] < r) { pk[ho[u]] = s4[2 * u]; pq[ho[u]] = s4[2 * u + 1]; }
         }
       }
+      named_wait(2);                         // the stream warp has taken its sums out of y
+      *reinterpret_cast<float4 *>(y + 4 * lane) = make_float4(rk_rec[0], rk_rec[1], rk_rec[2], rk_rec[3]);
+      *reinterpret_cast<float4 *>(y + D + 4 * lane) = make_float4(rq_rec[0], rq_rec[1], rq_rec[2], rq_rec[3]);
       __syncwarp();
       LQ_TICK(4);
-      named_arrive(1);                       // the projections are in shared memory; this warp is done with the slot
+      named_arrive(1);                       // projections and record terms are in shared memory; this warp is done with the slot
       LQ_TICK(5);
       // append the key side of the record (and its decay)
       {
@@ -535,7 +564,8 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
         const float v4[4] = {__uint_as_float(v_raw.x << 16), __uint_as_float(v_raw.x & 0xFFFF0000u),
                              __uint_as_float(v_raw.y << 16), __uint_as_float(v_raw.y & 0xFFFF0000u)};
         LQ_TICK(6);
-        named_wait(1);                       // pk, pq are complete
+        named_arrive(2);                     // y has been read: the dot warp may put the record terms there
+        named_wait(1);                       // the compensator projections and the record terms are complete
         LQ_TICK(7);
 #pragma unroll 2
         for (int h = 0; h < r; h++) {
@@ -543,19 +573,17 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
           const float2 f01 = __half22float2(*reinterpret_cast<const __half2 *>(&w.x));
           const float2 f23 = __half22float2(*reinterpret_cast<const __half2 *>(&w.y));
           const float uc[4] = {f01.x, f01.y, f23.x, f23.y};
-          const float pkh = pk[n + h], pqh = pq[n + h];
+          const float pkh = pk[h], pqh = pq[h];
 #pragma unroll
           for (int e = 0; e < 4; e++) { rk[e] = fmaf(uc[e], pkh, rk[e]); rq[e] = fmaf(uc[e], pqh, rq[e]); }
         }
-#pragma unroll 4
-        for (int jj = 0; jj < n; jj++) {
-          const float4 u4 = *reinterpret_cast<const float4 *>(rec + jj * RF + REC_U + 4 * lane);
-          const float uj[4] = {u4.x, u4.y, u4.z, u4.w};
-          const float pkj = pk[jj], pqj = pq[jj];
-#pragma unroll
-          for (int e = 0; e < 4; e++) { rk[e] = fmaf(uj[e], pkj, rk[e]); rq[e] = fmaf(uj[e], pqj, rq[e]); }
+        {
+          const float4 tk = *reinterpret_cast<const float4 *>(y + 4 * lane);
+          const float4 tq = *reinterpret_cast<const float4 *>(y + D + 4 * lane);
+          rk[0] = rk[0] + tk.x; rk[1] = rk[1] + tk.y; rk[2] = rk[2] + tk.z; rk[3] = rk[3] + tk.w;
+          rq[0] = rq[0] + tq.x; rq[1] = rq[1] + tq.y; rq[2] = rq[2] + tq.z; rq[3] = rq[3] + tq.w;
         }
-        const float ktq = pq[n + r];
+        const float ktq = pq[r + (idx & 1)];
         float u[4], o[4];
 #pragma unroll
         for (int e = 0; e < 4; e++) { u[e] = p.delta ? v4[e] - rk[e] : v4[e]; o[e] = fmaf(u[e], ktq, rq[e]); }
