@@ -191,12 +191,12 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
   int8_t *digits = reinterpret_cast<int8_t *>(slot + L.digits);
   float *y = reinterpret_cast<float *>(slot + L.y), *pk = reinterpret_cast<float *>(slot + L.pk);
   float *pq = reinterpret_cast<float *>(slot + L.pq);
-  const uint32_t bar = smem_addr(slot + L.mbar), slot_a = smem_addr(slot);
+  const uint32_t barA = smem_addr(slot + L.mbar), barR = barA + 8, slot_a = smem_addr(slot);   // head block, records
 
-  if (threadIdx.x == 0) mbar_init(bar, 1);
+  if (threadIdx.x == 0) { mbar_init(barA, 1); mbar_init(barR, 1); }
   __syncthreads();
   grid_dependency_wait();                    // no global memory is touched above this line
-  uint32_t parity = 0;
+  uint32_t parA = 0, parR = 0;
   const unsigned nh = static_cast<unsigned>(p.batch) * p.heads_v, G = gridDim.x, Hv = p.heads_v;
   const unsigned G_b = G / Hv, G_hv = G % Hv;       // one grid stride in (sequence, head) steps
   const int group = p.heads_v / p.heads_qk;
@@ -205,20 +205,34 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
   long long tick_ = clock64();
   unsigned acc_[12] = {0};
 #endif
-  // Requests head bh (n records buffered) into the slot: two bulk copies, issued by two lanes of the stream
-  // warp when nobody reads the slot any more.  (Asking for the codes alone right after the tensor-core pass,
-  // as a third copy on the same barrier phase, was measured and changes nothing: the wait is set by the part
-  // that can only be requested last.)
+  // The slot is filled by two bulk copies with a barrier each, because its two parts become free at different
+  // times.  The head block (codes, scales, compensators) of the next head is requested by the stream warp as soon
+  // as both warps have taken the last thing they need from it (the compensator rows), the records by the dot
+  // warp as soon as it has walked them: about half of a head's work later the wait for the next head starts, and
+  // by then the copies have been on their way for a while.
   // The regions the copies overwrite were only READ through ordinary loads, whose values have been used
   // before the call; the warps write only their scratch regions.  So nothing written by the generic proxy is
   // at stake and no cross-proxy fence is needed (it costs over a thousand cycles here).
-  auto request = [&](unsigned bh, int n) {
-    const uint32_t hb = head_bytes(r), rb = 4u * RF * n;
+  auto request_head = [&](unsigned bh) {
     if (lane == 0) {
-      mbar_expect_tx(bar, hb + rb);
-      bulk_g2s(slot_a + L.head, p.head(bh), hb, bar);
+      mbar_expect_tx(barA, head_bytes(r));
+      bulk_g2s(slot_a + L.head, p.head(bh), head_bytes(r), barA);
     }
-    if (lane == 1 && n > 0) bulk_g2s(slot_a + L.rec, p.record(bh, 0, DIAG), rb, bar);
+  };
+  auto request_records = [&](unsigned bh, int n) {
+    if (lane == 0) {
+      const uint32_t rb = 4u * RF * n;
+      mbar_expect_tx(barR, rb);              // with no records the phase completes at once
+      if (n > 0) bulk_g2s(slot_a + L.rec, p.record(bh, 0, DIAG), rb, barR);
+    }
+  };
+  // Bounded wait for one of the two.  A copy that never lands must not hang the GPU: when the limit runs out the
+  // error flag is set and the warp goes on (its results are garbage, the flag says so); the other warp, which
+  // meets this one at the named barriers, is not left waiting.
+  auto wait_for = [&](uint32_t bar_, uint32_t &par) {
+    if (!mbar_wait(bar_, par) && lane == 0) atomicOr(&g_device_error, 1);
+    par ^= 1u;
+    __syncwarp();
   };
 
   // Per-head scalars of this CTA's heads, 32 heads at a time: lane l holds those of the CTA's (32*batch+l)-th head
@@ -246,7 +260,10 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
   if (hd.bh < nh) load_token<GATE>(p, hd, group, lane, role, nxt);
   {
     const int n0 = __shfl_sync(FULL, sc_n, 0) & 0xFFFF;
-    if (role == 0 && blockIdx.x < nh && n0 < W) request(blockIdx.x, n0);
+    if (blockIdx.x < nh && n0 < W) {
+      if (role == 0) request_head(blockIdx.x);
+      else request_records(blockIdx.x, n0);
+    }
   }
 #ifdef LQ_TIMING
   tick_ = clock64();
@@ -267,7 +284,10 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
 
     if (!active) {                           // nothing was requested for this head; keep the pipeline going
       if (bh_next < nh) load_token<GATE>(p, hd1, group, lane, role, nxt);
-      if (role == 0 && next_active) request(bh_next, n_next);
+      if (next_active) {
+        if (role == 0) request_head(bh_next);
+        else request_records(bh_next, n_next);
+      }
       continue;
     }
 
@@ -308,14 +328,8 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
     }
     LQ_TICK(1);
 
-    // ---- wait for the slot (bounded: a copy that never lands must not hang the GPU) ----
-    if (!mbar_wait(bar, parity)) {
-      if (lane == 0) atomicOr(&g_device_error, 1);
-      mbar_wait(bar, parity);                // one more bounded wait for the copies in flight, then give up
-      return;
-    }
-    parity ^= 1u;
-    __syncwarp();
+    // ---- wait for the head block; the records are waited for where they are first needed ----
+    wait_for(barA, parA);
     LQ_TICK(2);
 
     if (role == 1) {
@@ -334,6 +348,53 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
         g2[cc] = a2[cc];
         kt2[cc] = __fmul2_rn(pair(beta), k2[cc]);
       }
+      if (DIAG) wait_for(barR, parR);        // diagonal gate: Gamma_{1:l} is built from the records' decays
+      // Compensator keys against Gamma_{1:l} k and Gamma_{1:l} q (the projections go to pk[h], pq[h]).
+      // g2 may have run past record 0 above: Gamma_{1:l} is taken from the exact chain.
+      if (r > 0) {
+        float2 gam[4];
+        if (DIAG) {
+#pragma unroll
+          for (int cc = 0; cc < 4; cc++) gam[cc] = a2[cc];
+#pragma unroll 4
+          for (int j = n - 1; j >= 0; j--) {
+            float2 aj[4];
+            load8p(rec + j * RF + REC_A + 8 * c, aj);
+#pragma unroll
+            for (int cc = 0; cc < 4; cc++) gam[cc] = __fmul2_rn(gam[cc], aj[cc]);
+          }
+        } else {
+#pragma unroll
+          for (int cc = 0; cc < 4; cc++) gam[cc] = pair(gsc);
+        }
+        float2 gk2[4], gq2[4];
+#pragma unroll
+        for (int cc = 0; cc < 4; cc++) { gk2[cc] = __fmul2_rn(gam[cc], k2[cc]); gq2[cc] = __fmul2_rn(gam[cc], q2[cc]); }
+        for (int hb = 0; hb < r; hb += 4) {
+          float s4[4];
+          int ho[2];
+#pragma unroll
+          for (int u = 0; u < 2; u++) {
+            ho[u] = hb + 2 * u + half;
+            const int h = ho[u] < r ? ho[u] : r - 1;
+            float x8[8];
+            widen8_f16(*reinterpret_cast<const uint4 *>(ckh + h * D + 8 * c), x8);
+            float2 x2[4];
+#pragma unroll
+            for (int cc = 0; cc < 4; cc++) x2[cc] = make_float2(x8[2 * cc], x8[2 * cc + 1]);
+            s4[2 * u] = block8(x2, gk2);
+            s4[2 * u + 1] = block8(x2, gq2);
+          }
+          tree16x4(s4);
+#pragma unroll
+          for (int u = 0; u < 2; u++)
+            if (c == 0 && ho[u] < r) { pk[ho[u]] = s4[2 * u]; pq[ho[u]] = s4[2 * u + 1]; }
+        }
+      }
+      __syncwarp();
+      named_arrive(3);                       // the compensator projections are in pk, pq; this warp is done with the head block
+      LQ_TICK(4);
+      if (!DIAG) wait_for(barR, parR);
       float rk_rec[4] = {0.0f, 0.0f, 0.0f, 0.0f}, rq_rec[4] = {0.0f, 0.0f, 0.0f, 0.0f};
       for (int jt = n - 1; jt >= 0; jt -= 4) {       // records jt, jt-1, jt-2, jt-3
         float s4[4];
@@ -390,54 +451,13 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
         }
       }
       LQ_TICK(3);
-      // Compensator keys against Gamma_{1:l} k and Gamma_{1:l} q (the projections go to pk[h], pq[h]).
-      // g2 may have run past record 0 above: Gamma_{1:l} is taken from the exact chain.
-      if (r > 0) {
-        float2 gam[4];
-        if (DIAG) {
-#pragma unroll
-          for (int cc = 0; cc < 4; cc++) gam[cc] = a2[cc];
-#pragma unroll 4
-          for (int j = n - 1; j >= 0; j--) {
-            float2 aj[4];
-            load8p(rec + j * RF + REC_A + 8 * c, aj);
-#pragma unroll
-            for (int cc = 0; cc < 4; cc++) gam[cc] = __fmul2_rn(gam[cc], aj[cc]);
-          }
-        } else {
-#pragma unroll
-          for (int cc = 0; cc < 4; cc++) gam[cc] = pair(gsc);
-        }
-        float2 gk2[4], gq2[4];
-#pragma unroll
-        for (int cc = 0; cc < 4; cc++) { gk2[cc] = __fmul2_rn(gam[cc], k2[cc]); gq2[cc] = __fmul2_rn(gam[cc], q2[cc]); }
-        for (int hb = 0; hb < r; hb += 4) {
-          float s4[4];
-          int ho[2];
-#pragma unroll
-          for (int u = 0; u < 2; u++) {
-            ho[u] = hb + 2 * u + half;
-            const int h = ho[u] < r ? ho[u] : r - 1;
-            float x8[8];
-            widen8_f16(*reinterpret_cast<const uint4 *>(ckh + h * D + 8 * c), x8);
-            float2 x2[4];
-#pragma unroll
-            for (int cc = 0; cc < 4; cc++) x2[cc] = make_float2(x8[2 * cc], x8[2 * cc + 1]);
-            s4[2 * u] = block8(x2, gk2);
-            s4[2 * u + 1] = block8(x2, gq2);
-          }
-          tree16x4(s4);
-#pragma unroll
-          for (int u = 0; u < 2; u++)
-            if (c == 0 && ho[u] < r) { pk[ho[u]] = s4[2 * u]; pq[ho[u]] = s4[2 * u + 1]; }
-        }
-      }
+      if (DIAG) named_wait(4);               // diagonal gate: the stream warp read the records' decays too
+      if (next_active) request_records(bh_next, n_next);
       named_wait(2);                         // the stream warp has taken its sums out of y
       *reinterpret_cast<float4 *>(y + 4 * lane) = make_float4(rk_rec[0], rk_rec[1], rk_rec[2], rk_rec[3]);
       *reinterpret_cast<float4 *>(y + D + 4 * lane) = make_float4(rq_rec[0], rq_rec[1], rq_rec[2], rq_rec[3]);
       __syncwarp();
-      LQ_TICK(4);
-      named_arrive(1);                       // projections and record terms are in shared memory; this warp is done with the slot
+      named_arrive(1);                       // the record terms are in shared memory
       LQ_TICK(5);
       // append the key side of the record (and its decay)
       {
@@ -457,6 +477,7 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
 #pragma unroll
       for (int e = 0; e < 8; e++) gam[e] = a8[e];
       if (DIAG) {
+        wait_for(barR, parR);
 #pragma unroll 2
         for (int j = n - 1; j >= 0; j--) {
           float aj[8];
@@ -464,6 +485,8 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
 #pragma unroll
           for (int e = 0; e < 8; e++) gam[e] = gam[e] * aj[e];
         }
+        __syncwarp();
+        named_arrive(4);                     // this warp is done with the records
       } else {
 #pragma unroll
         for (int e = 0; e < 8; e++) gam[e] = gsc;
@@ -565,7 +588,7 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
                              __uint_as_float(v_raw.y << 16), __uint_as_float(v_raw.y & 0xFFFF0000u)};
         LQ_TICK(6);
         named_arrive(2);                     // y has been read: the dot warp may put the record terms there
-        named_wait(1);                       // the compensator projections and the record terms are complete
+        named_wait(3);                       // the compensator projections are complete
         LQ_TICK(7);
 #pragma unroll 2
         for (int h = 0; h < r; h++) {
@@ -577,6 +600,9 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
 #pragma unroll
           for (int e = 0; e < 4; e++) { rk[e] = fmaf(uc[e], pkh, rk[e]); rq[e] = fmaf(uc[e], pqh, rq[e]); }
         }
+        __syncwarp();                        // nobody reads the head block any more (the dot warp finished with
+        if (next_active) request_head(bh_next);   // it before barrier 3): the next head's may land
+        named_wait(1);                       // the record terms are complete
         {
           const float4 tk = *reinterpret_cast<const float4 *>(y + 4 * lane);
           const float4 tq = *reinterpret_cast<const float4 *>(y + D + 4 * lane);
@@ -587,9 +613,7 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
         float u[4], o[4];
 #pragma unroll
         for (int e = 0; e < 4; e++) { u[e] = p.delta ? v4[e] - rk[e] : v4[e]; o[e] = fmaf(u[e], ktq, rq[e]); }
-        __syncwarp();                        // every lane is done reading the slot, and so is the dot warp (it
-        LQ_TICK(8);                          // arrived at barrier 1 after its last read): the next head may land
-        if (next_active) request(bh_next, n_next);
+        LQ_TICK(8);
         *reinterpret_cast<float4 *>(p.o + bh * D + 4 * lane) = make_float4(o[0], o[1], o[2], o[3]);
         *reinterpret_cast<float4 *>(p.record(bh, n, DIAG) + REC_U + 4 * lane) = make_float4(u[0], u[1], u[2], u[3]);
       }
