@@ -121,11 +121,12 @@ __device__ __forceinline__ void reconstruct_tile(const Params &p, const Boundary
     // column v = 8 tx + b of the tile: bytes 8 ty .. 8 ty + 7 of row v of Z^T (chunk ty / 2, swizzled by tx)
     const uint2 zz = *reinterpret_cast<const uint2 *>(sm.zt + (8 * t.tx + b) * D + 16 * ((t.ty >> 1) ^ (t.tx & 7)) +
                                                       8 * (t.ty & 1));
-    const uint32_t lo = zz.x, hi = zz.y;
+    // int8 -> fp32 without the conversion unit: byte + 128 placed in the low mantissa bits of 2^23, minus 2^23 + 128
+    const uint32_t lo = zz.x ^ 0x80808080u, hi = zz.y ^ 0x80808080u;
 #pragma unroll
     for (int a = 0; a < 8; a++) {
       const uint32_t word = a < 4 ? lo : hi;
-      const float zf = static_cast<float>(static_cast<int8_t>((word >> (8 * (a & 3))) & 0xFF));
+      const float zf = __uint_as_float(__byte_perm(word, 0x4B000000u, 0x7540 | (a & 3))) - 8388736.0f;
       M[a][b] = ci[a] * (zf * sj[b]);
     }
   }
@@ -298,7 +299,8 @@ __device__ __forceinline__ void quantize_tile(const Params &p, const BoundarySme
     // |X * inv| <= 127 (1 + 2^-23), so the nearest integer (ties to even) is already inside [-127, 127]
     int z[8];
 #pragma unroll
-    for (int a = 0; a < 8; a++) z[a] = __float2int_rn(M[a][b] * inv[b]);
+    for (int a = 0; a < 8; a++) z[a] = __float_as_int(M[a][b] * inv[b] + 12582912.0f);   // + 1.5 * 2^23: the low
+    // mantissa byte of the sum is the nearest integer (ties to even) in two's complement
     const uint32_t lo = __byte_perm(__byte_perm(z[0], z[1], 0x0040), __byte_perm(z[2], z[3], 0x0040), 0x5410);
     const uint32_t hi = __byte_perm(__byte_perm(z[4], z[5], 0x0040), __byte_perm(z[6], z[7], 0x0040), 0x5410);
     *reinterpret_cast<uint2 *>(ZT + (8 * t.tx + b) * D + 8 * t.ty) = make_uint2(lo, hi);
