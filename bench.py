@@ -697,6 +697,56 @@ def run_ladder(args):
             f"{r['state_bytes_per_head']:8d}   {r['rel_err_o_vs_fp32']:.3e}")
 
 
+# --------------------------------------------------------------------------------------------------
+# Long-chain drift: GDN, 64 x 16 heads, heavy-tailed values, 4096 consecutive tokens, W = 16.  Error of o of
+# the 8-bit per-window path (and of the bf16-state baseline) against the fp32 recurrence fed the same tokens,
+# per block of 256 steps.  All on the GPU through the library; the code parity of the same chain against the
+# oracle is a test (tests/test_gpu_parity.py, tests/test_gpu_fullsize.py).
+# --------------------------------------------------------------------------------------------------
+def run_drift(args):
+    import torch
+    from paper_2609_38166_b200 import build, lq
+
+    torch.cuda.set_device(0)
+    build.build()
+    lq.lib()
+    wl = synth.config("gdn_drift")
+    sh = lq.Shape(wl.batch, wl.heads_v, wl.heads_qk, 128, 128, wl.W, wl.r, wl.n_iter, wl.gate, wl.smooth)
+    st = lq.State(sh)
+    S = torch.zeros((wl.batch, wl.heads_v, 128, 128), dtype=torch.float32, device="cuda")
+    S16 = torch.zeros((wl.batch, wl.heads_v, 128, 128), dtype=torch.int16, device="cuda")
+    lq.quantize_state(sh, S, st)
+    o_ref = torch.empty((wl.batch, wl.heads_v, 128), dtype=torch.float32, device="cuda")
+    o_q, o_b = torch.empty_like(o_ref), torch.empty_like(o_ref)
+    steps, block = args.drift_steps, 256
+    acc = {"8bit": [], "bf16": []}
+    rows = []
+    for t in range(steps):
+        d = to_dev(synth.token_inputs(wl, t), torch)
+        a = (d["q"], d["k"], d["v"], d["beta"], d["alpha"])
+        lq.ref_decode_step_f32(sh, S, *a, o_ref)
+        lq.decode_step(sh, st, *a, o_q)
+        lq.ref_decode_step_bf16(sh, S16, *a, o_b)
+        den = o_ref.flatten(2).norm(dim=2)                       # per (sequence, head)
+        acc["8bit"].append((o_q - o_ref).flatten(2).norm(dim=2) / den)
+        acc["bf16"].append((o_b - o_ref).flatten(2).norm(dim=2) / den)
+        if (t + 1) % block == 0:
+            row = {"drift": True, "workload": wl.name, "steps": [t + 1 - block, t + 1]}
+            for k in acc:
+                e = torch.stack(acc[k])                           # [block, B, H]
+                row[k] = {"mean": float(e.mean()), "max_over_heads_of_block_mean": float(e.mean(dim=0).max())}
+                acc[k] = []
+            rows.append(row)
+            print(json.dumps(row), flush=True)
+    flags = lq.check_device()
+    print(f"[drift] device error flags {flags}", file=sys.stderr)
+    print("[drift] steps            8-bit per window: mean   max head     bf16 state: mean   max head", file=sys.stderr)
+    for r_ in rows:
+        print(f"[drift] {r_['steps'][0]:5d}-{r_['steps'][1]:5d}        {r_['8bit']['mean']:.3e}  "
+              f"{r_['8bit']['max_over_heads_of_block_mean']:.3e}           {r_['bf16']['mean']:.3e}  "
+              f"{r_['bf16']['max_over_heads_of_block_mean']:.3e}", file=sys.stderr)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -717,6 +767,10 @@ def main():
     ap.add_argument("--ladder", action="store_true",
                     help="ablation ladder: fp32 / bf16 / int8 per token / int8 per window / + compensators / + smoothing, "
                          "speed and error against the fp32 recurrence (one JSON line per rung)")
+    ap.add_argument("--drift", action="store_true",
+                    help="long-chain drift of the 8-bit path and of the bf16-state baseline against the fp32 recurrence, "
+                         "per 256 steps (GDN 64 x 16 heads, Student-t values)")
+    ap.add_argument("--drift-steps", type=int, default=4096)
     ap.add_argument("--sweep-batches", default="32,128,256,512,1024")
     ap.add_argument("--sweep-W", default="8,16,32,64")
     ap.add_argument("--sweep-r", default="4,8")
@@ -728,6 +782,9 @@ def main():
         return
     if args.ladder:
         run_ladder(args)
+        return
+    if args.drift:
+        run_drift(args)
         return
     wl = synth.config("gdn_b256").with_(W=args.W, batch=args.batch, r=args.r)
     if args.gate == "kda":
