@@ -43,22 +43,29 @@ def state_bytes(r: int) -> int:
 
 def metric_name(wl) -> str:
     """The headline metric's name; other shapes (flags --gate/--batch/--W/--r) are named after themselves."""
-    if wl.gate == synth.GATE_SCALAR and wl.batch == 256 and wl.W == 16 and wl.r == 4:
+    if wl.gate == synth.GATE_SCALAR and wl.batch == 256 and wl.W == 16 and wl.r == 4 and not wl.rec16:
         return METRIC
-    return "%s decode state-GB/s at bs%d (8-bit per-window state, W=%d, r=%d)" % (
-        "GDN" if wl.gate == synth.GATE_SCALAR else "KDA", wl.batch, wl.W, wl.r)
+    return "%s decode state-GB/s at bs%d (8-bit per-window state, W=%d, r=%d%s)" % (
+        "GDN" if wl.gate == synth.GATE_SCALAR else "KDA", wl.batch, wl.W, wl.r, ", fp16 records" if wl.rec16 else "")
 
 # DRAM bytes per launch from the ncu captures summarised under profiles/ (dram__bytes_read.sum +
 # dram__bytes_write.sum of one full-batch launch of the gdn_b256 workload, W = 16), or None when not captured.
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {"decode_kernel": 238.4e6, "boundary_kernel": 18.4e6}
 
 
-def algorithmic_bytes_per_head_step(W: int, r: int, diag: bool, group: int, launches_fused: bool) -> float:
+def record_bytes(diag: bool, rec16: int) -> int:
+    """One buffered record (kt, u, decay): fp32 rows, or fp16 rows whose scalar-gate decay stays fp32."""
+    if rec16:
+        return 2 * 384 if diag else 2 * 256 + 4
+    return 4 * (256 + (128 if diag else 1))
+
+
+def algorithmic_bytes_per_head_step(W: int, r: int, diag: bool, group: int, launches_fused: bool, rec16: int = 0) -> float:
     """Bytes that must move per (head, token): quantized state + average record buffer + inputs + appended
     record + output + the window boundary amortised over W tokens."""
     g = 128 if diag else 1
     state = 128 * 128 + 512 + 512 + 512 * r
-    rec = 4 * (256 + g)
+    rec = record_bytes(diag, rec16)
     buf_read = (W - 1) / 2.0 * rec
     inputs = 512 / group + 256 + 2 + 2 * g
     flush = state + (0 if launches_fused else state + W * rec)      # write back (+ re-read when a second kernel does it)
@@ -70,7 +77,7 @@ def config_dict(wl, world: int, warm_tokens: int) -> dict:
     return {"workload": wl.name, "batch": wl.batch, "heads_v": wl.heads_v, "heads_qk": wl.heads_qk,
             "d_k": wl.d_k, "d_v": wl.d_v, "W": wl.W, "r": wl.r, "n_iter": wl.n_iter,
             "gate": "scalar (GDN)" if wl.gate == synth.GATE_SCALAR else "diagonal (KDA)",
-            "state_dtype": "int8 + fp32 scales + fp16 compensators", "record_buffer_dtype": "f32",
+            "state_dtype": "int8 + fp32 scales + fp16 compensators", "record_buffer_dtype": "f16" if wl.rec16 else "f32",
             "inputs_dtype": "bf16", "warmup_tokens": warm_tokens, "window_offsets": "uniform over [0,W)",
             "l2": "working set %.0f MB per step exceeds the 126 MB L2; no flush needed" %
                   (heads * (state_bytes(wl.r) + wl.W * (1028 if wl.gate == synth.GATE_SCALAR else 1536)) / 1e6),
@@ -229,7 +236,8 @@ def to_dev(tok, torch):
 def prepare_state(wl, lq, torch, log, WARM_TOKENS=WARM_TOKENS):
     """512 warm-up tokens on the fp32-state kernel, quantized group by group so that at the end group g
     (a contiguous slice of the batch) holds g buffered records: window offsets uniform over [0, W)."""
-    sh = lq.Shape(wl.batch, wl.heads_v, wl.heads_qk, wl.d_k, wl.d_v, wl.W, wl.r, wl.n_iter, wl.gate, wl.smooth)
+    sh = lq.Shape(wl.batch, wl.heads_v, wl.heads_qk, wl.d_k, wl.d_v, wl.W, wl.r, wl.n_iter, wl.gate, wl.smooth, wl.delta,
+                  wl.rec16)
     B, W = wl.batch, wl.W
     st = lq.State(sh)
     S = torch.zeros((B, wl.heads_v, wl.d_k, wl.d_v), dtype=torch.float32, device="cuda")
@@ -410,10 +418,9 @@ def run_cuda(args, wl):
     launches = lq.decode_launches(sh)
     peak, peak_src = peaks()
     group = wl.heads_v // wl.heads_qk
-    bytes_hs = algorithmic_bytes_per_head_step(wl.W, wl.r, wl.gate == synth.GATE_DIAG, group, launches == 1)
+    bytes_hs = algorithmic_bytes_per_head_step(wl.W, wl.r, wl.gate == synth.GATE_DIAG, group, launches == 1, wl.rec16)
     achieved = heads * bytes_hs / (ms_per_step / 1e3) / 1e9
-    g = 128 if wl.gate == synth.GATE_DIAG else 1
-    rec = 4 * (256 + g)
+    rec = record_bytes(wl.gate == synth.GATE_DIAG, wl.rec16)
     # what each kernel has to move per launch: the decode kernel everything but the boundary; the boundary
     # kernel, for the 1/W of the heads whose window is full, the window representation in and the head block out
     decode_bytes = heads * (bytes_hs - (2 * state_bytes(wl.r) + wl.W * rec) / wl.W)
@@ -505,6 +512,7 @@ def run_sweep(args):
     windows = [int(x) for x in args.sweep_W.split(",")]
     ranks = [int(x) for x in args.sweep_r.split(",")]
     gates = [g for g in args.sweep_gates.split(",")]
+    rec16s = [int(x) for x in args.sweep_rec16.split(",")]
     warm = max(windows) + 8
     rows = []
     for gate_name in gates:
@@ -544,9 +552,10 @@ def run_sweep(args):
             del S16
             for W in windows:
                 for r in ranks:
-                    wl = base_wl.with_(W=W, r=r)
+                  for rec16 in rec16s:
+                    wl = base_wl.with_(W=W, r=r, rec16=rec16)
                     # same staggering as the headline run, with a short pre-fill (speed does not depend on it)
-                    sh = lq.Shape(B, 32, wl.heads_qk, 128, 128, W, r, wl.n_iter, wl.gate, 1)
+                    sh = lq.Shape(B, 32, wl.heads_qk, 128, 128, W, r, wl.n_iter, wl.gate, 1, 1, rec16)
                     st = lq.State(sh)
                     S = torch.zeros((B, 32, 128, 128), dtype=torch.float32, device="cuda")
                     per = max(B // W, 1)
@@ -573,10 +582,11 @@ def run_sweep(args):
                                                                   ("q", "k", "v", "beta", "alpha")], o, stream), nrep, W)
                     flags = lq.check_device()
                     heads = B * 32
-                    bytes_hs = algorithmic_bytes_per_head_step(W, r, diag, wl.heads_v // wl.heads_qk, False)
-                    foot = st.heads.numel() + st.records.numel() * 4
+                    bytes_hs = algorithmic_bytes_per_head_step(W, r, diag, wl.heads_v // wl.heads_qk, False, rec16)
+                    foot = st.heads.numel() + st.records.numel() * st.records.element_size()
                     state_b = 128 * 128 + 4 * 128 + 4 * 128 + 2 * r * 256
                     row = {"sweep": True, "gate": gate_name, "batch": B, "W": W, "r": r, "n_iter": wl.n_iter,
+                           "records": "f16" if rec16 else "f32",
                            "steps": nrep, "ms_per_step": ms, "tokens_heads_per_s": heads / (ms / 1e3),
                            "state_GBps": heads * state_b / (ms / 1e3) / 1e9,
                            "total_GBps": heads * bytes_hs / (ms / 1e3) / 1e9,
@@ -590,9 +600,9 @@ def run_sweep(args):
                     del st
             cache.clear()
             torch.cuda.empty_cache()
-    log("gate  batch   W   r   us/step   state GB/s  total GB/s  %peak   x fp32   x bf16")
+    log("gate  batch   W   r  rec   us/step   state GB/s  total GB/s  %peak   x fp32   x bf16")
     for x in rows:
-        log(f"{x['gate']:4s} {x['batch']:6d} {x['W']:3d} {x['r']:3d} {1e3 * x['ms_per_step']:9.1f} "
+        log(f"{x['gate']:4s} {x['batch']:6d} {x['W']:3d} {x['r']:3d}  {x['records']} {1e3 * x['ms_per_step']:9.1f} "
             f"{x['state_GBps']:11.0f} {x['total_GBps']:11.0f} {x['pct_hbm_peak_measured']:6.1f} "
             f"{x['speedup_vs_fp32_state']:8.2f} {x['speedup_vs_bf16_state']:8.2f}"
             f"{'  (L2-resident)' if x['l2'].startswith('L2-res') else ''}")
@@ -776,6 +786,9 @@ def main():
     ap.add_argument("--sweep-r", default="4,8")
     ap.add_argument("--sweep-gates", default="gdn,kda")
     ap.add_argument("--sweep-steps", type=int, default=512)
+    ap.add_argument("--sweep-rec16", default="0", help="record buffer: 0 fp32, 1 fp16, or 0,1 for both")
+    ap.add_argument("--rec16", type=int, default=0, choices=[0, 1],
+                    help="1: fp16 record buffer (the paper's storage) instead of the fp32 buffer of the headline")
     args = ap.parse_args()
     if args.sweep:
         run_sweep(args)
@@ -791,6 +804,8 @@ def main():
         wl = wl.with_(name="kda_b%d" % args.batch, gate=synth.GATE_DIAG, heads_qk=wl.heads_v)
     if args.n_iter is not None:
         wl = wl.with_(n_iter=args.n_iter)
+    if args.rec16:
+        wl = wl.with_(rec16=1, name=wl.name + "_rec16")
     if args.impl == "reference":
         run_reference(args, wl)
     else:

@@ -76,6 +76,10 @@ typedef struct {
                 /* 0: b = 0, u = v (the other instances of the paper's Table 4:     */
                 /* linear attention, RetNet, Mamba2 with the scalar gate; GLA,      */
                 /* RWKV6, HGRN2 with the diagonal gate; pass beta = 1 for k~ = k)   */
+  int rec16;    /* 1: the record buffer holds fp16 values, as in the paper's storage      */
+                /* accounting (kt, u and the diagonal gate's alpha are rounded, with       */
+                /* saturation, when a record is appended; the scalar gate's decays stay    */
+                /* fp32; `o` of the appending token uses the unrounded u); 0: fp32 records */
 } lq_shape;
 
 /*
@@ -93,7 +97,7 @@ typedef struct {
  *     + 2*r*d_k                       comp_u     fp16 [r][d_v]    value side (carries the magnitude)
  *   (17408 + 512 r bytes at d_k = d_v = 128: 19456 for r = 4, i.e. 1.19 bytes per state element.)
  *
- * records: one row of lq_record_floats(shape) fp32 values per buffered record, [B,Hv,W] rows:
+ * records: one row of lq_record_floats(shape) values (fp32, or fp16 with shape.rec16) per buffered record, [B,Hv,W] rows:
  *     kt[d_k] | u[d_v]                write key kt = beta*k and correction u = v - S^T(alpha.k)  (Eq. 3)
  *     | alpha[d_k]                    diagonal gate only: the record's decay
  * decays: scalar gate only, fp32 [B,Hv,W]: the decay of each buffered record (ignored for the diagonal gate).
@@ -102,7 +106,7 @@ typedef struct {
  */
 typedef struct {
   uint8_t *heads;
-  float *records;
+  void *records;   /* float rows, or (shape.rec16) fp16 rows of the same element counts */
   float *decays;
   int32_t *win_pos;
 } lq_state;

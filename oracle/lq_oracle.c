@@ -68,6 +68,9 @@ typedef struct {
   int smooth;    /* 1: residual smoothing (Sec. 3.4); 0: c == 1             */
   int delta;     /* 1: delta rule, read vector b = alpha (.) k (DeltaNet, Gated DeltaNet, KDA);
                     0: b = 0, so u = v (linear attention, RetNet, Mamba2, GLA, RWKV6, HGRN2: Table 4) */
+  int rec16;     /* 1: the buffered records are kept in fp16 as in the paper's storage accounting (kt, u and, for the
+                    diagonal gate, alpha are rounded when a record is appended; the scalar gate's decay stays
+                    fp32); 0: fp32 records */
 } lqo_shape;
 
 typedef struct {
@@ -142,6 +145,8 @@ uint16_t lqo_f32_to_f16(float f) {
 }
 
 static float clamp_f16_range(float x) { return fminf(fmaxf(x, -65504.0f), 65504.0f); }
+/* the fp32 value of x after a round trip through saturating fp16 storage */
+static float as_stored_f16(float x) { return lqo_f16_to_f32(lqo_f32_to_f16(clamp_f16_range(x))); }
 
 /* ------------------------------------------------------------------ */
 /* the one place where sums are taken                                  */
@@ -528,10 +533,12 @@ static void head_decode(const lqo_shape *sh, const head_view *hv, int n, const t
   }
 
   /* append the record (alpha, kt, u) */
-  if (sh->gate == LQO_GATE_DIAG) memcpy(hv->ba + (size_t)n * K, t->a, sizeof(float) * K);
+  /* (fp16 records: what is stored is the rounded value, widened again; o above used the unrounded u) */
+  if (sh->gate == LQO_GATE_DIAG)
+    for (int i = 0; i < K; i++) hv->ba[(size_t)n * K + i] = sh->rec16 ? as_stored_f16(t->a[i]) : t->a[i];
   else hv->ba[n] = t->a[0];
-  memcpy(hv->bk + (size_t)n * K, kt, sizeof(float) * K);
-  memcpy(hv->bu + (size_t)n * V, u, sizeof(float) * V);
+  for (int i = 0; i < K; i++) hv->bk[(size_t)n * K + i] = sh->rec16 ? as_stored_f16(kt[i]) : kt[i];
+  for (int j = 0; j < V; j++) hv->bu[(size_t)n * V + j] = sh->rec16 ? as_stored_f16(u[j]) : u[j];
 
   free(kt); free(g); free(gk); free(gq); free(dec); free(col); free(pk); free(pq); free(ck); free(u);
   free(xk); free(xq); free(Xk); free(Xq);
@@ -544,7 +551,8 @@ static void head_decode(const lqo_shape *sh, const head_view *hv, int n, const t
 static int shape_ok(const lqo_shape *sh) {
   return sh && sh->batch >= 0 && sh->heads_v > 0 && sh->heads_qk > 0 && sh->heads_v % sh->heads_qk == 0 &&
          sh->d_k > 0 && sh->d_v > 0 && sh->W > 0 && sh->r >= 0 && sh->n_iter >= 1 &&
-         (sh->gate == LQO_GATE_SCALAR || sh->gate == LQO_GATE_DIAG) && (sh->delta == 0 || sh->delta == 1);
+         (sh->gate == LQO_GATE_SCALAR || sh->gate == LQO_GATE_DIAG) && (sh->delta == 0 || sh->delta == 1) &&
+         (sh->rec16 == 0 || sh->rec16 == 1);
 }
 
 int lqo_threads(void) {

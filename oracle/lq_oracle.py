@@ -37,7 +37,7 @@ def build(force: bool = False) -> None:
 
 class _Shape(C.Structure):
     _fields_ = [(n, C.c_int) for n in
-                ("batch", "heads_v", "heads_qk", "d_k", "d_v", "W", "r", "n_iter", "gate", "smooth", "delta")]
+                ("batch", "heads_v", "heads_qk", "d_k", "d_v", "W", "r", "n_iter", "gate", "smooth", "delta", "rec16")]
 
 
 class _State(C.Structure):
@@ -58,10 +58,11 @@ class Shape:
     gate: int = GATE_SCALAR
     smooth: int = 1
     delta: int = 1
+    rec16: int = 0
 
     def c(self) -> _Shape:
         return _Shape(self.batch, self.heads_v, self.heads_qk, self.d_k, self.d_v, self.W, self.r, self.n_iter,
-                      self.gate, self.smooth, self.delta)
+                      self.gate, self.smooth, self.delta, self.rec16)
 
 
 class State:

@@ -15,7 +15,7 @@ namespace lq {
 // MODE 0: flush (window representation -> dense -> new window representation)
 // MODE 1: quantize dense fp32 states         MODE 2: dequantize to dense fp32 states
 // ---------------------------------------------------------------------------------------------
-template <int GATE, int MODE>
+template <int GATE, int MODE, bool R16>
 __global__ void __launch_bounds__(256, 2) boundary_kernel(const Params p, const int stage_bufs) {
   extern __shared__ float4 lq_smem4[];
   float *smem = reinterpret_cast<float *>(lq_smem4);
@@ -55,7 +55,7 @@ __global__ void __launch_bounds__(256, 2) boundary_kernel(const Params p, const 
       const size_t bh = base + kbit * (size_t)gridDim.x;
       const int b = static_cast<int>(bh / p.heads_v);
       const int n = todo_n[kbit];
-      const BoundarySmem sm(smem, p.W, p.r, DIAG, buf);
+      const BoundarySmem sm(smem, p.W, p.r, DIAG, R16, buf);
       float M[8][8];
       if (MODE == 1) {
         const float *S = p.S + bh * (size_t)(D * D);
@@ -64,14 +64,14 @@ __global__ void __launch_bounds__(256, 2) boundary_kernel(const Params p, const 
       } else {
         // (the barrier that ended the previous head's work also freed both staging buffers for writing)
         if (!staged) {
-          stage_issue<GATE>(p, sm, t, bh, n);
+          stage_issue<GATE, R16>(p, sm, t, bh, n);
           cp_async_commit();
         }
         staged = false;
         if (mask && stage_bufs > 1) {
           const int knext = __ffs(mask) - 1;
-          const BoundarySmem nx(smem, p.W, p.r, DIAG, buf ^ 1);
-          stage_issue<GATE>(p, nx, t, base + knext * (size_t)gridDim.x, todo_n[knext]);
+          const BoundarySmem nx(smem, p.W, p.r, DIAG, R16, buf ^ 1);
+          stage_issue<GATE, R16>(p, nx, t, base + knext * (size_t)gridDim.x, todo_n[knext]);
           cp_async_commit();
           staged = true;
           cp_async_wait_but_one();
@@ -80,7 +80,7 @@ __global__ void __launch_bounds__(256, 2) boundary_kernel(const Params p, const 
         }
         __syncthreads();
         LQ_BTICK(1);
-        reconstruct_tile<GATE>(p, sm, t, bh, n, M);
+        reconstruct_tile<GATE, R16>(p, sm, t, bh, n, M);
       }
       if (MODE == 2) {
         float *S = p.S + bh * (size_t)(D * D);
@@ -189,7 +189,7 @@ static lq_status check_shape(const lq_shape *s) {
   if (!s) return LQ_ERR_NULL;
   if (s->batch < 0 || s->heads_v <= 0 || s->heads_qk <= 0 || s->d_k <= 0 || s->d_v <= 0 || s->W <= 0 || s->r < 0 ||
       s->n_iter < 1 || s->heads_v % s->heads_qk != 0 || (s->gate != LQ_GATE_SCALAR && s->gate != LQ_GATE_DIAG) ||
-      (s->delta != 0 && s->delta != 1))
+      (s->delta != 0 && s->delta != 1) || (s->rec16 != 0 && s->rec16 != 1))
     return LQ_ERR_SHAPE;
   if (s->d_k != D || s->d_v != D || s->W > MAX_W || s->r > MAX_R) return LQ_ERR_UNSUPPORTED;
   return LQ_OK;
@@ -227,7 +227,7 @@ static lq_status check_state(const lq_shape *s, const lq_state *st, bool need_bu
 static Params make_params(const lq_shape *s, const lq_state *st) {
   Params p{};
   p.batch = s->batch; p.heads_v = s->heads_v; p.heads_qk = s->heads_qk; p.W = s->W; p.r = s->r;
-  p.n_iter = s->n_iter; p.smooth = s->smooth; p.delta = s->delta; p.force = 0;
+  p.n_iter = s->n_iter; p.smooth = s->smooth; p.delta = s->delta; p.rec16 = s->rec16; p.force = 0;
   if (st) {
     p.heads = st->heads; p.records = st->records; p.decays = st->decays; p.win_pos = st->win_pos;
   }
@@ -335,13 +335,17 @@ static lq_status launch_boundary_kernel(K kernel, int grid, size_t smem, cudaStr
 template <int MODE>
 static lq_status launch_boundary(const lq_shape *s, const Params &p, cudaStream_t stream) {
   const bool diag = s->gate == LQ_GATE_DIAG;
-  const int bufs = MODE == 1 ? 1 : BoundarySmem::buffers(s->W, s->r, diag);
-  const size_t smem = BoundarySmem::bytes(s->W, s->r, diag, bufs);
+  const bool r16 = MODE != 1 && s->rec16 != 0;               // quantizing a dense state reads no records
+  const int bufs = MODE == 1 ? 1 : BoundarySmem::buffers(s->W, s->r, diag, r16);
+  const size_t smem = BoundarySmem::bytes(s->W, s->r, diag, r16, bufs);
   const long nh = (long)s->batch * s->heads_v;
   // persistent: the CTAs that are resident at once (two per SM), each striding over the heads
   const int grid = static_cast<int>(nh < 2L * sm_count() ? nh : 2L * sm_count());
-  return diag ? launch_boundary_kernel(boundary_kernel<LQ_GATE_DIAG, MODE>, grid, smem, stream, p, bufs)
-              : launch_boundary_kernel(boundary_kernel<LQ_GATE_SCALAR, MODE>, grid, smem, stream, p, bufs);
+  if (r16)
+    return diag ? launch_boundary_kernel(boundary_kernel<LQ_GATE_DIAG, MODE == 1 ? 0 : MODE, true>, grid, smem, stream, p, bufs)
+                : launch_boundary_kernel(boundary_kernel<LQ_GATE_SCALAR, MODE == 1 ? 0 : MODE, true>, grid, smem, stream, p, bufs);
+  return diag ? launch_boundary_kernel(boundary_kernel<LQ_GATE_DIAG, MODE, false>, grid, smem, stream, p, bufs)
+              : launch_boundary_kernel(boundary_kernel<LQ_GATE_SCALAR, MODE, false>, grid, smem, stream, p, bufs);
 }
 
 }  // namespace lq
@@ -364,10 +368,15 @@ static lq_status decode_step_impl(const lq_shape *shape, const lq_state *state, 
   const bool diag = shape->gate == LQ_GATE_DIAG;
   const long nh = (long)shape->batch * shape->heads_v;
   // persistent two-warp CTAs, each with its own shared-memory slot: as many as are resident at once
-  const size_t smem = DecodeSlot(shape->W, shape->r, diag).bytes;
+  const bool r16 = shape->rec16 != 0;
+  const size_t smem = DecodeSlot(shape->W, shape->r, diag, r16).bytes;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-  rc = diag ? launch_persistent(decode_kernel<LQ_GATE_DIAG>, nh, 64, smem, st, p)
-            : launch_persistent(decode_kernel<LQ_GATE_SCALAR>, nh, 64, smem, st, p);
+  if (r16)
+    rc = diag ? launch_persistent(decode_kernel<LQ_GATE_DIAG, true>, nh, 64, smem, st, p)
+              : launch_persistent(decode_kernel<LQ_GATE_SCALAR, true>, nh, 64, smem, st, p);
+  else
+    rc = diag ? launch_persistent(decode_kernel<LQ_GATE_DIAG, false>, nh, 64, smem, st, p)
+              : launch_persistent(decode_kernel<LQ_GATE_SCALAR, false>, nh, 64, smem, st, p);
   if (rc != LQ_OK) return rc;
   if (between && cudaEventRecord(between, st) != cudaSuccess) {
     cudaGetLastError();
@@ -630,7 +639,7 @@ lq_status lq_decode_step_host_pipelined(const lq_shape *shape, const lq_state *s
     sub.batch = static_cast<int>(nb);
     lq_state ss = *state;
     ss.heads += b0 * Hv * head_bytes(shape->r);
-    ss.records += b0 * Hv * shape->W * record_floats(diag);
+    ss.records = static_cast<char *>(ss.records) + b0 * Hv * shape->W * record_floats(diag) * (shape->rec16 ? 2 : 4);
     if (ss.decays) ss.decays += b0 * Hv * shape->W;
     ss.win_pos += b0;
     rc = decode_step_impl(&sub, &ss, q_d + b0 * eqk, k_d + b0 * eqk, v_d + b0 * ev, b_d + b0 * eb, a_d + b0 * ea,
@@ -804,6 +813,6 @@ const char *lq_status_string(lq_status status) {
   return "unknown status";
 }
 
-int lq_version(void) { return 2; }
+int lq_version(void) { return 3; }
 
 }  // extern "C"

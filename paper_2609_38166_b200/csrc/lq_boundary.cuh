@@ -27,27 +27,29 @@ struct BoundarySmem {
   uint16_t *ckh; // [r][128]  compensator keys as stored (fp16 bits)
   uint16_t *cuh; // [r][128]  compensator values as stored
   uint8_t *zt;   // [128][128] codes Z^T, 16-byte chunk q of row v stored at chunk q ^ ((v >> 3) & 7)
+  __half *raw;   // fp16 records only: [W] rows as stored (kt | u | (alpha)), widened into kd, bu by the decay scan
   __host__ __device__ static constexpr int fixed_floats(int r) { return 2 * r * D + 11 * D; }
-  __host__ __device__ static constexpr int stage_floats(int W, int r, bool diag) {
-    return 2 * W * D + (diag ? W * D : MAX_W) + 2 * D + r * D + D * D / 4;
+  __host__ __device__ static constexpr int stage_floats(int W, int r, bool diag, bool rec16) {
+    return 2 * W * D + (diag ? W * D : MAX_W) + 2 * D + r * D + D * D / 4 + (rec16 ? W * record_floats(diag) / 2 : 0);
   }
-  __device__ __forceinline__ BoundarySmem(float *base, int W, int r, bool diag, int buf) {
+  __device__ __forceinline__ BoundarySmem(float *base, int W, int r, bool diag, bool rec16, int buf) {
     ck = base; cu = ck + r * D; vec = cu + r * D; colv = vec + D; part = colv + D; gam = part + 8 * D;
-    kd = base + fixed_floats(r) + buf * stage_floats(W, r, diag);
+    kd = base + fixed_floats(r) + buf * stage_floats(W, r, diag, rec16);
     bu = kd + W * D; ba = bu + W * D; cs = ba + (diag ? W * D : MAX_W); ss = cs + D;
     ckh = reinterpret_cast<uint16_t *>(ss + D); cuh = ckh + r * D;
     zt = reinterpret_cast<uint8_t *>(cuh + r * D);
+    raw = reinterpret_cast<__half *>(zt + D * D);
   }
-  static size_t bytes(int W, int r, bool diag, int bufs) {
-    return sizeof(float) * (size_t)(fixed_floats(r) + bufs * stage_floats(W, r, diag));
+  static size_t bytes(int W, int r, bool diag, bool rec16, int bufs) {
+    return sizeof(float) * (size_t)(fixed_floats(r) + bufs * stage_floats(W, r, diag, rec16));
   }
   // two staging buffers while two CTAs with two buffers each still fit on an SM
-  static int buffers(int W, int r, bool diag) { return bytes(W, r, diag, 2) <= 110 * 1024 ? 2 : 1; }
+  static int buffers(int W, int r, bool diag, bool rec16) { return bytes(W, r, diag, rec16, 2) <= 110 * 1024 ? 2 : 1; }
 };
 
 // Issue the asynchronous copies that bring head bh (its codes, scales, compensators and n records) into the
 // staging buffer of sm.  The caller commits the group and later waits for it.
-template <int GATE>
+template <int GATE, bool R16>
 __device__ __forceinline__ void stage_issue(const Params &p, const BoundarySmem &sm, const Tile &t, size_t bh, int n) {
   constexpr bool DIAG = GATE == LQ_GATE_DIAG;
   constexpr int RF = record_floats(DIAG);
@@ -57,12 +59,17 @@ __device__ __forceinline__ void stage_issue(const Params &p, const BoundarySmem 
     const int v = e >> 3, q = e & 7;
     cp_async16(sm.zt + v * D + 16 * (q ^ ((v >> 3) & 7)), hb + HB_CODES + 16 * e);
   }
-  const float *rec = p.record(bh, 0, DIAG);
-  for (int e = t.tid; e < n * (D / 4); e += 256) {
-    const int j = e / (D / 4), q4 = 4 * (e % (D / 4));
-    cp_async16(sm.kd + j * D + q4, rec + j * RF + REC_KT + q4);
-    cp_async16(sm.bu + j * D + q4, rec + j * RF + REC_U + q4);
-    if (DIAG) cp_async16(sm.ba + j * D + q4, rec + j * RF + REC_A + q4);
+  if (R16) {                                                  // the n rows are one contiguous piece of fp16 values
+    const __half *rec = p.record<__half>(bh, 0, DIAG);
+    for (int e = t.tid; e < n * (RF / 8); e += 256) cp_async16(sm.raw + 8 * e, rec + 8 * e);
+  } else {
+    const float *rec = p.record<float>(bh, 0, DIAG);
+    for (int e = t.tid; e < n * (D / 4); e += 256) {
+      const int j = e / (D / 4), q4 = 4 * (e % (D / 4));
+      cp_async16(sm.kd + j * D + q4, rec + j * RF + REC_KT + q4);
+      cp_async16(sm.bu + j * D + q4, rec + j * RF + REC_U + q4);
+      if (DIAG) cp_async16(sm.ba + j * D + q4, rec + j * RF + REC_A + q4);
+    }
   }
   if (!DIAG && t.tid < n) cp_async4(sm.ba + t.tid, p.decays + bh * (size_t)p.W + t.tid);
   if (t.tid < D / 4) cp_async16(sm.ss + 4 * t.tid, hb + HB_COL_SCALE + 16 * t.tid);
@@ -75,7 +82,7 @@ __device__ __forceinline__ void stage_issue(const Params &p, const BoundarySmem 
 // evaluated per element as  base = c_i*(Z_ij*s_j) with s_j the stored code step; base = fma(kc_hi, uc_hj, base) for h = 0..r-1;
 // x = gamma_i*base; x = fma(kd_ji, u_jj, x) for j = 0..n-1.  No sum crosses threads.
 // Leaves the CTA's shared memory holding the records; ends after its last read of it (no trailing barrier).
-template <int GATE>
+template <int GATE, bool R16>
 __device__ __forceinline__ void reconstruct_tile(const Params &p, const BoundarySmem &sm, const Tile &t, size_t bh,
                                                  int n, float (&M)[8][8]) {
   const int r = p.r;
@@ -86,14 +93,19 @@ __device__ __forceinline__ void reconstruct_tile(const Params &p, const Boundary
   // the other half of the CTA widens the compensators meanwhile
   if (t.tid < D) {
     const int i = t.tid;
+    // record j's write key and decay for channel i (fp16 records are widened here, on the way into kd)
+    auto kt_at = [&](int jj) { return R16 ? __half2float(sm.raw[jj * RF + REC_KT + i]) : sm.kd[jj * D + i]; };
+    auto a_at = [&](int jj) {
+      return !DIAG ? sm.ba[jj] : R16 ? __half2float(sm.raw[jj * RF + REC_A + i]) : sm.ba[jj * D + i];
+    };
     float g = 1.0f;
     int j = n - 1;
     for (; j >= 3; j -= 4) {                                  // four records per trip: the loads go out together
       float kt[4], a[4];
 #pragma unroll
       for (int e = 0; e < 4; e++) {
-        kt[e] = sm.kd[(j - e) * D + i];
-        a[e] = GATE == LQ_GATE_DIAG ? sm.ba[(j - e) * D + i] : sm.ba[j - e];
+        kt[e] = kt_at(j - e);
+        a[e] = a_at(j - e);
       }
 #pragma unroll
       for (int e = 0; e < 4; e++) {
@@ -102,12 +114,14 @@ __device__ __forceinline__ void reconstruct_tile(const Params &p, const Boundary
       }
     }
     for (; j >= 0; j--) {
-      sm.kd[j * D + i] = g * sm.kd[j * D + i];
-      g = g * (GATE == LQ_GATE_DIAG ? sm.ba[j * D + i] : sm.ba[j]);
+      sm.kd[j * D + i] = g * kt_at(j);
+      g = g * a_at(j);
     }
     sm.gam[i] = g;
   } else {
     for (int e = t.tid - D; e < 2 * r * D; e += 256 - D) sm.ck[e] = f16_bits(sm.ckh[e]);   // ck and cu are adjacent
+    if (R16)                                                  // fp16 records: the u rows, widened
+      for (int e = t.tid - D; e < n * D; e += 256 - D) sm.bu[e] = __half2float(sm.raw[(e / D) * RF + REC_U + (e % D)]);
   }
   __syncthreads();
   LQ_BTICK(2);

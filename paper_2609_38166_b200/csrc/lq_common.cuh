@@ -35,9 +35,9 @@ constexpr int REC_KT = 0, REC_U = D, REC_A = 2 * D;
 
 // Launch-time description of one call, passed to the kernels by value.
 struct Params {
-  int batch, heads_v, heads_qk, W, r, n_iter, smooth, delta, force;
+  int batch, heads_v, heads_qk, W, r, n_iter, smooth, delta, rec16, force;
   uint8_t *heads;    // [B*Hv] head blocks of head_bytes(r)
-  float *records;    // [B*Hv][W] record rows of record_floats(gate)
+  void *records;     // [B*Hv][W] record rows of record_floats(gate) elements, fp32 or (rec16) fp16
   float *decays;     // scalar gate: [B*Hv][W]
   int32_t *win_pos;
   const uint16_t *q, *k, *v, *beta, *alpha;
@@ -51,9 +51,10 @@ struct Params {
   __device__ __forceinline__ float *row_smooth(size_t bh) const { return reinterpret_cast<float *>(head(bh) + HB_ROW_SMOOTH); }
   __device__ __forceinline__ uint16_t *comp_k(size_t bh) const { return reinterpret_cast<uint16_t *>(head(bh) + HB_COMP_K); }
   __device__ __forceinline__ uint16_t *comp_u(size_t bh) const { return reinterpret_cast<uint16_t *>(head(bh) + hb_comp_u(r)); }
-  // row of record j of head bh; `diag` selects the row length
-  __device__ __forceinline__ float *record(size_t bh, int j, bool diag) const {
-    return records + (bh * W + j) * (size_t)record_floats(diag);
+  // row of record j of head bh; `diag` selects the row length, T the element type (float, or __half with rec16)
+  template <typename T>
+  __device__ __forceinline__ T *record(size_t bh, int j, bool diag) const {
+    return static_cast<T *>(records) + (bh * W + j) * (size_t)record_floats(diag);
   }
 };
 
@@ -178,6 +179,45 @@ __device__ __forceinline__ void load8(const float *src, float (&x)[8]) {
 __device__ __forceinline__ void store8(float *dst, const float (&x)[8]) {
   *reinterpret_cast<float4 *>(dst) = make_float4(x[0], x[1], x[2], x[3]);
   *reinterpret_cast<float4 *>(dst + 4) = make_float4(x[4], x[5], x[6], x[7]);
+}
+
+// ---- record rows kept in fp16: the same accessors on __half rows (widening is exact; narrowing saturates to
+// the finite range and rounds to nearest even, like the compensators) ----
+__device__ __forceinline__ void load8p(const __half *src, float2 (&x)[4]) {
+  const uint4 raw = *reinterpret_cast<const uint4 *>(src);
+  const __half2 *h = reinterpret_cast<const __half2 *>(&raw);
+#pragma unroll
+  for (int i = 0; i < 4; i++) x[i] = __half22float2(h[i]);
+}
+__device__ __forceinline__ void load8(const __half *src, float (&x)[8]) {
+  float2 v[4];
+  load8p(src, v);
+#pragma unroll
+  for (int i = 0; i < 4; i++) { x[2 * i] = v[i].x; x[2 * i + 1] = v[i].y; }
+}
+__device__ __forceinline__ float4 load4(const float *src) { return *reinterpret_cast<const float4 *>(src); }
+__device__ __forceinline__ float4 load4(const __half *src) {
+  const uint2 raw = *reinterpret_cast<const uint2 *>(src);
+  const float2 a = __half22float2(*reinterpret_cast<const __half2 *>(&raw.x));
+  const float2 b = __half22float2(*reinterpret_cast<const __half2 *>(&raw.y));
+  return make_float4(a.x, a.y, b.x, b.y);
+}
+__device__ __forceinline__ uint32_t pack2_f16_sat(float a, float b) {
+  return (uint32_t)to_f16_bits_sat(a) | ((uint32_t)to_f16_bits_sat(b) << 16);
+}
+__device__ __forceinline__ void store8p(__half *dst, const float2 (&x)[4]) {
+  *reinterpret_cast<uint4 *>(dst) = make_uint4(pack2_f16_sat(x[0].x, x[0].y), pack2_f16_sat(x[1].x, x[1].y),
+                                               pack2_f16_sat(x[2].x, x[2].y), pack2_f16_sat(x[3].x, x[3].y));
+}
+__device__ __forceinline__ void store8(__half *dst, const float (&x)[8]) {
+  *reinterpret_cast<uint4 *>(dst) = make_uint4(pack2_f16_sat(x[0], x[1]), pack2_f16_sat(x[2], x[3]),
+                                               pack2_f16_sat(x[4], x[5]), pack2_f16_sat(x[6], x[7]));
+}
+__device__ __forceinline__ void store4(float *dst, float a, float b, float c, float d) {
+  *reinterpret_cast<float4 *>(dst) = make_float4(a, b, c, d);
+}
+__device__ __forceinline__ void store4(__half *dst, float a, float b, float c, float d) {
+  *reinterpret_cast<uint2 *>(dst) = make_uint2(pack2_f16_sat(a, b), pack2_f16_sat(c, d));
 }
 
 // Row sums.  In: p[a] = this thread's block result for row 8ty+a (block index tx).

@@ -27,6 +27,8 @@
 // index is then contiguous, as the MMA operand layout needs.  The small dot products against records and
 // compensators run on the fp32 pipes in the library's fixed summation order.
 #pragma once
+#include <type_traits>
+
 #include "lq_common.cuh"
 
 namespace lq {
@@ -38,11 +40,11 @@ __device__ int g_device_error = 0;
 struct DecodeSlot {
   // byte offsets inside the slot; every region starts on a 16-byte boundary
   int head, rec, bas, digits, y, pk, pq, mbar, bytes;
-  __host__ __device__ DecodeSlot(int W, int r, bool diag) {
+  __host__ __device__ DecodeSlot(int W, int r, bool diag, bool rec16 = false) {
     const int rows = W > 1 ? W - 1 : 1;   // a window holds at most W-1 records when a token arrives
     int o = 0;
     head = o; o += head_bytes(r);          // the head block: codes | col_scale | row_smooth | comp_k | comp_u
-    rec = o; o += 4 * record_floats(diag) * rows;   // buffered record rows
+    rec = o; o += (rec16 ? 2 : 4) * record_floats(diag) * rows;   // buffered record rows (fp32 or fp16)
     bas = o; o += diag ? 0 : 2 * 4 * MAX_W;         // scalar gate: the records' decays, one copy per warp
     digits = o; o += 8 * D;               // digit planes: plane 4v+d = digit d of vector v (0: k, 1: q)
     y = o; o += 2 * 4 * D;                // exact integer sums of the state stream, rounded to fp32: [2][128]
@@ -172,13 +174,14 @@ __device__ __forceinline__ void load_token(const Params &p, const HeadIdx h, int
 }
 
 // Persistent kernel of two-warp CTAs: CTA `blockIdx.x` takes heads blockIdx.x, blockIdx.x + gridDim.x, ...
-template <int GATE>
+template <int GATE, bool R16>
 __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
   extern __shared__ __align__(128) unsigned char slot[];
   constexpr bool DIAG = GATE == LQ_GATE_DIAG;
   constexpr int RF = record_floats(DIAG);
   const int W = p.W, r = p.r;
-  const DecodeSlot L(W, r, DIAG);
+  using rec_t = typename std::conditional<R16, __half, float>::type;   // element type of the record rows
+  const DecodeSlot L(W, r, DIAG, R16);
   const int lane = threadIdx.x & 31, role = threadIdx.x >> 5;      // role 0: stream warp, role 1: dot warp
   const int c = lane & 15, half = lane >> 4, g = lane >> 2, t = lane & 3;
   const int8_t *zt = reinterpret_cast<const int8_t *>(slot + L.head + HB_CODES);
@@ -186,7 +189,7 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
   const float *cs = reinterpret_cast<const float *>(slot + L.head + HB_ROW_SMOOTH);
   const uint16_t *ckh = reinterpret_cast<const uint16_t *>(slot + L.head + HB_COMP_K);
   const uint16_t *cuh = reinterpret_cast<const uint16_t *>(slot + L.head + hb_comp_u(r));
-  const float *rec = reinterpret_cast<const float *>(slot + L.rec);     // rows of RF floats: kt | u | (alpha)
+  const rec_t *rec = reinterpret_cast<const rec_t *>(slot + L.rec);     // rows of RF elements: kt | u | (alpha)
   float *bas = reinterpret_cast<float *>(slot + L.bas) + role * MAX_W;   // this warp's copy of the decays
   int8_t *digits = reinterpret_cast<int8_t *>(slot + L.digits);
   float *y = reinterpret_cast<float *>(slot + L.y), *pk = reinterpret_cast<float *>(slot + L.pk);
@@ -221,9 +224,9 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
   };
   auto request_records = [&](unsigned bh, int n) {
     if (lane == 0) {
-      const uint32_t rb = 4u * RF * n;
+      const uint32_t rb = static_cast<uint32_t>(sizeof(rec_t)) * RF * n;
       mbar_expect_tx(barR, rb);              // with no records the phase completes at once
-      if (n > 0) bulk_g2s(slot_a + L.rec, p.record(bh, 0, DIAG), rb, barR);
+      if (n > 0) bulk_g2s(slot_a + L.rec, p.record<rec_t>(bh, 0, DIAG), rb, barR);
     }
   };
   // Bounded wait for one of the two.  A copy that never lands must not hang the GPU: when the limit runs out the
@@ -442,7 +445,7 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
             const int u = i4 >> 1;
             const bool mine = (i4 & 1) == half;
             const float pkj = mine ? s4[2 * u] : oth[2 * u], pqj = mine ? s4[2 * u + 1] : oth[2 * u + 1];
-            const float4 u4 = *reinterpret_cast<const float4 *>(rec + j * RF + REC_U + 4 * lane);
+            const float4 u4 = load4(rec + j * RF + REC_U + 4 * lane);
             rk_rec[0] = fmaf(u4.x, pkj, rk_rec[0]); rq_rec[0] = fmaf(u4.x, pqj, rq_rec[0]);
             rk_rec[1] = fmaf(u4.y, pkj, rk_rec[1]); rq_rec[1] = fmaf(u4.y, pqj, rq_rec[1]);
             rk_rec[2] = fmaf(u4.z, pkj, rk_rec[2]); rq_rec[2] = fmaf(u4.z, pqj, rq_rec[2]);
@@ -461,7 +464,7 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
       LQ_TICK(5);
       // append the key side of the record (and its decay)
       {
-        float *row = p.record(bh, n, DIAG);
+        rec_t *row = p.record<rec_t>(bh, n, DIAG);
         if (half == 0) {
           store8p(row + REC_KT + 8 * c, kt2);
           if (DIAG) store8(row + REC_A + 8 * c, a8);
@@ -615,7 +618,7 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
         for (int e = 0; e < 4; e++) { u[e] = p.delta ? v4[e] - rk[e] : v4[e]; o[e] = fmaf(u[e], ktq, rq[e]); }
         LQ_TICK(8);
         *reinterpret_cast<float4 *>(p.o + bh * D + 4 * lane) = make_float4(o[0], o[1], o[2], o[3]);
-        *reinterpret_cast<float4 *>(p.record(bh, n, DIAG) + REC_U + 4 * lane) = make_float4(u[0], u[1], u[2], u[3]);
+        store4(p.record<rec_t>(bh, n, DIAG) + REC_U + 4 * lane, u[0], u[1], u[2], u[3]);
       }
       LQ_TICK(9);
     }

@@ -31,7 +31,7 @@ class LqError(RuntimeError):
 
 class _Shape(C.Structure):
     _fields_ = [(n, C.c_int) for n in
-                ("batch", "heads_v", "heads_qk", "d_k", "d_v", "W", "r", "n_iter", "gate", "smooth", "delta")]
+                ("batch", "heads_v", "heads_qk", "d_k", "d_v", "W", "r", "n_iter", "gate", "smooth", "delta", "rec16")]
 
 
 class _State(C.Structure):
@@ -76,10 +76,11 @@ class Shape:
     gate: int = GATE_SCALAR
     smooth: int = 1
     delta: int = 1
+    rec16: int = 0
 
     def c(self) -> _Shape:
         return _Shape(self.batch, self.heads_v, self.heads_qk, self.d_k, self.d_v, self.W, self.r, self.n_iter,
-                      self.gate, self.smooth, self.delta)
+                      self.gate, self.smooth, self.delta, self.rec16)
 
 
 def head_bytes(sh: Shape) -> int:
@@ -104,7 +105,7 @@ class State:
         hb, rf = head_bytes(sh), record_floats(sh)
         assert hb > 0 and rf > 0, "shape not supported by the library"
         self.heads = torch.zeros((B, H, hb), dtype=torch.uint8, device=device)
-        self.records = torch.zeros((B, H, W, rf), dtype=torch.float32, device=device)
+        self.records = torch.zeros((B, H, W, rf), dtype=torch.float16 if sh.rec16 else torch.float32, device=device)
         self.decays = torch.zeros((B, H, W), dtype=torch.float32, device=device)
         self.win_pos = torch.zeros((B,), dtype=torch.int32, device=device)
         o = 0
@@ -150,7 +151,7 @@ def _ptr(t: Optional[torch.Tensor], b0: int = 0) -> C.c_void_p:
 
 def _sub(sh: Shape, b0: int, nb: Optional[int]) -> Shape:
     nb = sh.batch - b0 if nb is None else nb
-    return Shape(nb, sh.heads_v, sh.heads_qk, sh.d_k, sh.d_v, sh.W, sh.r, sh.n_iter, sh.gate, sh.smooth, sh.delta)
+    return Shape(nb, sh.heads_v, sh.heads_qk, sh.d_k, sh.d_v, sh.W, sh.r, sh.n_iter, sh.gate, sh.smooth, sh.delta, sh.rec16)
 
 
 def decode_step(sh: Shape, st: State, q, k, v, beta, alpha, o, stream=None, b0: int = 0, nb: Optional[int] = None):

@@ -47,6 +47,7 @@ class Workload:
     gate: int = GATE_SCALAR
     smooth: int = 1
     delta: int = 1                  # 1: delta rule (GDN, KDA); 0: no read-back, u = v (Mamba2, GLA, ...)
+    rec16: int = 0                  # 1: fp16 record buffer (the paper's storage), 0: fp32
     v_dist: str = "normal"          # "normal" | "student3"
     outlier_frac: float = 0.0
     outlier_mag: float = 1.0

@@ -8,7 +8,7 @@ from paper_2609_38166_b200 import lq, synth
 
 def shapes(wl):
     """(oracle shape, library shape) of a workload."""
-    args = (wl.batch, wl.heads_v, wl.heads_qk, wl.d_k, wl.d_v, wl.W, wl.r, wl.n_iter, wl.gate, wl.smooth, wl.delta)
+    args = (wl.batch, wl.heads_v, wl.heads_qk, wl.d_k, wl.d_v, wl.W, wl.r, wl.n_iter, wl.gate, wl.smooth, wl.delta, wl.rec16)
     return OShape(*args), lq.Shape(*args)
 
 
@@ -26,6 +26,11 @@ def host(t: torch.Tensor) -> np.ndarray:
     if a.dtype == torch.int16:
         return a.numpy().view(np.uint16)
     return a.numpy()
+
+
+def host_f32(t: torch.Tensor) -> np.ndarray:
+    """values as fp32 (record buffers may be fp16 tensors)"""
+    return t.detach().float().cpu().contiguous().numpy()
 
 
 def tok_dev(tok: dict) -> dict:
@@ -61,8 +66,8 @@ def assert_state_parity(st: "lq.State", ost: OState, r: int, what: str = "", exa
     frac, worst = code_mismatch(gpu_codes(st), ost.codes)
     assert worst <= 1 and frac <= 1e-4, (what, frac, worst)
     pairs = [("col_scale", host(st.col_scale), ost.col_scale), ("row_smooth", host(st.row_smooth), ost.row_smooth),
-             ("buf_k", host(st.buf_k), ost.buf_k), ("buf_u", host(st.buf_u), ost.buf_u),
-             ("buf_a", host(st.buf_a), ost.buf_a)]
+             ("buf_k", host_f32(st.buf_k), ost.buf_k), ("buf_u", host_f32(st.buf_u), ost.buf_u),
+             ("buf_a", host_f32(st.buf_a), ost.buf_a)]
     if r > 0:
         pairs += [("comp_k", host(st.comp_k).view(np.float16).astype(np.float32), ost.comp_k_f32()),
                   ("comp_u", host(st.comp_u).view(np.float16).astype(np.float32), ost.comp_u_f32())]

@@ -144,6 +144,22 @@ def test_chain_without_the_delta_rule(oracle, gate):
     assert np.array_equal(S_d.cpu().numpy(), S_o)
 
 
+@pytest.mark.parametrize("gate", GATES)
+@pytest.mark.parametrize("W,r", [(16, 4), (5, 2), (32, 0)])
+def test_chain_with_fp16_records(oracle, gate, W, r):
+    """The record buffer in fp16 (the paper's storage): append rounds kt, u (and the diagonal gate's alpha) with
+    saturation; decode, boundaries, forced flush and dequantization against the oracle, bit for bit."""
+    wl = synth.Workload("r16", 6, 4, 2, W=W, r=r, gate=gate, seed=480 + W, rec16=1)
+    ost, st = _run_chain(oracle, wl, 2 * W + 3 if W <= 16 else W + 5, init="dense", stagger=True, check_every=4)
+    osh, lsh = gu.shapes(wl)
+    S = torch.empty((wl.batch, wl.heads_v, 128, 128), dtype=torch.float32, device="cuda")
+    lq.dequantize_state(lsh, st, S)
+    assert np.array_equal(S.cpu().numpy(), oracle.dequantize_state(osh, ost))
+    oracle.window_flush(osh, ost, force=True)
+    lq.window_flush(lsh, st, force=True)
+    gu.assert_state_parity(st, ost, wl.r, "forced flush, fp16 records")
+
+
 def test_kda_outlier_chain(oracle):
     wl = synth.config("kda_b128_outlier").with_(batch=3, heads_v=4, heads_qk=4)
     _run_chain(oracle, wl, 40, stagger=True, check_every=5)

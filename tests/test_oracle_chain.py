@@ -10,7 +10,7 @@ from tests import refmath as rm
 
 
 def _shape(wl):
-    return Shape(wl.batch, wl.heads_v, wl.heads_qk, wl.d_k, wl.d_v, wl.W, wl.r, wl.n_iter, wl.gate, wl.smooth, wl.delta)
+    return Shape(wl.batch, wl.heads_v, wl.heads_qk, wl.d_k, wl.d_v, wl.W, wl.r, wl.n_iter, wl.gate, wl.smooth, wl.delta, wl.rec16)
 
 
 def _naive_quant64(S):
@@ -102,3 +102,33 @@ def test_error_ordering_on_a_chain(oracle):
     m = {k: float(np.mean(v)) for k, v in err.items()}
     assert m["full"] < m["window"] < m["step"], m
     assert m["full"] < 2e-3, m
+
+
+@pytest.mark.parametrize("gate", [synth.GATE_SCALAR, synth.GATE_DIAG])
+def test_fp16_record_buffer_holds_rounded_values_and_costs_little(oracle, gate):
+    """rec16: what is appended is the fp16 rounding of (kt, u, diagonal alpha), every later use reads those values;
+    the scalar gate's decay stays fp32.  The buffer must hold fp16-representable numbers only, the output of the
+    appending token must not depend on the rounding of its own record, and the error against the fp32-record
+    chain must stay at the fp16 rounding level (2^-11 relative per record)."""
+    wl = synth.Workload("t", 2, 2, 2, 128, 128, W=8, r=2, gate=gate, seed=77)
+    sh32, sh16 = _shape(wl), _shape(wl.with_(rec16=1))
+    S = synth.dense_states(wl, 5)
+    a, b = State(sh32), State(sh16)
+    oracle.quantize_state(sh32, S, a)
+    oracle.quantize_state(sh16, S, b)
+    for t in range(7):
+        tok = synth.token_inputs(wl, t)
+        o32 = oracle.decode_step(sh32, a, **tok)
+        o16 = oracle.decode_step(sh16, b, **tok)
+        if t == 0:
+            assert np.array_equal(o32, o16)                   # nothing rounded has been read yet
+        else:
+            assert np.allclose(o16, o32, rtol=0, atol=4e-3 * np.abs(o32).max())
+    n = int(b.win_pos[0])
+    assert n == 7
+    for arr in (b.buf_k[:, :, :n], b.buf_u[:, :, :n]) + ((b.buf_a[:, :, :n],) if gate == synth.GATE_DIAG else ()):
+        assert np.array_equal(arr, arr.astype(np.float16).astype(np.float32))
+    assert not np.array_equal(a.buf_u[:, :, :n], b.buf_u[:, :, :n])
+    assert np.allclose(b.buf_k[:, :, 0], a.buf_k[:, :, 0], rtol=2.0 ** -11, atol=1e-7)   # first record: same kt, rounded
+    if gate == synth.GATE_SCALAR:
+        assert np.array_equal(a.buf_a, b.buf_a)                # bf16 inputs widened: stored as they are
