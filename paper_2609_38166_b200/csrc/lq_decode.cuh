@@ -7,17 +7,20 @@
 //
 // Data movement: a head's block (16 KiB of codes, the two scale vectors, the compensators: 19 KiB) and
 // its n buffered record rows are each contiguous in memory and are brought into the CTA's shared-memory slot
-// by TWO TMA bulk copies that complete on an mbarrier: a few large bulk requests keep the memory system busy
-// where thousands of 16-byte loads could not (plain loads are limited per warp), and about 64 KB in flight
-// per SM saturate HBM.  The slot is small enough for six CTAs per SM.  CTAs are persistent and walk over
-// the heads with a grid stride.  No load sits on a head's critical path (with the memory system kept full a
-// load takes microseconds to return): the token's vectors are loaded into registers one head ahead, the
-// per-head scalars (window position, beta, scalar alpha) for 32 heads at a time, one per lane.
+// by TWO TMA bulk copies, each completing on its own mbarrier: a few large bulk requests keep the memory
+// system busy where thousands of 16-byte loads could not (plain loads are limited per warp), and about 64 KB
+// in flight per SM saturate HBM.  The slot is small enough for six CTAs per SM.  CTAs are persistent and walk
+// over the heads with a grid stride.  No load sits on a head's critical path (with the memory system kept
+// full a load takes microseconds to return): the token's vectors are loaded into registers one head ahead,
+// the per-head scalars (window position, beta, scalar alpha) for 32 heads at a time, one per lane; whatever
+// needs only the token (the scalar-gate decay chain, kt^T q) is computed before the wait for the slot.
 //
-// Roles: the STREAM warp turns C Gamma x into fixed-point digits, runs the tensor-core pass over the codes
-// and finishes u and o; the DOT warp meanwhile takes the projections onto the buffered records and the
-// compensators, appends the new record and, once the stream warp is done with the slot, requests the next
-// head.  They meet at two named barriers per head.
+// Roles: the STREAM warp turns C Gamma x into fixed-point digits, runs the tensor-core pass over the codes,
+// adds the compensator terms, requests the next head's block as soon as nobody needs this one's any more,
+// adds the record terms and finishes u and o; the DOT warp meanwhile projects onto the compensators, walks
+// the buffered records (projections and the records' terms of the readout in one pass), requests the next
+// head's records, appends the new record and makes the window-position arrival.  They meet at named barriers
+// (three per head, four with the diagonal gate, whose decays both warps read from the records).
 //
 // Arithmetic: the first term is a dense int8 contraction, Z^T [128 x 128] against the two vectors.  The
 // vectors are put on a 30-bit block fixed-point grid and split into four signed base-256 digits each, which
@@ -33,7 +36,7 @@
 
 namespace lq {
 
-// Set when a bounded wait gave up (bit 0: a decode warp's wait for its bulk copies).  Never cleared by kernels.
+// Set when a bounded wait gave up (bit 0: a decode warp's wait for one of its bulk copies).  Never cleared by kernels.
 __device__ int g_device_error = 0;
 
 // ---- shared-memory slot of one CTA ----
@@ -47,9 +50,9 @@ struct DecodeSlot {
     rec = o; o += (rec16 ? 2 : 4) * record_floats(diag) * rows;   // buffered record rows (fp32 or fp16)
     bas = o; o += diag ? 0 : 2 * 4 * MAX_W;         // scalar gate: the records' decays, one copy per warp
     digits = o; o += 8 * D;               // digit planes: plane 4v+d = digit d of vector v (0: k, 1: q)
-    y = o; o += 2 * 4 * D;                // exact integer sums of the state stream, rounded to fp32: [2][128]
-    pk = o; o += (4 * (W + r + 1) + 15) / 16 * 16;
-    pq = o; o += (4 * (W + r + 1) + 15) / 16 * 16;   // projections; pq[n+r] holds kt^T q
+    y = o; o += 2 * 4 * D;                // [2][128]: the rounded sums of the state stream, later the record terms
+    pk = o; o += (4 * (r + 2) + 15) / 16 * 16;      // compensator projections against Gamma k
+    pq = o; o += (4 * (r + 2) + 15) / 16 * 16;      // ... against Gamma q; pq[r], pq[r+1] hold kt^T q of alternate heads
     mbar = o; o += 16;
     bytes = (o + 127) / 128 * 128;
   }
