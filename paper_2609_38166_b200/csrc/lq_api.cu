@@ -263,8 +263,8 @@ static lq_status launch(K kernel, int grid, int block, size_t smem, cudaStream_t
 // launch): its CTAs become resident as SM resources free up and sit in griddepcontrol.wait until that kernel
 // has completed and its writes are visible.  Only for kernels that execute griddepcontrol.wait before their
 // first access to global memory.
-template <typename K, typename P>
-static lq_status launch_dependent(K kernel, int grid, int block, size_t smem, cudaStream_t stream, const P &p) {
+template <typename K, typename... Args>
+static lq_status launch_dependent(K kernel, int grid, int block, size_t smem, cudaStream_t stream, const Args &...args) {
   if (grid <= 0) return LQ_OK;
   if (smem > 48 * 1024 &&
       cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess) {
@@ -281,7 +281,7 @@ static lq_status launch_dependent(K kernel, int grid, int block, size_t smem, cu
   cfg.stream = stream;
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
-  if (cudaLaunchKernelEx(&cfg, kernel, p) != cudaSuccess) {
+  if (cudaLaunchKernelEx(&cfg, kernel, args...) != cudaSuccess) {
     cudaGetLastError();
     return LQ_ERR_CUDA;
   }
@@ -306,32 +306,6 @@ static lq_status launch_persistent(K kernel, long items, int block, size_t smem,
   return launch_dependent(kernel, static_cast<int>(items < resident ? items : resident), block, smem, stream, p);
 }
 
-// launch with one extra kernel argument (programmatic dependent, like launch_dependent)
-template <typename K>
-static lq_status launch_boundary_kernel(K kernel, int grid, size_t smem, cudaStream_t stream, const Params &p, int bufs) {
-  if (grid <= 0) return LQ_OK;
-  if (smem > 48 * 1024 &&
-      cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess) {
-    cudaGetLastError();
-    return LQ_ERR_CUDA;
-  }
-  cudaLaunchAttribute attr;
-  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr.val.programmaticStreamSerializationAllowed = 1;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(grid);
-  cfg.blockDim = dim3(256);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = stream;
-  cfg.attrs = &attr;
-  cfg.numAttrs = 1;
-  if (cudaLaunchKernelEx(&cfg, kernel, p, bufs) != cudaSuccess) {
-    cudaGetLastError();
-    return LQ_ERR_CUDA;
-  }
-  return LQ_OK;
-}
-
 template <int MODE>
 static lq_status launch_boundary(const lq_shape *s, const Params &p, cudaStream_t stream) {
   const bool diag = s->gate == LQ_GATE_DIAG;
@@ -342,10 +316,10 @@ static lq_status launch_boundary(const lq_shape *s, const Params &p, cudaStream_
   // persistent: the CTAs that are resident at once (two per SM), each striding over the heads
   const int grid = static_cast<int>(nh < 2L * sm_count() ? nh : 2L * sm_count());
   if (r16)
-    return diag ? launch_boundary_kernel(boundary_kernel<LQ_GATE_DIAG, MODE == 1 ? 0 : MODE, true>, grid, smem, stream, p, bufs)
-                : launch_boundary_kernel(boundary_kernel<LQ_GATE_SCALAR, MODE == 1 ? 0 : MODE, true>, grid, smem, stream, p, bufs);
-  return diag ? launch_boundary_kernel(boundary_kernel<LQ_GATE_DIAG, MODE, false>, grid, smem, stream, p, bufs)
-              : launch_boundary_kernel(boundary_kernel<LQ_GATE_SCALAR, MODE, false>, grid, smem, stream, p, bufs);
+    return diag ? launch_dependent(boundary_kernel<LQ_GATE_DIAG, MODE == 1 ? 0 : MODE, true>, grid, 256, smem, stream, p, bufs)
+                : launch_dependent(boundary_kernel<LQ_GATE_SCALAR, MODE == 1 ? 0 : MODE, true>, grid, 256, smem, stream, p, bufs);
+  return diag ? launch_dependent(boundary_kernel<LQ_GATE_DIAG, MODE, false>, grid, 256, smem, stream, p, bufs)
+              : launch_dependent(boundary_kernel<LQ_GATE_SCALAR, MODE, false>, grid, 256, smem, stream, p, bufs);
 }
 
 }  // namespace lq

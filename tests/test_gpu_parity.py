@@ -160,6 +160,35 @@ def test_chain_with_fp16_records(oracle, gate, W, r):
     gu.assert_state_parity(st, ost, wl.r, "forced flush, fp16 records")
 
 
+@pytest.mark.parametrize("gate", GATES)
+@pytest.mark.parametrize("rec16", [0, 1])
+def test_largest_supported_shape(oracle, gate, rec16):
+    """W = 64 and r = 16 together (the largest shared-memory plans of both kernels), windows nearly full so that
+    the step crosses a boundary with 64 records; without the delta rule for one of the combinations."""
+    wl = synth.Workload("max", 2, 2, 1, W=64, r=16, gate=gate, seed=490 + rec16, rec16=rec16,
+                        delta=0 if (gate == synth.GATE_DIAG and rec16) else 1)
+    osh, lsh = gu.shapes(wl)
+    ost = OState(osh)
+    S0 = synth.dense_states(wl, 3)
+    oracle.quantize_state(osh, S0, ost)
+    rng = np.random.default_rng(5)
+    n0 = 62                                                    # two tokens later the window is full
+    ost.buf_k[:, :, :n0] = (rng.standard_normal(ost.buf_k[:, :, :n0].shape) / 16).astype(np.float16).astype(np.float32)
+    ost.buf_u[:, :, :n0] = (rng.standard_normal(ost.buf_u[:, :, :n0].shape) / 4).astype(np.float16).astype(np.float32)
+    ost.buf_a[:, :, :n0] = rng.uniform(0.9, 1.0, ost.buf_a[:, :, :n0].shape).astype(np.float16).astype(np.float32)
+    ost.win_pos[:] = n0
+    st = gu.state_to_dev(ost, lsh)
+    o = torch.empty((wl.batch, wl.heads_v, 128), dtype=torch.float32, device="cuda")
+    for step in range(4):
+        tok = synth.token_inputs(wl, step)
+        want = oracle.decode_step(osh, ost, **tok)
+        td = gu.tok_dev(tok)
+        lq.decode_step(lsh, st, td["q"], td["k"], td["v"], td["beta"], td["alpha"], o)
+        _close(o.cpu().numpy(), want, f"largest shape, step {step}")
+        gu.assert_state_parity(st, ost, wl.r, f"largest shape, step {step}")
+    assert int(ost.win_pos[0]) == 2 and lq.check_device() == 0
+
+
 def test_kda_outlier_chain(oracle):
     wl = synth.config("kda_b128_outlier").with_(batch=3, heads_v=4, heads_qk=4)
     _run_chain(oracle, wl, 40, stagger=True, check_every=5)
