@@ -19,7 +19,7 @@ def _oracle_sequence(oracle, wl, b, toks, warm, steps):
     groups = (wl.batch + per - 1) // per
     g = min(b // per, groups - 1)                       # sequence b is quantized after warm - g tokens
     one = wl.with_(batch=1)
-    sh = OShape(1, wl.heads_v, wl.heads_qk, wl.d_k, wl.d_v, wl.W, wl.r, wl.n_iter, wl.gate, wl.smooth)
+    sh = OShape(1, wl.heads_v, wl.heads_qk, wl.d_k, wl.d_v, wl.W, wl.r, wl.n_iter, wl.gate, wl.smooth, wl.delta, wl.rec16)
     cut = lambda tok: {k: np.ascontiguousarray(v[b:b + 1]) for k, v in tok.items()}
     S = np.zeros((1, wl.heads_v, wl.d_k, wl.d_v), np.float32)
     st = OState(sh)
@@ -36,10 +36,12 @@ def _oracle_sequence(oracle, wl, b, toks, warm, steps):
     return st, outs
 
 
-@pytest.mark.parametrize("name,W,warm,steps", [("gdn_b256", 16, 24, 20), ("gdn_b256", 8, 12, 10),
-                                               ("kda_b128_outlier", 16, 20, 18)])
-def test_full_batch_against_sampled_oracle_sequences(oracle, name, W, warm, steps):
-    wl = synth.config(name).with_(W=W)
+@pytest.mark.parametrize("name,W,warm,steps,rec16", [("gdn_b256", 16, 24, 20, 0), ("gdn_b256", 8, 12, 10, 0),
+                                                     ("gdn_b256", 32, 40, 34, 0), ("gdn_b256", 16, 24, 20, 1),
+                                                     ("kda_b128_outlier", 16, 20, 18, 0),
+                                                     ("kda_b128_outlier", 16, 20, 18, 1)])
+def test_full_batch_against_sampled_oracle_sequences(oracle, name, W, warm, steps, rec16):
+    wl = synth.config(name).with_(W=W, rec16=rec16)
     toks = [synth.token_inputs(wl, t) for t in range(warm + steps)]
     sh, st, o = bench.prepare_state(wl, lq, torch, lambda m: None, warm)
     sample = sorted({0, 1, wl.batch // W, wl.batch // 2 + 3, wl.batch - wl.batch // W - 1, wl.batch - 1})
@@ -63,7 +65,7 @@ def test_full_batch_against_sampled_oracle_sequences(oracle, name, W, warm, step
         assert int(st.win_pos[b]) == int(ost.win_pos[0])
         for name_, g, w in (("col_scale", st.col_scale, ost.col_scale), ("row_smooth", st.row_smooth, ost.row_smooth),
                             ("buf_u", st.buf_u, ost.buf_u), ("buf_k", st.buf_k, ost.buf_k)):
-            assert np.array_equal(gu.host(g[b]), w[0]), (b, name_)
+            assert np.array_equal(gu.host_f32(g[b]), w[0]), (b, name_)
         assert np.array_equal(gu.host(st.comp_u[b]), ost.comp_u[0]), b
 
 
