@@ -176,16 +176,23 @@ __device__ __forceinline__ void load_token(const Params &p, const HeadIdx h, int
   }
 }
 
-// Persistent kernel of two-warp CTAs: CTA `blockIdx.x` takes heads blockIdx.x, blockIdx.x + gridDim.x, ...
-template <int GATE, bool R16>
-__global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
-  extern __shared__ __align__(128) unsigned char slot[];
+// Counters of the fused step kernel (lq_fused.cuh): decode slots that are through with the heads whose window
+// becomes full, and CTAs that have left; the last CTA to leave clears both.
+__device__ unsigned g_fused_boundary_heads_done = 0, g_fused_exit_ticket = 0;
+
+// The work of one pair of warps (role 0: stream warp, role 1: dot warp) on its shared-memory slot: heads
+// first, first + G, first + 2G, ...  The named barriers it uses are bar0 + 1 .. bar0 + 5.
+// FUSED (the step kernel that also takes the window boundaries): two passes over the heads, first those whose
+// window becomes full with this token, so that their boundaries can start while the rest is decoded; the
+// arrival on win_pos comes after BOTH warps' global writes of the head, because another CTA acts on it.
+template <int GATE, bool R16, bool FUSED>
+__device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot, const int lane, const int role,
+                                            const int bar0, const unsigned first, const unsigned G) {
   constexpr bool DIAG = GATE == LQ_GATE_DIAG;
   constexpr int RF = record_floats(DIAG);
   const int W = p.W, r = p.r;
   using rec_t = typename std::conditional<R16, __half, float>::type;   // element type of the record rows
   const DecodeSlot L(W, r, DIAG, R16);
-  const int lane = threadIdx.x & 31, role = threadIdx.x >> 5;      // role 0: stream warp, role 1: dot warp
   const int c = lane & 15, half = lane >> 4, g = lane >> 2, t = lane & 3;
   const int8_t *zt = reinterpret_cast<const int8_t *>(slot + L.head + HB_CODES);
   const float *bs = reinterpret_cast<const float *>(slot + L.head + HB_COL_SCALE);
@@ -199,11 +206,10 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
   float *pq = reinterpret_cast<float *>(slot + L.pq);
   const uint32_t barA = smem_addr(slot + L.mbar), barR = barA + 8, slot_a = smem_addr(slot);   // head block, records
 
-  if (threadIdx.x == 0) { mbar_init(barA, 1); mbar_init(barR, 1); }
-  __syncthreads();
-  grid_dependency_wait();                    // no global memory is touched above this line
+  if (role == 0 && lane == 0) { mbar_init(barA, 1); mbar_init(barR, 1); }
+  named_wait(bar0 + 1);                      // both warps: the barriers are initialised
   uint32_t parA = 0, parR = 0;
-  const unsigned nh = static_cast<unsigned>(p.batch) * p.heads_v, G = gridDim.x, Hv = p.heads_v;
+  const unsigned nh = static_cast<unsigned>(p.batch) * p.heads_v, Hv = p.heads_v;
   const unsigned G_b = G / Hv, G_hv = G % Hv;       // one grid stride in (sequence, head) steps
   const int group = p.heads_v / p.heads_qk;
 
@@ -257,24 +263,27 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
   // value, which this head did when its scalars were loaded.  The dot warp makes the arrival, at the end of its
   // work: it has slack, the stream warp (the longer of the two) has none to sit out the atomic's round trip.
   // A head whose window is already full (n >= W) gets no token: it is neither requested nor waited for.
-  load_scalars(blockIdx.x);
+  for (int pass = 0; pass < (FUSED ? 2 : 1); pass++) {
+  // which heads this pass takes: all that get a token, or (fused) those at / not at their last free record
+  auto wanted = [&](int n_) { return n_ < W && (!FUSED || (n_ == W - 1) == (pass == 0)); };
+  load_scalars(first);
   TokenRaw nxt;                               // the token of the head about to start
   nxt.ba_lo = nxt.ba_hi = 1.0f;
-  HeadIdx hd{blockIdx.x, blockIdx.x / Hv, blockIdx.x % Hv};      // this head and the next one
+  HeadIdx hd{first, first / Hv, first % Hv};  // this head and the next one
   HeadIdx hd1 = hd;
   hd1.step(G, G_b, G_hv, Hv);
-  if (hd.bh < nh) load_token<GATE>(p, hd, group, lane, role, nxt);
   {
     const int n0 = __shfl_sync(FULL, sc_n, 0) & 0xFFFF;
-    if (blockIdx.x < nh && n0 < W) {
-      if (role == 0) request_head(blockIdx.x);
-      else request_records(blockIdx.x, n0);
+    if (first < nh && wanted(n0)) {
+      load_token<GATE>(p, hd, group, lane, role, nxt);
+      if (role == 0) request_head(first);
+      else request_records(first, n0);
     }
   }
 #ifdef LQ_TIMING
   tick_ = clock64();
 #endif
-  int idx = 0;                               // position of the head in this CTA's list
+  int idx = 0;                               // position of the head in this slot's list
   for (; hd.bh < nh; hd = hd1, hd1.step(G, G_b, G_hv, Hv), idx++) {
     const size_t bh = hd.bh;
     const int n = __shfl_sync(FULL, sc_n, idx & 31) & 0xFFFF;
@@ -284,13 +293,13 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
     const unsigned bh_next = hd1.bh;
     if ((idx & 31) == 31) load_scalars(bh_next);
     const int n_next = bh_next < nh ? (__shfl_sync(FULL, sc_n, (idx + 1) & 31) & 0xFFFF) : W;
-    const bool active = n < W, next_active = n_next < W;
+    const bool active = wanted(n), next_active = wanted(n_next);
     const int b = static_cast<int>(hd.b);
     LQ_TICK(0);
 
     if (!active) {                           // nothing was requested for this head; keep the pipeline going
-      if (bh_next < nh) load_token<GATE>(p, hd1, group, lane, role, nxt);
       if (next_active) {
+        load_token<GATE>(p, hd1, group, lane, role, nxt);
         if (role == 0) request_head(bh_next);
         else request_records(bh_next, n_next);
       }
@@ -311,7 +320,7 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
       bas[lane] = nxt.ba_lo;
       bas[lane + 32] = nxt.ba_hi;
     }
-    if (bh_next < nh) load_token<GATE>(p, hd1, group, lane, role, nxt);       // used one trip from now
+    if (next_active) load_token<GATE>(p, hd1, group, lane, role, nxt);       // used one trip from now
     // scalar gate: Gamma_{1:l}, the chain of decays from the newest record back (Appendix B.2), needs nothing
     // from the slot, so the stream warp takes it before it waits
     float gsc = alpha_s;
@@ -398,7 +407,7 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
         }
       }
       __syncwarp();
-      named_arrive(3);                       // the compensator projections are in pk, pq; this warp is done with the head block
+      named_arrive(bar0 + 3);                       // the compensator projections are in pk, pq; this warp is done with the head block
       LQ_TICK(4);
       if (!DIAG) wait_for(barR, parR);
       float rk_rec[4] = {0.0f, 0.0f, 0.0f, 0.0f}, rq_rec[4] = {0.0f, 0.0f, 0.0f, 0.0f};
@@ -457,13 +466,13 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
         }
       }
       LQ_TICK(3);
-      if (DIAG) named_wait(4);               // diagonal gate: the stream warp read the records' decays too
+      if (DIAG) named_wait(bar0 + 4);               // diagonal gate: the stream warp read the records' decays too
       if (next_active) request_records(bh_next, n_next);
-      named_wait(2);                         // the stream warp has taken its sums out of y
+      named_wait(bar0 + 2);                         // the stream warp has taken its sums out of y
       *reinterpret_cast<float4 *>(y + 4 * lane) = make_float4(rk_rec[0], rk_rec[1], rk_rec[2], rk_rec[3]);
       *reinterpret_cast<float4 *>(y + D + 4 * lane) = make_float4(rq_rec[0], rq_rec[1], rq_rec[2], rq_rec[3]);
       __syncwarp();
-      named_arrive(1);                       // the record terms are in shared memory
+      named_arrive(bar0 + 1);                       // the record terms are in shared memory
       LQ_TICK(5);
       // append the key side of the record (and its decay)
       {
@@ -473,6 +482,10 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
           if (DIAG) store8(row + REC_A + 8 * c, a8);
           else if (lane == 0) p.decays[bh * (size_t)W + n] = a8[0];
         }
+      }
+      if (FUSED) {                           // the stream warp's o and u are out as well
+        named_wait(bar0 + 5);
+        __threadfence();
       }
       if (lane == 0) arrive_and_set(p.win_pos, b, p.heads_v, n + 1);
       LQ_TICK(7);
@@ -492,7 +505,7 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
           for (int e = 0; e < 8; e++) gam[e] = gam[e] * aj[e];
         }
         __syncwarp();
-        named_arrive(4);                     // this warp is done with the records
+        named_arrive(bar0 + 4);                     // this warp is done with the records
       } else {
 #pragma unroll
         for (int e = 0; e < 8; e++) gam[e] = gsc;
@@ -593,8 +606,8 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
         const float v4[4] = {__uint_as_float(v_raw.x << 16), __uint_as_float(v_raw.x & 0xFFFF0000u),
                              __uint_as_float(v_raw.y << 16), __uint_as_float(v_raw.y & 0xFFFF0000u)};
         LQ_TICK(6);
-        named_arrive(2);                     // y has been read: the dot warp may put the record terms there
-        named_wait(3);                       // the compensator projections are complete
+        named_arrive(bar0 + 2);                     // y has been read: the dot warp may put the record terms there
+        named_wait(bar0 + 3);                       // the compensator projections are complete
         LQ_TICK(7);
 #pragma unroll 2
         for (int h = 0; h < r; h++) {
@@ -608,7 +621,7 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
         }
         __syncwarp();                        // nobody reads the head block any more (the dot warp finished with
         if (next_active) request_head(bh_next);   // it before barrier 3): the next head's may land
-        named_wait(1);                       // the record terms are complete
+        named_wait(bar0 + 1);                       // the record terms are complete
         {
           const float4 tk = *reinterpret_cast<const float4 *>(y + 4 * lane);
           const float4 tq = *reinterpret_cast<const float4 *>(y + D + 4 * lane);
@@ -622,14 +635,31 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
         LQ_TICK(8);
         *reinterpret_cast<float4 *>(p.o + bh * D + 4 * lane) = make_float4(o[0], o[1], o[2], o[3]);
         store4(p.record<rec_t>(bh, n, DIAG) + REC_U + 4 * lane, u[0], u[1], u[2], u[3]);
+        if (FUSED) {
+          __threadfence();
+          named_arrive(bar0 + 5);
+        }
       }
       LQ_TICK(9);
     }
   }
+  if (FUSED && pass == 0 && role == 1 && lane == 0) {       // every head of this slot whose window fills has arrived
+    __threadfence();
+    atomicAdd(&g_fused_boundary_heads_done, 1u);
+  }
+  }  // pass
 #ifdef LQ_TIMING
   if (lane == 0)
     for (int i = 0; i < 12; i++) atomicAdd(&g_phase_cycles[16 * role + i], (unsigned long long)acc_[i]);
 #endif
+}
+
+// Persistent kernel of two-warp CTAs: CTA `blockIdx.x` takes heads blockIdx.x, blockIdx.x + gridDim.x, ...
+template <int GATE, bool R16>
+__global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
+  extern __shared__ __align__(128) unsigned char lq_slot[];
+  grid_dependency_wait();                    // no global memory is touched above this line
+  decode_slot<GATE, R16, false>(p, lq_slot, threadIdx.x & 31, threadIdx.x >> 5, 0, blockIdx.x, gridDim.x);
 }
 
 }  // namespace lq
