@@ -3,10 +3,12 @@
 #include <algorithm>
 #include <atomic>
 #include <cstdio>
+#include <cstdlib>
 #include <mutex>
 
 #include "lq_boundary.cuh"
 #include "lq_decode.cuh"
+#include "lq_fused.cuh"
 
 namespace lq {
 
@@ -322,6 +324,51 @@ static lq_status launch_boundary(const lq_shape *s, const Params &p, cudaStream_
               : launch_dependent(boundary_kernel<LQ_GATE_SCALAR, MODE, false>, grid, 256, smem, stream, p, bufs);
 }
 
+// The step as one cooperative kernel (lq_fused.cuh): one decode CTA and one boundary CTA per SM.
+static bool fused_step_wanted(long nh) {
+  // Off unless LQ_FUSED_STEP=1 is set: on B200 the fused kernel is slower than the two kernels (a boundary CTA
+  // alone on an SM is latency-bound and takes 21 us per head where two of them sharing an SM take 12 us each,
+  // and the registers of an SM do not hold two boundary CTAs next to the decode slots).
+  (void)nh;
+  const char *e = getenv("LQ_FUSED_STEP");
+  return e && atoi(e) != 0;
+}
+
+template <int GATE, bool R16>
+static lq_status launch_fused_step_t(const lq_shape *s, const Params &p, cudaStream_t stream) {
+  const bool diag = GATE == LQ_GATE_DIAG;
+  const size_t smem = fused_smem_bytes(s->W, s->r, diag, R16);
+  auto kernel = fused_step_kernel<GATE, R16>;
+  if (smem > 227 * 1024) return LQ_ERR_UNSUPPORTED;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess) {
+    cudaGetLastError();
+    return LQ_ERR_UNSUPPORTED;
+  }
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, 256, smem) != cudaSuccess || per_sm < 2) {
+    cudaGetLastError();
+    return LQ_ERR_UNSUPPORTED;               // two CTAs per SM are the design
+  }
+  const long nh = (long)s->batch * s->heads_v;
+  const int sms = sm_count();
+  if (nh > (long)sms * FUSED_SLOTS * FUSED_NBUF || nh > (long)sms * 2048) return LQ_ERR_UNSUPPORTED;
+  int decode_ctas = sms;
+  Params pp = p;
+  void *args[] = {&pp, &decode_ctas};
+  if (cudaLaunchCooperativeKernel(reinterpret_cast<void *>(kernel), dim3(2 * sms), dim3(256), args, smem, stream) !=
+      cudaSuccess) {
+    cudaGetLastError();
+    return LQ_ERR_CUDA;
+  }
+  return LQ_OK;
+}
+
+static lq_status launch_fused_step(const lq_shape *s, const Params &p, cudaStream_t stream) {
+  const bool diag = s->gate == LQ_GATE_DIAG;
+  if (s->rec16) return diag ? launch_fused_step_t<LQ_GATE_DIAG, true>(s, p, stream) : launch_fused_step_t<LQ_GATE_SCALAR, true>(s, p, stream);
+  return diag ? launch_fused_step_t<LQ_GATE_DIAG, false>(s, p, stream) : launch_fused_step_t<LQ_GATE_SCALAR, false>(s, p, stream);
+}
+
 }  // namespace lq
 
 using namespace lq;
@@ -343,8 +390,12 @@ static lq_status decode_step_impl(const lq_shape *shape, const lq_state *state, 
   const long nh = (long)shape->batch * shape->heads_v;
   // persistent two-warp CTAs, each with its own shared-memory slot: as many as are resident at once
   const bool r16 = shape->rec16 != 0;
-  const size_t smem = DecodeSlot(shape->W, shape->r, diag, r16).bytes;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (!between && fused_step_wanted(nh)) {
+    lq_status frc = launch_fused_step(shape, p, st);
+    if (frc != LQ_ERR_UNSUPPORTED) return frc;       // does not fit this device or shape: the two kernels below
+  }
+  const size_t smem = DecodeSlot(shape->W, shape->r, diag, r16).bytes;
   if (r16)
     rc = diag ? launch_persistent(decode_kernel<LQ_GATE_DIAG, true>, nh, 64, smem, st, p)
               : launch_persistent(decode_kernel<LQ_GATE_SCALAR, true>, nh, 64, smem, st, p);

@@ -302,9 +302,15 @@ __device__ __forceinline__ void row_blocks(const float (&M)[8][8], const float (
 // the value in bits 0..15.  The head that arrives last (all heads_v have read the old value by then)
 // stores the new value and thereby clears the counter.  Call from one thread per head, after a
 // __syncthreads() that follows the head's last global write.
+// FENCED: for readers inside the same kernel, who take the new value as the sign that every head's writes are
+// there (each arriving head fences before the call, the last one again before it stores).
+template <bool FENCED = false>
 __device__ __forceinline__ void arrive_and_set(int32_t *win_pos, int b, int heads_v, int new_value) {
   const int old = atomicAdd(win_pos + b, 0x10000);
-  if ((old >> 16) == heads_v - 1) win_pos[b] = new_value;
+  if ((old >> 16) == heads_v - 1) {
+    if (FENCED) __threadfence();
+    win_pos[b] = new_value;
+  }
 }
 
 }  // namespace lq

@@ -184,10 +184,32 @@ __device__ unsigned g_fused_boundary_heads_done = 0, g_fused_exit_ticket = 0;
 // first, first + G, first + 2G, ...  The named barriers it uses are bar0 + 1 .. bar0 + 5.
 // FUSED (the step kernel that also takes the window boundaries): two passes over the heads, first those whose
 // window becomes full with this token, so that their boundaries can start while the rest is decoded; the
-// arrival on win_pos comes after BOTH warps' global writes of the head, because another CTA acts on it.
+// arrival on win_pos comes after BOTH warps' global writes of the head, because another CTA acts on it;
+// and the window positions of all of the slot's heads are read once, up front, into nbuf (a sequence whose
+// boundary is taken meanwhile goes back to position 0, which must not be mistaken for a fresh window).
+// Before the first pass: the slot's two copy barriers, and (fused) the window positions of all its heads.
 template <int GATE, bool R16, bool FUSED>
+__device__ __forceinline__ void decode_slot_init(const Params &p, unsigned char *slot, const int lane, const int role,
+                                                 const int bar0, const unsigned first, const unsigned G, uint16_t *nbuf) {
+  const DecodeSlot L(p.W, p.r, GATE == LQ_GATE_DIAG, R16);
+  const uint32_t barA = smem_addr(slot + L.mbar), barR = barA + 8;
+  if (role == 0 && lane == 0) { mbar_init(barA, 1); mbar_init(barR, 1); }
+  if (FUSED) {
+    const unsigned nh = static_cast<unsigned>(p.batch) * p.heads_v;
+    for (unsigned k = 32 * role + lane; first + k * G < nh; k += 64)
+      nbuf[k] = static_cast<uint16_t>(p.win_pos[(first + k * G) / p.heads_v] & 0xFFFF);
+  }
+  named_wait(bar0 + 1);                      // both warps: the barriers are initialised, nbuf is complete
+}
+
+// PASS: 0 in the ordinary kernel; in the fused one 0 = the heads whose window fills with this token, 1 = the
+// others (two instances of the code: only the first carries the fences that publish a head to other CTAs, and a
+// fence anywhere in the loop costs every trip).  parA, parR: the phases of the two copy barriers, carried over.
+template <int GATE, bool R16, bool FUSED, int PASS>
 __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot, const int lane, const int role,
-                                            const int bar0, const unsigned first, const unsigned G) {
+                                            const int bar0, const unsigned first, const unsigned G,
+                                            uint16_t *nbuf, uint32_t &parA, uint32_t &parR) {
+  constexpr int pass = PASS;
   constexpr bool DIAG = GATE == LQ_GATE_DIAG;
   constexpr int RF = record_floats(DIAG);
   const int W = p.W, r = p.r;
@@ -206,9 +228,6 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
   float *pq = reinterpret_cast<float *>(slot + L.pq);
   const uint32_t barA = smem_addr(slot + L.mbar), barR = barA + 8, slot_a = smem_addr(slot);   // head block, records
 
-  if (role == 0 && lane == 0) { mbar_init(barA, 1); mbar_init(barR, 1); }
-  named_wait(bar0 + 1);                      // both warps: the barriers are initialised
-  uint32_t parA = 0, parR = 0;
   const unsigned nh = static_cast<unsigned>(p.batch) * p.heads_v, Hv = p.heads_v;
   const unsigned G_b = G / Hv, G_hv = G % Hv;       // one grid stride in (sequence, head) steps
   const int group = p.heads_v / p.heads_qk;
@@ -253,7 +272,8 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
   auto load_scalars = [&](unsigned first_bh) {
     const unsigned bh = first_bh + lane * G;  // (once per 32 heads: a division is fine here)
     if (bh < nh) {
-      sc_n = p.win_pos[bh / Hv];            // bits 16.. are the arrival counter of this launch: masked at use
+      sc_n = FUSED ? nbuf[(first_bh - first) / G + lane]
+                   : p.win_pos[bh / Hv];    // bits 16.. are the arrival counter of this launch: masked at use
       sc_beta = p.beta[bh];
       if (!DIAG) sc_alpha = p.alpha[bh];
     }
@@ -263,7 +283,6 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
   // value, which this head did when its scalars were loaded.  The dot warp makes the arrival, at the end of its
   // work: it has slack, the stream warp (the longer of the two) has none to sit out the atomic's round trip.
   // A head whose window is already full (n >= W) gets no token: it is neither requested nor waited for.
-  for (int pass = 0; pass < (FUSED ? 2 : 1); pass++) {
   // which heads this pass takes: all that get a token, or (fused) those at / not at their last free record
   auto wanted = [&](int n_) { return n_ < W && (!FUSED || (n_ == W - 1) == (pass == 0)); };
   load_scalars(first);
@@ -483,11 +502,11 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
           else if (lane == 0) p.decays[bh * (size_t)W + n] = a8[0];
         }
       }
-      if (FUSED) {                           // the stream warp's o and u are out as well
-        named_wait(bar0 + 5);
+      if (FUSED && pass == 0) {              // a boundary CTA will read this head's record: the stream warp's u is
+        named_wait(bar0 + 5);                // out as well, and both warps' writes are ordered before the arrival
         __threadfence();
       }
-      if (lane == 0) arrive_and_set(p.win_pos, b, p.heads_v, n + 1);
+      if (lane == 0) arrive_and_set<FUSED && PASS == 0>(p.win_pos, b, p.heads_v, n + 1);
       LQ_TICK(7);
     } else {
       // =========================== STREAM WARP ===========================
@@ -635,7 +654,7 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
         LQ_TICK(8);
         *reinterpret_cast<float4 *>(p.o + bh * D + 4 * lane) = make_float4(o[0], o[1], o[2], o[3]);
         store4(p.record<rec_t>(bh, n, DIAG) + REC_U + 4 * lane, u[0], u[1], u[2], u[3]);
-        if (FUSED) {
+        if (FUSED && pass == 0) {
           __threadfence();
           named_arrive(bar0 + 5);
         }
@@ -647,7 +666,6 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
     __threadfence();
     atomicAdd(&g_fused_boundary_heads_done, 1u);
   }
-  }  // pass
 #ifdef LQ_TIMING
   if (lane == 0)
     for (int i = 0; i < 12; i++) atomicAdd(&g_phase_cycles[16 * role + i], (unsigned long long)acc_[i]);
@@ -659,7 +677,10 @@ template <int GATE, bool R16>
 __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
   extern __shared__ __align__(128) unsigned char lq_slot[];
   grid_dependency_wait();                    // no global memory is touched above this line
-  decode_slot<GATE, R16, false>(p, lq_slot, threadIdx.x & 31, threadIdx.x >> 5, 0, blockIdx.x, gridDim.x);
+  const int lane = threadIdx.x & 31, role = threadIdx.x >> 5;
+  uint32_t parA = 0, parR = 0;
+  decode_slot_init<GATE, R16, false>(p, lq_slot, lane, role, 0, blockIdx.x, gridDim.x, nullptr);
+  decode_slot<GATE, R16, false, 0>(p, lq_slot, lane, role, 0, blockIdx.x, gridDim.x, nullptr, parA, parR);
 }
 
 }  // namespace lq

@@ -189,6 +189,16 @@ def test_largest_supported_shape(oracle, gate, rec16):
     assert int(ost.win_pos[0]) == 2 and lq.check_device() == 0
 
 
+@pytest.mark.parametrize("gate", GATES)
+def test_fused_step_kernel_gives_the_same_bits(oracle, gate, monkeypatch):
+    """The step as one cooperative kernel (decode slots and boundary CTAs side by side; off by default because it
+    is slower on this GPU): same chain, same oracle, bit for bit, with boundaries in every call."""
+    monkeypatch.setenv("LQ_FUSED_STEP", "1")
+    wl = synth.Workload("fu", 40, 4, 2, W=4, r=2, gate=gate, seed=495)
+    _run_chain(oracle, wl, 11, init="dense", stagger=True, check_every=2)
+    assert lq.check_device() == 0
+
+
 def test_kda_outlier_chain(oracle):
     wl = synth.config("kda_b128_outlier").with_(batch=3, heads_v=4, heads_qk=4)
     _run_chain(oracle, wl, 40, stagger=True, check_every=5)
