@@ -439,7 +439,7 @@ def run_cuda(args, wl):
                               "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH["decode_kernel"]},
             "boundary_kernel": {"ms": bk, "algorithmic_bytes": boundary_bytes, "achieved": boundary_bytes / bk / 1e6,
                                 "frac": boundary_bytes / bk / 1e6 / peak,
-                                "bound": "fp32 issue/latency (see DESIGN.md 6.2), not hbm",
+                                "bound": "fp32 issue and dependency latency, not hbm",
                                 "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH["boundary_kernel"]},
             "how": "CUDA events on the launching stream around each kernel, mean of %d steps in a second loop" %
                    kern["steps"]}
