@@ -184,8 +184,8 @@ def oracle_sample_state(oracle, wl, seed_tokens: int = 48):
     return sh, st
 
 
-def time_oracle(wl, steps: int, warmup: int, budget_s: float):
-    """Times oracle.decode_step on a sub-batch sized to fit `budget_s`; returns (head-steps/s, cores, sample)."""
+def time_oracle(wl, steps: int, warmup: int, limit_s: float):
+    """Times oracle.decode_step on a sub-batch sized to fit `limit_s`; returns (head-steps/s, cores, sample)."""
     from oracle.lq_oracle import Oracle
     oracle = Oracle()
     probe = wl.with_(batch=2)
@@ -195,7 +195,7 @@ def time_oracle(wl, steps: int, warmup: int, budget_s: float):
     for t in range(4):
         oracle.decode_step(sh, st, **toks[t])
     rate = 4 * probe.batch * probe.heads_v / (time.perf_counter() - t0)          # head-steps per second, rough
-    nb = int(max(1, min(wl.batch, budget_s * rate / ((steps + warmup) * wl.heads_v))))
+    nb = int(max(1, min(wl.batch, limit_s * rate / ((steps + warmup) * wl.heads_v))))
     sub = wl.with_(batch=nb)
     sh, st = oracle_sample_state(oracle, sub)
     toks = [synth.token_inputs(sub, 2000 + t) for t in range(wl.W)]
@@ -214,7 +214,7 @@ def run_reference(args, wl):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    hs, cores, sample, s_per_step = time_oracle(wl, args.steps, args.warmup, budget_s=150.0)
+    hs, cores, sample, s_per_step = time_oracle(wl, args.steps, args.warmup, limit_s=150.0)
     value = hs * state_bytes(wl.r) / 1e9
     line = {"impl": "reference", "metric": metric_name(wl), "value": value, "unit": "GB/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": s_per_step * 1e3, "higher_is_better": True,
@@ -476,7 +476,7 @@ def run_cuda(args, wl):
 
     cpu = None
     if not args.only_timed:
-        hs_cpu, cores, sample, _ = time_oracle(wl.with_(seed=wl.seed), steps=8 * wl.W, warmup=2, budget_s=25.0)
+        hs_cpu, cores, sample, _ = time_oracle(wl.with_(seed=wl.seed), steps=8 * wl.W, warmup=2, limit_s=25.0)
         cpu = {"value": hs_cpu * state_bytes(wl.r) / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
                "sample": sample, "tokens_heads_per_s": hs_cpu}
 

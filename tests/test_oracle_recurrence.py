@@ -202,7 +202,7 @@ def test_without_the_delta_rule_the_state_is_a_decayed_sum_of_outer_products(ora
     """b_t = 0 (Table 4: linear attention, RetNet, Mamba2 with the scalar gate; GLA, RWKV6, HGRN2 with the diagonal
     one): nothing is read back, so S_t = sum_i (prod_{i<j<=t} D_j) k~_i v_i^T in closed form and
     o_t = sum_i <prod D_j k~_i, q_t> v_i.  Checked for the dense reference step and, with a quantized state, for
-    the windowed decode (error within the 8-bit budget) and with the quantizer off (equal up to fp32 rounding)."""
+    the windowed decode (error at the 8-bit level) and with the quantizer off (equal up to fp32 rounding)."""
     wl = synth.Workload("t", 2, 4, 2, 128, 128, W=4, r=2, gate=gate, seed=61, delta=0)
     sh = _shape(wl)
     B, H, T = 2, 4, 11
