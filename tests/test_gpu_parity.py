@@ -199,6 +199,41 @@ def test_fused_step_kernel_gives_the_same_bits(oracle, gate, monkeypatch):
     assert lq.check_device() == 0
 
 
+def test_steps_captured_in_a_cuda_graph_replay_identically():
+    """W steps captured once (the two kernels of a step are programmatic dependents of each other) and replayed
+    must leave the same state and outputs as the same steps issued directly."""
+    wl = synth.Workload("cg", 24, 4, 2, W=4, r=2, seed=497)
+    _, lsh = gu.shapes(wl)
+    S0 = gu.dev(synth.dense_states(wl, 4))
+    toks = [gu.tok_dev(synth.token_inputs(wl, t)) for t in range(4)]
+    outs = {}
+    for mode in ("direct", "graph"):
+        st = lq.State(lsh)
+        lq.quantize_state(lsh, S0, st)
+        o = torch.zeros((4, wl.batch, wl.heads_v, 128), dtype=torch.float32, device="cuda")
+        stream = torch.cuda.Stream()
+        with torch.cuda.stream(stream):
+            def steps():
+                for t in range(4):
+                    d = toks[t]
+                    lq.decode_step(lsh, st, d["q"], d["k"], d["v"], d["beta"], d["alpha"], o[t], stream)
+            if mode == "direct":
+                for _ in range(3):
+                    steps()
+            else:
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=stream):
+                    steps()
+                for _ in range(3):                  # (the capture itself runs nothing)
+                    g.replay()
+        stream.synchronize()
+        outs[mode] = (o.cpu().numpy(), [t.cpu().numpy() for t in st.tensors()])
+    assert np.array_equal(outs["direct"][0], outs["graph"][0])
+    for a, b in zip(outs["direct"][1], outs["graph"][1]):
+        assert np.array_equal(a, b)
+    assert lq.check_device() == 0
+
+
 def test_kda_outlier_chain(oracle):
     wl = synth.config("kda_b128_outlier").with_(batch=3, heads_v=4, heads_qk=4)
     _run_chain(oracle, wl, 40, stagger=True, check_every=5)
