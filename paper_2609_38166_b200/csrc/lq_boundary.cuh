@@ -177,18 +177,31 @@ __device__ __forceinline__ void quantize_tile(const Params &p, const BoundarySme
                                               int n, float (&M)[8][8]) {
   const int r = p.r;
   __syncthreads();
+  // The scales 1 / |u| of all start vectors at once, one per group of sixteen lanes (they depend on the records
+  // only; taken one by one inside the loop each would cost a reduction and a reciprocal square root of latency).
+  // 0 marks "no such record, or a zero one": start from the all-equal vector.  Kept in sm.gam, which is free now.
+  float *start_scale = sm.gam;
+  {
+    // (every thread takes part in the warp-wide reduction, whatever r and n: groups without a record of
+    // their own reduce record 0 and drop the result)
+    const int g16 = t.tid >> 4;                               // r <= 16 = the number of groups
+    const bool mine = g16 < r && g16 < n;
+    const float *u = sm.bu + (mine ? n - 1 - g16 : 0) * D;
+    const float nu0 = dot128_shared(u, u, t.lane & 15);
+    const float s0 = mine && nu0 >= 1e-30f ? 1.0f / sqrtf(nu0) : 0.0f;
+    if (g16 < r && (t.lane & 15) == 0) start_scale[g16] = s0;
+  }
+  __syncthreads();
   int h = 0;
   for (; h < r; h++) {
     float w[8], tn[8];
     const float w0 = 1.0f / sqrtf(static_cast<float>(D));
 #pragma unroll
     for (int b = 0; b < 8; b++) w[b] = w0;
-    if (h < n) {
-      const float *u = sm.bu + (n - 1 - h) * D;
-      const float nu0 = dot128_shared(u, u, t.lane & 15);     // same value in every thread
-      if (nu0 >= 1e-30f) {
-        const float s0 = 1.0f / sqrtf(nu0);
-        load8(u + 8 * t.tx, w);
+    {
+      const float s0 = start_scale[h];
+      if (s0 != 0.0f) {
+        load8(sm.bu + (n - 1 - h) * D + 8 * t.tx, w);
 #pragma unroll
         for (int b = 0; b < 8; b++) w[b] = w[b] * s0;
       }
