@@ -71,6 +71,10 @@ typedef struct {
   int rec16;     /* 1: the buffered records are kept in fp16 as in the paper's storage accounting (kt, u and, for the
                     diagonal gate, alpha are rounded when a record is appended; the scalar gate's decay stays
                     fp32); 0: fp32 records */
+  int state_bf16; /* 1: "per-window BF16" (the -w baseline of Fig. 3 and Table 2): the boundary state is the dense
+                    state rounded to bfloat16 element by element, with no scale, smoothing or compensator;
+                    needs the S0 array of lqo_state, whose entries are then bfloat16 values; 0: the 8-bit
+                    representation (or, with S0 given, no quantization at all) */
 } lqo_shape;
 
 typedef struct {
@@ -441,12 +445,19 @@ static void head_quantize(const lqo_shape *sh, float *M, const head_view *hv, co
   free(w); free(t); free(col); free(kf); free(uf);
 }
 
+/* the boundary state without the 8-bit quantizer: the dense state itself, or (per-window BF16) each element
+ * rounded to the nearest bfloat16, ties to even */
+static void head_store_dense(const lqo_shape *sh, const float *S, const head_view *hv) {
+  size_t KV = (size_t)sh->d_k * sh->d_v;
+  for (size_t e = 0; e < KV; e++) hv->S0[e] = sh->state_bf16 ? bf16_to_f32(lqo_f32_to_bf16(S[e])) : S[e];
+}
+
 /* boundary: rebuild S_W from the window representation and start the next window from it */
 static void head_flush(const lqo_shape *sh, const head_view *hv, int n) {
   int K = sh->d_k, V = sh->d_v;
   float *S = (float *)malloc(sizeof(float) * (size_t)K * V);
   head_reconstruct(sh, hv, n, S);
-  if (hv->S0) memcpy(hv->S0, S, sizeof(float) * (size_t)K * V);
+  if (hv->S0) head_store_dense(sh, S, hv);
   else head_quantize(sh, S, hv, hv->bu, n);
   free(S);
 }
@@ -552,7 +563,11 @@ static int shape_ok(const lqo_shape *sh) {
   return sh && sh->batch >= 0 && sh->heads_v > 0 && sh->heads_qk > 0 && sh->heads_v % sh->heads_qk == 0 &&
          sh->d_k > 0 && sh->d_v > 0 && sh->W > 0 && sh->r >= 0 && sh->n_iter >= 1 &&
          (sh->gate == LQO_GATE_SCALAR || sh->gate == LQO_GATE_DIAG) && (sh->delta == 0 || sh->delta == 1) &&
-         (sh->rec16 == 0 || sh->rec16 == 1);
+         (sh->rec16 == 0 || sh->rec16 == 1) && (sh->state_bf16 == 0 || sh->state_bf16 == 1);
+}
+/* per-window BF16 lives in the S0 array and has no compensators */
+static int state_ok(const lqo_shape *sh, const lqo_state *st) {
+  return !sh->state_bf16 || (st && st->S0 && sh->r == 0);
 }
 
 int lqo_threads(void) {
@@ -603,13 +618,13 @@ int lqo_ref_step_bf16(const lqo_shape *sh, uint16_t *S16, const uint16_t *q, con
 
 /* dense fp32 state -> window representation with an empty window */
 int lqo_quantize_state(const lqo_shape *sh, const float *S, lqo_state *st) {
-  if (!shape_ok(sh)) return 1;
+  if (!shape_ok(sh) || !state_ok(sh, st)) return 1;
   long nh = (long)sh->batch * sh->heads_v;
   size_t KV = (size_t)sh->d_k * sh->d_v;
 #pragma omp parallel for schedule(dynamic, 1)
   for (long bh = 0; bh < nh; bh++) {
     head_view hv = view_of(sh, st, (int)(bh / sh->heads_v), (int)(bh % sh->heads_v));
-    if (hv.S0) { memcpy(hv.S0, S + (size_t)bh * KV, sizeof(float) * KV); continue; }
+    if (hv.S0) { head_store_dense(sh, S + (size_t)bh * KV, &hv); continue; }
     float *M = (float *)malloc(sizeof(float) * KV);
     memcpy(M, S + (size_t)bh * KV, sizeof(float) * KV);
     head_quantize(sh, M, &hv, NULL, 0);
@@ -621,7 +636,7 @@ int lqo_quantize_state(const lqo_shape *sh, const float *S, lqo_state *st) {
 
 /* window representation -> the dense state it stands for right now (all buffered records applied) */
 int lqo_dequantize_state(const lqo_shape *sh, const lqo_state *st, float *S) {
-  if (!shape_ok(sh)) return 1;
+  if (!shape_ok(sh) || !state_ok(sh, st)) return 1;
   long nh = (long)sh->batch * sh->heads_v;
   size_t KV = (size_t)sh->d_k * sh->d_v;
 #pragma omp parallel for schedule(dynamic, 1)
@@ -635,7 +650,7 @@ int lqo_dequantize_state(const lqo_shape *sh, const lqo_state *st, float *S) {
 
 /* Flush sequences whose window is full (force == 0) or that hold any record (force != 0). */
 int lqo_window_flush(const lqo_shape *sh, lqo_state *st, int force) {
-  if (!shape_ok(sh)) return 1;
+  if (!shape_ok(sh) || !state_ok(sh, st)) return 1;
   long nh = (long)sh->batch * sh->heads_v;
 #pragma omp parallel for schedule(dynamic, 1)
   for (long bh = 0; bh < nh; bh++) {
@@ -657,7 +672,7 @@ int lqo_window_flush(const lqo_shape *sh, lqo_state *st, int force) {
  * (Eq. 4: the state is materialised and quantized only at l = p). */
 int lqo_decode_step(const lqo_shape *sh, lqo_state *st, const uint16_t *q, const uint16_t *k, const uint16_t *v,
                     const uint16_t *beta, const uint16_t *alpha, float *o) {
-  if (!shape_ok(sh)) return 1;
+  if (!shape_ok(sh) || !state_ok(sh, st)) return 1;
   for (int b = 0; b < sh->batch; b++)
     if (st->win_pos[b] < 0 || st->win_pos[b] >= sh->W) return 2;
   long nh = (long)sh->batch * sh->heads_v;

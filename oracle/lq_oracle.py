@@ -37,7 +37,7 @@ def build(force: bool = False) -> None:
 
 class _Shape(C.Structure):
     _fields_ = [(n, C.c_int) for n in
-                ("batch", "heads_v", "heads_qk", "d_k", "d_v", "W", "r", "n_iter", "gate", "smooth", "delta", "rec16")]
+                ("batch", "heads_v", "heads_qk", "d_k", "d_v", "W", "r", "n_iter", "gate", "smooth", "delta", "rec16", "state_bf16")]
 
 
 class _State(C.Structure):
@@ -59,10 +59,11 @@ class Shape:
     smooth: int = 1
     delta: int = 1
     rec16: int = 0
+    state_bf16: int = 0
 
     def c(self) -> _Shape:
         return _Shape(self.batch, self.heads_v, self.heads_qk, self.d_k, self.d_v, self.W, self.r, self.n_iter,
-                      self.gate, self.smooth, self.delta, self.rec16)
+                      self.gate, self.smooth, self.delta, self.rec16, self.state_bf16)
 
 
 class State:
@@ -70,11 +71,13 @@ class State:
 
     ``quant=False`` keeps the boundary state in fp32 (``S0``) and uses no
     compensators: the windowed algebra with the quantizer replaced by the
-    identity.
+    identity.  With ``sh.state_bf16`` (per-window BF16) the boundary state
+    lives in ``S0`` as well, as bfloat16 values held in fp32.
     """
 
     def __init__(self, sh: Shape, quant: bool = True):
         B, H, K, V, W, r = sh.batch, sh.heads_v, sh.d_k, sh.d_v, sh.W, sh.r
+        quant = quant and not sh.state_bf16
         self.shape = sh
         self.quant = quant
         self.codes = np.zeros((B, H, K, V), np.int8)

@@ -48,6 +48,7 @@ class Workload:
     smooth: int = 1
     delta: int = 1                  # 1: delta rule (GDN, KDA); 0: no read-back, u = v (Mamba2, GLA, ...)
     rec16: int = 0                  # 1: fp16 record buffer (the paper's storage), 0: fp32
+    state_bf16: int = 0             # 1: per-window BF16 boundary state (the -w baseline; r = 0), 0: the 8-bit method
     v_dist: str = "normal"          # "normal" | "student3"
     outlier_frac: float = 0.0
     outlier_mag: float = 1.0

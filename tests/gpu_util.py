@@ -8,7 +8,7 @@ from paper_2609_38166_b200 import lq, synth
 
 def shapes(wl):
     """(oracle shape, library shape) of a workload."""
-    args = (wl.batch, wl.heads_v, wl.heads_qk, wl.d_k, wl.d_v, wl.W, wl.r, wl.n_iter, wl.gate, wl.smooth, wl.delta, wl.rec16)
+    args = (wl.batch, wl.heads_v, wl.heads_qk, wl.d_k, wl.d_v, wl.W, wl.r, wl.n_iter, wl.gate, wl.smooth, wl.delta, wl.rec16, wl.state_bf16)
     return OShape(*args), lq.Shape(*args)
 
 

@@ -12,7 +12,7 @@ GATES = [synth.GATE_SCALAR, synth.GATE_DIAG]
 
 
 def _shape(wl):
-    return Shape(wl.batch, wl.heads_v, wl.heads_qk, wl.d_k, wl.d_v, wl.W, wl.r, wl.n_iter, wl.gate, wl.smooth, wl.delta, wl.rec16)
+    return Shape(wl.batch, wl.heads_v, wl.heads_qk, wl.d_k, wl.d_v, wl.W, wl.r, wl.n_iter, wl.gate, wl.smooth, wl.delta, wl.rec16, wl.state_bf16)
 
 
 def _rel(a, b):
