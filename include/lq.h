@@ -80,6 +80,11 @@ typedef struct {
                 /* accounting (kt, u and the diagonal gate's alpha are rounded, with       */
                 /* saturation, when a record is appended; the scalar gate's decays stay    */
                 /* fp32; `o` of the appending token uses the unrounded u); 0: fp32 records */
+  int state_bf16; /* 1: "per-window BF16", the -w baseline of the paper's Fig. 3 and Table 2: the    */
+                /* boundary state is the dense state rounded to bfloat16 (nearest even) once per  */
+                /* window, with no scale, smoothing or compensator; needs r = 0 and smooth = 0;   */
+                /* the readout is S0^T x in binary32 in the fixed summation order.  0: the 8-bit  */
+                /* representation of Eq. 7                                                        */
 } lq_shape;
 
 /*
@@ -96,6 +101,8 @@ typedef struct {
  *     + 4*d_k                         comp_k     fp16 [r][d_k]    unit-length key side of the compensators
  *     + 2*r*d_k                       comp_u     fp16 [r][d_v]    value side (carries the magnitude)
  *   (17408 + 512 r bytes at d_k = d_v = 128: 19456 for r = 4, i.e. 1.19 bytes per state element.)
+ *   With shape.state_bf16 the block is instead   state  bf16 [d_v][d_k]   S0^T: S0[i][j] sits at [j][i]
+ *   (32768 bytes).
  *
  * records: one row of lq_record_floats(shape) values (fp32, or fp16 with shape.rec16) per buffered record, [B,Hv,W] rows:
  *     kt[d_k] | u[d_v]                write key kt = beta*k and correction u = v - S^T(alpha.k)  (Eq. 3)

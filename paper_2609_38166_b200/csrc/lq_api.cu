@@ -6,6 +6,7 @@
 #include <cstdlib>
 #include <mutex>
 
+#include "lq_bf16w.cuh"
 #include "lq_boundary.cuh"
 #include "lq_decode.cuh"
 #include "lq_fused.cuh"
@@ -191,7 +192,8 @@ static lq_status check_shape(const lq_shape *s) {
   if (!s) return LQ_ERR_NULL;
   if (s->batch < 0 || s->heads_v <= 0 || s->heads_qk <= 0 || s->d_k <= 0 || s->d_v <= 0 || s->W <= 0 || s->r < 0 ||
       s->n_iter < 1 || s->heads_v % s->heads_qk != 0 || (s->gate != LQ_GATE_SCALAR && s->gate != LQ_GATE_DIAG) ||
-      (s->delta != 0 && s->delta != 1) || (s->rec16 != 0 && s->rec16 != 1))
+      (s->delta != 0 && s->delta != 1) || (s->rec16 != 0 && s->rec16 != 1) ||
+      (s->state_bf16 != 0 && s->state_bf16 != 1) || (s->state_bf16 && (s->r != 0 || s->smooth != 0)))
     return LQ_ERR_SHAPE;
   if (s->d_k != D || s->d_v != D || s->W > MAX_W || s->r > MAX_R) return LQ_ERR_UNSUPPORTED;
   return LQ_OK;
@@ -308,8 +310,23 @@ static lq_status launch_persistent(K kernel, long items, int block, size_t smem,
   return launch_dependent(kernel, static_cast<int>(items < resident ? items : resident), block, smem, stream, p);
 }
 
+// per-window BF16: one CTA per head, those whose sequence is not due leave at once
+template <int MODE>
+static lq_status launch_bf16w_boundary(const lq_shape *s, const Params &p, cudaStream_t stream) {
+  const bool diag = s->gate == LQ_GATE_DIAG;
+  const bool r16 = MODE != 1 && s->rec16 != 0;
+  const size_t smem = bf16w_boundary_smem(s->W);
+  const int grid = s->batch * s->heads_v;
+  if (r16)
+    return diag ? launch_dependent(bf16w_boundary_kernel<LQ_GATE_DIAG, MODE == 1 ? 0 : MODE, true>, grid, 256, smem, stream, p)
+                : launch_dependent(bf16w_boundary_kernel<LQ_GATE_SCALAR, MODE == 1 ? 0 : MODE, true>, grid, 256, smem, stream, p);
+  return diag ? launch_dependent(bf16w_boundary_kernel<LQ_GATE_DIAG, MODE, false>, grid, 256, smem, stream, p)
+              : launch_dependent(bf16w_boundary_kernel<LQ_GATE_SCALAR, MODE, false>, grid, 256, smem, stream, p);
+}
+
 template <int MODE>
 static lq_status launch_boundary(const lq_shape *s, const Params &p, cudaStream_t stream) {
+  if (s->state_bf16) return launch_bf16w_boundary<MODE>(s, p, stream);
   const bool diag = s->gate == LQ_GATE_DIAG;
   const bool r16 = MODE != 1 && s->rec16 != 0;               // quantizing a dense state reads no records
   const int bufs = MODE == 1 ? 1 : BoundarySmem::buffers(s->W, s->r, diag, r16);
@@ -391,6 +408,21 @@ static lq_status decode_step_impl(const lq_shape *shape, const lq_state *state, 
   // persistent two-warp CTAs, each with its own shared-memory slot: as many as are resident at once
   const bool r16 = shape->rec16 != 0;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (shape->state_bf16) {                   // per-window BF16: one CTA per head
+    const int grid = static_cast<int>(nh);
+    if (r16)
+      rc = diag ? launch_dependent(bf16w_decode_kernel<LQ_GATE_DIAG, true>, grid, 256, 0, st, p)
+                : launch_dependent(bf16w_decode_kernel<LQ_GATE_SCALAR, true>, grid, 256, 0, st, p);
+    else
+      rc = diag ? launch_dependent(bf16w_decode_kernel<LQ_GATE_DIAG, false>, grid, 256, 0, st, p)
+                : launch_dependent(bf16w_decode_kernel<LQ_GATE_SCALAR, false>, grid, 256, 0, st, p);
+    if (rc != LQ_OK) return rc;
+    if (between && cudaEventRecord(between, st) != cudaSuccess) {
+      cudaGetLastError();
+      return LQ_ERR_CUDA;
+    }
+    return launch_boundary<0>(shape, p, st);
+  }
   if (!between && fused_step_wanted(nh)) {
     lq_status frc = launch_fused_step(shape, p, st);
     if (frc != LQ_ERR_UNSUPPORTED) return frc;       // does not fit this device or shape: the two kernels below
@@ -421,7 +453,10 @@ lq_status lq_decode_step_profiled(const lq_shape *shape, const lq_state *state, 
   return decode_step_impl(shape, state, q, k, v, beta, alpha, o, stream, static_cast<cudaEvent_t>(event_between));
 }
 
-uint64_t lq_head_bytes(const lq_shape *s) { return check_shape(s) == LQ_OK ? (uint64_t)head_bytes(s->r) : 0; }
+uint64_t lq_head_bytes(const lq_shape *s) {
+  if (check_shape(s) != LQ_OK) return 0;
+  return s->state_bf16 ? (uint64_t)BF16W_HEAD_BYTES : (uint64_t)head_bytes(s->r);
+}
 
 uint64_t lq_record_floats(const lq_shape *s) {
   return check_shape(s) == LQ_OK ? (uint64_t)record_floats(s->gate == LQ_GATE_DIAG) : 0;
@@ -770,7 +805,7 @@ lq_status lq_dequantize_state(const lq_shape *shape, const lq_state *state, floa
 static lq_status ref_step(const lq_shape *shape, float *S, uint16_t *S16, const uint16_t *q, const uint16_t *k,
                           const uint16_t *v, const uint16_t *beta, const uint16_t *alpha, float *o, lq_stream stream) {
   lq_shape s = *shape;
-  s.W = 1; s.r = 0; s.n_iter = 1;      // unused by the baseline
+  s.W = 1; s.r = 0; s.n_iter = 1; s.state_bf16 = 0;      // unused by the baseline
   lq_status rc = check_shape(&s);
   if (rc != LQ_OK) return rc;
   if ((rc = check_ptrs({S ? (const void *)S : (const void *)S16, q, k, v, o})) != LQ_OK) return rc;

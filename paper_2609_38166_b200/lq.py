@@ -31,7 +31,7 @@ class LqError(RuntimeError):
 
 class _Shape(C.Structure):
     _fields_ = [(n, C.c_int) for n in
-                ("batch", "heads_v", "heads_qk", "d_k", "d_v", "W", "r", "n_iter", "gate", "smooth", "delta", "rec16")]
+                ("batch", "heads_v", "heads_qk", "d_k", "d_v", "W", "r", "n_iter", "gate", "smooth", "delta", "rec16", "state_bf16")]
 
 
 class _State(C.Structure):
@@ -77,10 +77,11 @@ class Shape:
     smooth: int = 1
     delta: int = 1
     rec16: int = 0
+    state_bf16: int = 0
 
     def c(self) -> _Shape:
         return _Shape(self.batch, self.heads_v, self.heads_qk, self.d_k, self.d_v, self.W, self.r, self.n_iter,
-                      self.gate, self.smooth, self.delta, self.rec16)
+                      self.gate, self.smooth, self.delta, self.rec16, self.state_bf16)
 
 
 def head_bytes(sh: Shape) -> int:
@@ -108,6 +109,12 @@ class State:
         self.records = torch.zeros((B, H, W, rf), dtype=torch.float16 if sh.rec16 else torch.float32, device=device)
         self.decays = torch.zeros((B, H, W), dtype=torch.float32, device=device)
         self.win_pos = torch.zeros((B,), dtype=torch.int32, device=device)
+        if sh.state_bf16:                    # per-window BF16: the head block is S^T in bfloat16, nothing else
+            assert hb == 2 * K * V
+            self.state16 = self.heads.view(torch.bfloat16).unflatten(-1, (V, K))
+            self.codes = self.col_scale = self.row_smooth = self.comp_k = self.comp_u = None
+            self._record_views(sh)
+            return
         o = 0
         self.codes = self.heads[..., o:o + K * V].view(torch.int8).unflatten(-1, (V, K)); o += K * V   # Z^T
         self.col_scale = self.heads[..., o:o + 4 * V].view(torch.float32); o += 4 * V
@@ -116,6 +123,10 @@ class State:
         self.comp_u = self.heads[..., o:o + 2 * r * V].view(torch.float16).unflatten(-1, (r, V)); o += 2 * r * V
         assert o == hb
         self.row_smooth.fill_(1.0)
+        self._record_views(sh)
+
+    def _record_views(self, sh: Shape) -> None:
+        K, V = sh.d_k, sh.d_v
         self.buf_k = self.records[..., 0:K]
         self.buf_u = self.records[..., K:K + V]
         self.buf_a = self.records[..., K + V:K + V + K] if sh.gate == GATE_DIAG else self.decays
@@ -151,7 +162,7 @@ def _ptr(t: Optional[torch.Tensor], b0: int = 0) -> C.c_void_p:
 
 def _sub(sh: Shape, b0: int, nb: Optional[int]) -> Shape:
     nb = sh.batch - b0 if nb is None else nb
-    return Shape(nb, sh.heads_v, sh.heads_qk, sh.d_k, sh.d_v, sh.W, sh.r, sh.n_iter, sh.gate, sh.smooth, sh.delta, sh.rec16)
+    return Shape(nb, sh.heads_v, sh.heads_qk, sh.d_k, sh.d_v, sh.W, sh.r, sh.n_iter, sh.gate, sh.smooth, sh.delta, sh.rec16, sh.state_bf16)
 
 
 def decode_step(sh: Shape, st: State, q, k, v, beta, alpha, o, stream=None, b0: int = 0, nb: Optional[int] = None):

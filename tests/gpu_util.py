@@ -39,6 +39,11 @@ def tok_dev(tok: dict) -> dict:
 
 def state_to_dev(ost: OState, lsh) -> "lq.State":
     st = lq.State(lsh)
+    if lsh.state_bf16:
+        st.state16.copy_(dev(np.ascontiguousarray(ost.S0.transpose(0, 1, 3, 2))).to(torch.bfloat16))   # exact: bfloat16 values
+        st.buf_k.copy_(dev(ost.buf_k)); st.buf_u.copy_(dev(ost.buf_u)); st.buf_a.copy_(dev(ost.buf_a))
+        st.win_pos.copy_(dev(ost.win_pos))
+        return st
     st.codes.copy_(dev(np.ascontiguousarray(ost.codes.transpose(0, 1, 3, 2)))); st.col_scale.copy_(dev(ost.col_scale)); st.row_smooth.copy_(dev(ost.row_smooth))
     if lsh.r > 0:
         st.comp_k.copy_(dev(ost.comp_k).view(torch.float16)); st.comp_u.copy_(dev(ost.comp_u).view(torch.float16))
@@ -63,6 +68,18 @@ def assert_state_parity(st: "lq.State", ost: OState, r: int, what: str = "", exa
     within 1e-3 relative / 1e-5 absolute.  With `exact` (the default) every array must match bit for bit,
     which the fixed summation order makes possible."""
     torch.cuda.synchronize()
+    if st.shape.state_bf16:                  # per-window BF16: the boundary state is S0^T in bfloat16
+        got = np.ascontiguousarray(st.state16.float().cpu().numpy().transpose(0, 1, 3, 2))
+        if exact:
+            assert np.array_equal(got, ost.S0), (what, "state16", float(np.abs(got - ost.S0).max()))
+        else:
+            assert np.allclose(got, ost.S0, rtol=2.0 ** -7, atol=1e-5), (what, "state16")
+        for name, g, w in (("buf_k", host_f32(st.buf_k), ost.buf_k), ("buf_u", host_f32(st.buf_u), ost.buf_u),
+                           ("buf_a", host_f32(st.buf_a), ost.buf_a)):
+            assert np.allclose(g, w, rtol=1e-3, atol=1e-5), (what, name)
+            assert not exact or np.array_equal(g, w), (what, name, float(np.abs(g - w).max()))
+        assert np.array_equal(host(st.win_pos), ost.win_pos), (what, host(st.win_pos), ost.win_pos)
+        return
     frac, worst = code_mismatch(gpu_codes(st), ost.codes)
     assert worst <= 1 and frac <= 1e-4, (what, frac, worst)
     pairs = [("col_scale", host(st.col_scale), ost.col_scale), ("row_smooth", host(st.row_smooth), ost.row_smooth),

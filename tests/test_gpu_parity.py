@@ -372,3 +372,50 @@ def test_pipelined_host_entry_point(oracle, gate, batch):
         _close(o_h.numpy(), want, f"pipelined host-buffer step {step}")
     gu.assert_state_parity(st, ost, wl.r, "pipelined host-buffer chain")
     assert lq.check_device() == 0
+
+
+# ---- per-window BF16 (the -w baseline): bfloat16 boundary state, no scale, smoothing or compensators ----
+
+def _bf16w(name, batch, heads_v, heads_qk, **kw):
+    return synth.Workload(name, batch, heads_v, heads_qk, r=0, smooth=0, state_bf16=1, **kw)
+
+
+@pytest.mark.parametrize("gate", GATES)
+@pytest.mark.parametrize("W,rec16,delta", [(16, 0, 1), (1, 0, 1), (5, 1, 1), (64, 0, 1), (40, 1, 0)])
+def test_per_window_bf16_chain(oracle, gate, W, rec16, delta):
+    """Every output, the bfloat16 boundary state after every boundary and the record buffer, bit for bit."""
+    wl = _bf16w("w", 6, 4, 2, W=W, gate=gate, rec16=rec16, delta=delta, seed=600 + W)
+    _run_chain(oracle, wl, 2 * W + 3 if W <= 16 else W + 5, init="dense", stagger=True, check_every=4)
+
+
+@pytest.mark.parametrize("gate", GATES)
+def test_per_window_bf16_dequantize_and_forced_flush(oracle, gate):
+    wl = _bf16w("wd", 4, 3, 3, W=7, gate=gate, seed=610)
+    osh, lsh = gu.shapes(wl)
+    ost = OState(osh)
+    oracle.quantize_state(osh, synth.dense_states(wl, 2), ost)
+    rng = np.random.default_rng(7)
+    ost.win_pos[:] = [0, 1, 3, 6]
+    ost.buf_k[...] = rng.standard_normal(ost.buf_k.shape).astype(np.float32) * 0.1
+    ost.buf_u[...] = rng.standard_normal(ost.buf_u.shape).astype(np.float32)
+    ost.buf_a[...] = rng.uniform(0.2, 1.0, ost.buf_a.shape).astype(np.float32)
+    want = oracle.dequantize_state(osh, ost)
+    st = gu.state_to_dev(ost, lsh)
+    S = torch.empty((4, 3, 128, 128), dtype=torch.float32, device="cuda")
+    lq.dequantize_state(lsh, st, S)
+    torch.cuda.synchronize()
+    assert np.array_equal(gu.host(S), want)
+    gu.assert_state_parity(st, ost, 0, "dequantize leaves the state alone")
+    lq.window_flush(lsh, st, force=False)
+    gu.assert_state_parity(st, ost, 0, "unforced flush is a no-op")
+    oracle.window_flush(osh, ost, force=True)
+    lq.window_flush(lsh, st, force=True)
+    gu.assert_state_parity(st, ost, 0, "forced flush")
+    assert st.win_pos.tolist() == [0, 0, 0, 0]
+
+
+def test_per_window_bf16_refuses_compensators_and_smoothing():
+    for kw in ({"r": 2, "smooth": 0}, {"r": 0, "smooth": 1}):
+        sh = lq.Shape(1, 1, 1, 128, 128, 16, n_iter=2, state_bf16=1, **kw)
+        assert lq.head_bytes(sh) == 0
+    assert lq.head_bytes(lq.Shape(1, 1, 1, 128, 128, 16, r=0, smooth=0, state_bf16=1)) == 2 * 128 * 128
