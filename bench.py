@@ -237,7 +237,7 @@ def prepare_state(wl, lq, torch, log, WARM_TOKENS=WARM_TOKENS):
     """512 warm-up tokens on the fp32-state kernel, quantized group by group so that at the end group g
     (a contiguous slice of the batch) holds g buffered records: window offsets uniform over [0, W)."""
     sh = lq.Shape(wl.batch, wl.heads_v, wl.heads_qk, wl.d_k, wl.d_v, wl.W, wl.r, wl.n_iter, wl.gate, wl.smooth, wl.delta,
-                  wl.rec16)
+                  wl.rec16, wl.state_bf16)
     B, W = wl.batch, wl.W
     st = lq.State(sh)
     S = torch.zeros((B, wl.heads_v, wl.d_k, wl.d_v), dtype=torch.float32, device="cuda")
@@ -624,6 +624,7 @@ def run_ladder(args):
     stream = torch.cuda.current_stream()
     rungs = [("fp32 state, every token", None),
              ("bf16 state, every token", "bf16"),
+             ("bf16 per window (W=16): the -w baseline", dict(W=16, r=0, smooth=0, state_bf16=1)),
              ("int8 every token (W=1, no compensators, no smoothing)", dict(W=1, r=0, smooth=0)),
              ("int8 per window (W=16), no compensators, no smoothing", dict(W=16, r=0, smooth=0)),
              ("+ 4 Compensator Tokens", dict(W=16, r=4, smooth=0)),
@@ -639,7 +640,8 @@ def run_ladder(args):
         for label, var in rungs:
             # ---- error against the fp32 recurrence ----
             wl = small if not isinstance(var, dict) else small.with_(**var)
-            sh = lq.Shape(wl.batch, 32, wl.heads_qk, 128, 128, wl.W, wl.r, wl.n_iter, wl.gate, wl.smooth)
+            sh = lq.Shape(wl.batch, 32, wl.heads_qk, 128, 128, wl.W, wl.r, wl.n_iter, wl.gate, wl.smooth,
+                          state_bf16=wl.state_bf16)
             S = torch.zeros((wl.batch, 32, 128, 128), dtype=torch.float32, device="cuda")
             o_ref = torch.empty((wl.batch, 32, 128), dtype=torch.float32, device="cuda")
             o_var = torch.empty_like(o_ref)
@@ -668,12 +670,13 @@ def run_ladder(args):
             del S, S16, st
             # ---- speed on the full batch, windows staggered as in the headline run ----
             wlb = base if not isinstance(var, dict) else base.with_(**var)
-            shb = lq.Shape(wlb.batch, 32, wlb.heads_qk, 128, 128, wlb.W, wlb.r, wlb.n_iter, wlb.gate, wlb.smooth)
+            shb = lq.Shape(wlb.batch, 32, wlb.heads_qk, 128, 128, wlb.W, wlb.r, wlb.n_iter, wlb.gate, wlb.smooth,
+                           state_bf16=wlb.state_bf16)
             ob = torch.empty((wlb.batch, 32, 128), dtype=torch.float32, device="cuda")
             if isinstance(var, dict):
                 _, stb, ob = prepare_state(wlb, lq, torch, lambda m: None, 32)
                 fn = lambda t: lq.decode_step(shb, stb, *[toks_big[t % 16][k] for k in keys], ob, stream)
-                state_b = 128 * 128 + 1024 + 2 * wlb.r * 256
+                state_b = 2 * 128 * 128 if wlb.state_bf16 else 128 * 128 + 1024 + 2 * wlb.r * 256
             elif var == "bf16":
                 Sb = torch.zeros((wlb.batch, 32, 128, 128), dtype=torch.int16, device="cuda")
                 fn = lambda t: lq.ref_decode_step_bf16(shb, Sb, *[toks_big[t % 16][k] for k in keys], ob, stream)

@@ -270,7 +270,8 @@ static lq_status launch(K kernel, int grid, int block, size_t smem, cudaStream_t
 template <typename K, typename... Args>
 static lq_status launch_dependent(K kernel, int grid, int block, size_t smem, cudaStream_t stream, const Args &...args) {
   if (grid <= 0) return LQ_OK;
-  if (smem > 48 * 1024 &&
+  // (the opt-in is needed once static + dynamic shared memory pass 48 KB; the kernels here hold up to 20 KB static)
+  if (smem > 24 * 1024 &&
       cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess) {
     cudaGetLastError();
     return LQ_ERR_CUDA;
@@ -310,13 +311,14 @@ static lq_status launch_persistent(K kernel, long items, int block, size_t smem,
   return launch_dependent(kernel, static_cast<int>(items < resident ? items : resident), block, smem, stream, p);
 }
 
-// per-window BF16: one CTA per head, those whose sequence is not due leave at once
+// per-window BF16: persistent CTAs that stride over the heads
 template <int MODE>
 static lq_status launch_bf16w_boundary(const lq_shape *s, const Params &p, cudaStream_t stream) {
   const bool diag = s->gate == LQ_GATE_DIAG;
   const bool r16 = MODE != 1 && s->rec16 != 0;
-  const size_t smem = bf16w_boundary_smem(s->W);
-  const int grid = s->batch * s->heads_v;
+  const size_t smem = bf16w_boundary_smem(s->W, diag, r16);
+  const long nh = (long)s->batch * s->heads_v;
+  const int grid = static_cast<int>(nh < 2L * sm_count() ? nh : 2L * sm_count());      // persistent, two per SM
   if (r16)
     return diag ? launch_dependent(bf16w_boundary_kernel<LQ_GATE_DIAG, MODE == 1 ? 0 : MODE, true>, grid, 256, smem, stream, p)
                 : launch_dependent(bf16w_boundary_kernel<LQ_GATE_SCALAR, MODE == 1 ? 0 : MODE, true>, grid, 256, smem, stream, p);
@@ -410,12 +412,13 @@ static lq_status decode_step_impl(const lq_shape *shape, const lq_state *state, 
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   if (shape->state_bf16) {                   // per-window BF16: one CTA per head
     const int grid = static_cast<int>(nh);
+    const size_t rsm = bf16w_decode_smem(shape->W, diag, r16);
     if (r16)
-      rc = diag ? launch_dependent(bf16w_decode_kernel<LQ_GATE_DIAG, true>, grid, 256, 0, st, p)
-                : launch_dependent(bf16w_decode_kernel<LQ_GATE_SCALAR, true>, grid, 256, 0, st, p);
+      rc = diag ? launch_dependent(bf16w_decode_kernel<LQ_GATE_DIAG, true>, grid, 256, rsm, st, p)
+                : launch_dependent(bf16w_decode_kernel<LQ_GATE_SCALAR, true>, grid, 256, rsm, st, p);
     else
-      rc = diag ? launch_dependent(bf16w_decode_kernel<LQ_GATE_DIAG, false>, grid, 256, 0, st, p)
-                : launch_dependent(bf16w_decode_kernel<LQ_GATE_SCALAR, false>, grid, 256, 0, st, p);
+      rc = diag ? launch_dependent(bf16w_decode_kernel<LQ_GATE_DIAG, false>, grid, 256, rsm, st, p)
+                : launch_dependent(bf16w_decode_kernel<LQ_GATE_SCALAR, false>, grid, 256, rsm, st, p);
     if (rc != LQ_OK) return rc;
     if (between && cudaEventRecord(between, st) != cudaSuccess) {
       cudaGetLastError();

@@ -19,7 +19,8 @@ def _oracle_sequence(oracle, wl, b, toks, warm, steps):
     groups = (wl.batch + per - 1) // per
     g = min(b // per, groups - 1)                       # sequence b is quantized after warm - g tokens
     one = wl.with_(batch=1)
-    sh = OShape(1, wl.heads_v, wl.heads_qk, wl.d_k, wl.d_v, wl.W, wl.r, wl.n_iter, wl.gate, wl.smooth, wl.delta, wl.rec16)
+    sh = OShape(1, wl.heads_v, wl.heads_qk, wl.d_k, wl.d_v, wl.W, wl.r, wl.n_iter, wl.gate, wl.smooth, wl.delta, wl.rec16,
+                wl.state_bf16)
     cut = lambda tok: {k: np.ascontiguousarray(v[b:b + 1]) for k, v in tok.items()}
     S = np.zeros((1, wl.heads_v, wl.d_k, wl.d_v), np.float32)
     st = OState(sh)
@@ -67,6 +68,34 @@ def test_full_batch_against_sampled_oracle_sequences(oracle, name, W, warm, step
                             ("buf_u", st.buf_u, ost.buf_u), ("buf_k", st.buf_k, ost.buf_k)):
             assert np.array_equal(gu.host_f32(g[b]), w[0]), (b, name_)
         assert np.array_equal(gu.host(st.comp_u[b]), ost.comp_u[0]), b
+
+
+@pytest.mark.parametrize("name", ["gdn_b256", "kda_b128_outlier"])
+def test_full_batch_per_window_bf16_against_sampled_oracle_sequences(oracle, name):
+    """The -w baseline at the benchmark's size: outputs, the bfloat16 boundary state and the records of sampled
+    sequences, bit for bit."""
+    W, warm, steps = 16, 20, 18
+    wl = synth.config(name).with_(W=W, r=0, smooth=0, state_bf16=1)
+    toks = [synth.token_inputs(wl, t) for t in range(warm + steps)]
+    sh, st, o = bench.prepare_state(wl, lq, torch, lambda m: None, warm)
+    sample = sorted({0, 1, wl.batch // W, wl.batch // 2 + 3, wl.batch - 1})
+    got = {b: [] for b in sample}
+    for t in range(steps):
+        d = bench.to_dev(toks[warm + t], torch)
+        lq.decode_step(sh, st, d["q"], d["k"], d["v"], d["beta"], d["alpha"], o)
+        oh = o[sample].cpu().numpy()
+        for i, b in enumerate(sample):
+            got[b].append(oh[i])
+    torch.cuda.synchronize()
+    assert lq.check_device() == 0
+    for b in sample:
+        ost, want = _oracle_sequence(oracle, wl, b, toks, warm, steps)
+        for t in range(steps):
+            assert np.array_equal(got[b][t], want[t]), (b, t)
+        assert np.array_equal(st.state16[b].float().cpu().numpy().transpose(0, 2, 1), ost.S0[0]), b
+        assert int(st.win_pos[b]) == int(ost.win_pos[0])
+        for name_, g, w in (("buf_u", st.buf_u, ost.buf_u), ("buf_k", st.buf_k, ost.buf_k)):
+            assert np.array_equal(gu.host_f32(g[b]), w[0]), (b, name_)
 
 
 def test_drift_against_the_unquantized_recurrence():
