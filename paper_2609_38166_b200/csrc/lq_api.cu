@@ -876,6 +876,6 @@ const char *lq_status_string(lq_status status) {
   return "unknown status";
 }
 
-int lq_version(void) { return 3; }
+int lq_version(void) { return 4; }
 
 }  // extern "C"

@@ -87,6 +87,7 @@ __global__ void __launch_bounds__(256, 4) bf16w_decode_kernel(const Params p) {
   for (int top = n - 1; top >= 0; top -= BF16W_CHUNK) {
     const int cnt = top + 1 < BF16W_CHUNK ? top + 1 : BF16W_CHUNK;      // records top, top-1, ..., top-cnt+1
     if (tid < D) {
+#pragma unroll 4
       for (int e = 0; e < cnt; e++) {
         const int j = top - e;
         gk_s[e * D + tid] = g * k_i;
@@ -135,6 +136,7 @@ __global__ void __launch_bounds__(256, 4) bf16w_decode_kernel(const Params p) {
   if (tid < D) {
     // the records' terms: their own sum, from the newest record back, added as one number
     float sk = 0.0f, sq = 0.0f;
+#pragma unroll 4
     for (int jj = n - 1; jj >= 0; jj--) {
       const float uj = static_cast<float>(rec_s[jj * RF + REC_U + tid]);
       sk = fmaf(uj, pk_s[jj], sk);
