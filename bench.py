@@ -382,8 +382,8 @@ def run_cuda(args, wl):
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": o_h.numel() * 4, "steps": n_e2e,
                "ms_per_step": e2e_ms / n_e2e,
                "api": "lq_decode_step_host_pipelined, one call per step: pinned host q,k,v,beta,alpha in (read over the "
-                      "bus by a gather launch per half batch), o out to pinned host memory (copied while the "
-                      "window-boundary kernel runs)"}
+                      "bus by a gather launch per half batch, which may start while the step before is still at its "
+                      "window boundaries), o out to pinned host memory (copied while the window-boundary kernel runs)"}
     except Exception as exc:
         log(f"end-to-end timing failed: {exc!r}")
 

@@ -171,6 +171,15 @@ lq_status lq_decode_step_host(const lq_shape *shape, const lq_state *state, cons
  * pinned host memory, otherwise nothing overlaps.  Batches below sixteen sequences take the unpipelined path.
  * Calls from several host threads are serialised inside the library while they enqueue.
  *
+ * Consecutive calls with the same `stage`, `stream` and shape chain onto each other: the inputs of sub-batch c of
+ * the later call are brought in as soon as the earlier call's decode kernel of sub-batch c has consumed its own,
+ * i.e. next to the earlier call's window-boundary kernels and copies out, and possibly before other work that
+ * was enqueued on `stream` in between.  So the host input arrays must hold their final values when the call is
+ * made (not merely when `stream` reaches it), and between such calls `stage` belongs to the library.  A call of
+ * lq_decode_step_host or lq_decode_step_host_static, another `stage` or another stream ends the chain; the next
+ * pipelined call is then ordered after everything on `stream` again.  Outputs are always stream-ordered: what is
+ * enqueued on `stream` after a call finds o_h complete.
+ *
  * Both host-buffer entry points read the inputs with ONE gather launch (per sub-batch) instead of five copies
  * when all input arrays are pinned, mapped into the device (cudaHostAlloc / cudaHostRegister memory under
  * unified addressing) and 16-byte aligned with sizes that are multiples of 16 bytes; lq_decode_step_host

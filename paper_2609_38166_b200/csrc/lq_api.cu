@@ -4,7 +4,9 @@
 #include <atomic>
 #include <cstdio>
 #include <cstdlib>
+#include <map>
 #include <mutex>
+#include <tuple>
 
 #include "lq_bf16w.cuh"
 #include "lq_boundary.cuh"
@@ -251,14 +253,53 @@ static int sm_count() {
   return cached;
 }
 
+// What a launch needs to ask the runtime only once per (device, kernel): the opt-in to more than 48 KB of shared
+// memory and the number of CTAs of a kernel that an SM holds.  Both calls cost a few microseconds of host time,
+// which a step of two to ten launches would otherwise pay every token.
+static int current_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) {
+    cudaGetLastError();
+    return 0;
+  }
+  return dev;
+}
+
+// (the opt-in is needed once static + dynamic shared memory pass 48 KB; the kernels here hold up to 20 KB static)
+static bool smem_opt_in(const void *kernel, size_t smem) {
+  if (smem <= 24 * 1024) return true;
+  static std::mutex m;
+  static std::map<std::pair<int, const void *>, size_t> granted;
+  std::lock_guard<std::mutex> lock(m);
+  size_t &have = granted[{current_device(), kernel}];
+  if (have >= smem) return true;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess) {
+    cudaGetLastError();
+    return false;
+  }
+  have = smem;
+  return true;
+}
+
+// resident CTAs per SM of `kernel` with this block size and dynamic shared memory (0: the query failed)
+static int ctas_per_sm(const void *kernel, int block, size_t smem) {
+  static std::mutex m;
+  static std::map<std::tuple<int, const void *, int, size_t>, int> known;
+  std::lock_guard<std::mutex> lock(m);
+  int &per_sm = known[std::make_tuple(current_device(), kernel, block, smem)];
+  if (per_sm > 0) return per_sm;
+  int v = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&v, kernel, block, smem) != cudaSuccess || v < 1) {
+    cudaGetLastError();
+    return 0;
+  }
+  return per_sm = v;
+}
+
 template <typename K, typename P>
 static lq_status launch(K kernel, int grid, int block, size_t smem, cudaStream_t stream, const P &p) {
   if (grid <= 0) return LQ_OK;
-  if (smem > 48 * 1024 &&
-      cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess) {
-    cudaGetLastError();
-    return LQ_ERR_CUDA;
-  }
+  if (!smem_opt_in(reinterpret_cast<const void *>(kernel), smem)) return LQ_ERR_CUDA;
   kernel<<<grid, block, smem, stream>>>(p);
   return cudaGetLastError() == cudaSuccess ? LQ_OK : LQ_ERR_CUDA;
 }
@@ -270,12 +311,7 @@ static lq_status launch(K kernel, int grid, int block, size_t smem, cudaStream_t
 template <typename K, typename... Args>
 static lq_status launch_dependent(K kernel, int grid, int block, size_t smem, cudaStream_t stream, const Args &...args) {
   if (grid <= 0) return LQ_OK;
-  // (the opt-in is needed once static + dynamic shared memory pass 48 KB; the kernels here hold up to 20 KB static)
-  if (smem > 24 * 1024 &&
-      cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess) {
-    cudaGetLastError();
-    return LQ_ERR_CUDA;
-  }
+  if (!smem_opt_in(reinterpret_cast<const void *>(kernel), smem)) return LQ_ERR_CUDA;
   cudaLaunchAttribute attr;
   attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr.val.programmaticStreamSerializationAllowed = 1;
@@ -297,16 +333,9 @@ static lq_status launch_dependent(K kernel, int grid, int block, size_t smem, cu
 template <typename K>
 static lq_status launch_persistent(K kernel, long items, int block, size_t smem, cudaStream_t stream, const Params &p) {
   if (items <= 0) return LQ_OK;
-  if (smem > 48 * 1024 &&
-      cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess) {
-    cudaGetLastError();
-    return LQ_ERR_CUDA;
-  }
-  int per_sm = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, block, smem) != cudaSuccess || per_sm < 1) {
-    cudaGetLastError();
-    return LQ_ERR_CUDA;
-  }
+  if (!smem_opt_in(reinterpret_cast<const void *>(kernel), smem)) return LQ_ERR_CUDA;
+  const int per_sm = ctas_per_sm(reinterpret_cast<const void *>(kernel), block, smem);
+  if (per_sm < 1) return LQ_ERR_CUDA;
   const long resident = (long)per_sm * sm_count();
   return launch_dependent(kernel, static_cast<int>(items < resident ? items : resident), block, smem, stream, p);
 }
@@ -359,15 +388,9 @@ static lq_status launch_fused_step_t(const lq_shape *s, const Params &p, cudaStr
   const size_t smem = fused_smem_bytes(s->W, s->r, diag, R16);
   auto kernel = fused_step_kernel<GATE, R16>;
   if (smem > 227 * 1024) return LQ_ERR_UNSUPPORTED;
-  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess) {
-    cudaGetLastError();
-    return LQ_ERR_UNSUPPORTED;
-  }
-  int per_sm = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, 256, smem) != cudaSuccess || per_sm < 2) {
-    cudaGetLastError();
+  if (!smem_opt_in(reinterpret_cast<const void *>(kernel), smem)) return LQ_ERR_UNSUPPORTED;
+  if (ctas_per_sm(reinterpret_cast<const void *>(kernel), 256, smem) < 2)
     return LQ_ERR_UNSUPPORTED;               // two CTAs per SM are the design
-  }
   const long nh = (long)s->batch * s->heads_v;
   const int sms = sm_count();
   if (nh > (long)sms * FUSED_SLOTS * FUSED_NBUF || nh > (long)sms * 2048) return LQ_ERR_UNSUPPORTED;
@@ -514,6 +537,8 @@ T *device_alias(T *host) {
 
 extern "C" {
 
+static void host_pipe_break_chain();
+
 static lq_status host_step_impl(const lq_shape *shape, const lq_state *state, const uint16_t *q_h, const uint16_t *k_h,
                                 const uint16_t *v_h, const uint16_t *beta_h, const uint16_t *alpha_h, float *o_h,
                                 void *stage, lq_stream stream, bool direct_ok) {
@@ -534,6 +559,7 @@ static lq_status host_step_impl(const lq_shape *shape, const lq_state *state, co
   float *o_d = reinterpret_cast<float *>(base);
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   if (B == 0) return LQ_OK;
+  host_pipe_break_chain();                   // this call writes `stage` in stream order only
 
   // Fast path, when all six host arrays are pinned, mapped into the device and 16-byte aligned: one gather
   // launch reads the inputs over the bus, and the decode kernel writes o straight into the host array (posted
@@ -594,6 +620,13 @@ struct HostPipe {
   bool ready = false;
   cudaStream_t s_in = nullptr, s_out = nullptr;
   cudaEvent_t start = nullptr, out = nullptr, in[PIPE_CHUNKS] = {}, done[PIPE_CHUNKS] = {};
+  // The previous pipelined call on this device, if the next one may chain onto it: same staging buffer, stream
+  // and staging layout.  done[c] then still marks the moment that call's decode kernel had consumed the inputs
+  // of sub-batch c.
+  bool chain = false;
+  const void *stage = nullptr;
+  cudaStream_t stream = nullptr;
+  uint64_t layout[5] = {};                   // B, Hv, Hqk, gate, W
 };
 std::mutex g_pipe_mutex;
 HostPipe g_pipes[64];
@@ -624,12 +657,23 @@ lq_status host_pipe(HostPipe **out) {
 }
 }  // namespace
 
+// a later pipelined call must not start reading its inputs early: something else is about to use a staging buffer
+static void host_pipe_break_chain() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+    cudaGetLastError();
+    return;
+  }
+  std::lock_guard<std::mutex> lock(g_pipe_mutex);
+  g_pipes[dev].chain = false;
+}
+
 lq_status lq_decode_step_host_pipelined(const lq_shape *shape, const lq_state *state, const uint16_t *q_h,
                                         const uint16_t *k_h, const uint16_t *v_h, const uint16_t *beta_h,
                                         const uint16_t *alpha_h, float *o_h, void *stage, lq_stream stream) {
   lq_status rc = check_shape(shape);
   if (rc != LQ_OK) return rc;
-  if (shape->batch < 8 * PIPE_CHUNKS)          // nothing to overlap
+  if (shape->batch < 8 * PIPE_CHUNKS)          // nothing to overlap (breaks a chain of pipelined calls as well)
     return lq_decode_step_host(shape, state, q_h, k_h, v_h, beta_h, alpha_h, o_h, stage, stream);
   if ((rc = check_state(shape, state, true)) != LQ_OK) return rc;
   if (!q_h || !k_h || !v_h || !beta_h || !alpha_h || !o_h || !stage) return LQ_ERR_NULL;
@@ -670,12 +714,21 @@ lq_status lq_decode_step_host_pipelined(const lq_shape *shape, const lq_state *s
   std::lock_guard<std::mutex> lock(g_pipe_mutex);   // the events below are shared by all callers on a device
   HostPipe *hp = nullptr;
   if ((rc = host_pipe(&hp)) != LQ_OK) return rc;
-  bool ok = cudaEventRecord(hp->start, st) == cudaSuccess &&          // after everything already on `stream`
-            cudaStreamWaitEvent(hp->s_in, hp->start, 0) == cudaSuccess &&
-            cudaStreamWaitEvent(hp->s_out, hp->start, 0) == cudaSuccess;
+  // Chained onto the previous call (same staging buffer, stream and layout): the inputs of sub-batch c may be
+  // brought in as soon as that call's decode kernel of sub-batch c has read its own - next to that call's
+  // window-boundary kernels and copies out - instead of after everything on `stream`.
+  const uint64_t layout[5] = {B, Hv, Hqk, (uint64_t)shape->gate, (uint64_t)shape->W};
+  const bool chained = hp->chain && hp->stage == stage && hp->stream == st &&
+                       std::equal(layout, layout + 5, hp->layout);
+  hp->chain = false;                         // set again at the end, if everything was enqueued
+  // (the copy-out stream needs no tie at the start: all it does waits for a kernel of this call on `stream`)
+  bool ok = chained || (cudaEventRecord(hp->start, st) == cudaSuccess &&    // after everything already on `stream`
+                        cudaStreamWaitEvent(hp->s_in, hp->start, 0) == cudaSuccess);
   for (int c = 0; ok && c < PIPE_CHUNKS; c++) {
     const uint64_t b0 = lo[c], nb = lo[c + 1] - lo[c];
     if (nb == 0) continue;
+    if (chained) ok = cudaStreamWaitEvent(hp->s_in, hp->done[c], 0) == cudaSuccess;   // (the previous call's record)
+    if (!ok) break;
     if (mapped) {
       GatherSegs g;
       for (int i = 0; i < 5; i++) {
@@ -701,7 +754,7 @@ lq_status lq_decode_step_host_pipelined(const lq_shape *shape, const lq_state *s
     lq_shape sub = *shape;
     sub.batch = static_cast<int>(nb);
     lq_state ss = *state;
-    ss.heads += b0 * Hv * head_bytes(shape->r);
+    ss.heads += b0 * Hv * (shape->state_bf16 ? (uint64_t)BF16W_HEAD_BYTES : (uint64_t)head_bytes(shape->r));
     ss.records = static_cast<char *>(ss.records) + b0 * Hv * shape->W * record_floats(diag) * (shape->rec16 ? 2 : 4);
     if (ss.decays) ss.decays += b0 * Hv * shape->W;
     ss.win_pos += b0;
@@ -712,15 +765,21 @@ lq_status lq_decode_step_host_pipelined(const lq_shape *shape, const lq_state *s
          cudaMemcpyAsync(o_h + b0 * ev, o_d + b0 * ev, 4 * nb * ev, cudaMemcpyDeviceToHost, hp->s_out) == cudaSuccess;
   }
   // join: whatever was put on the side streams is waited for by `stream`, also after an error above
-  const bool joined = cudaEventRecord(hp->out, hp->s_out) == cudaSuccess &&
-                      cudaStreamWaitEvent(st, hp->out, 0) == cudaSuccess &&
-                      cudaEventRecord(hp->out, hp->s_in) == cudaSuccess &&
-                      cudaStreamWaitEvent(st, hp->out, 0) == cudaSuccess;
+  // (`stream` has waited for every copy-in of this call already, sub-batch by sub-batch, unless an error cut the
+  // loop above short)
+  bool joined = cudaEventRecord(hp->out, hp->s_out) == cudaSuccess && cudaStreamWaitEvent(st, hp->out, 0) == cudaSuccess;
+  if (rc != LQ_OK || !ok)
+    joined = cudaEventRecord(hp->out, hp->s_in) == cudaSuccess && cudaStreamWaitEvent(st, hp->out, 0) == cudaSuccess &&
+             joined;
   if (rc != LQ_OK) return rc;
   if (!ok || !joined) {
     cudaGetLastError();
     return LQ_ERR_CUDA;
   }
+  hp->chain = true;
+  hp->stage = stage;
+  hp->stream = st;
+  std::copy(layout, layout + 5, hp->layout);
   return LQ_OK;
 }
 

@@ -374,6 +374,42 @@ def test_pipelined_host_entry_point(oracle, gate, batch):
     assert lq.check_device() == 0
 
 
+@pytest.mark.parametrize("gate,state_bf16", [(synth.GATE_SCALAR, 0), (synth.GATE_DIAG, 0), (synth.GATE_SCALAR, 1)])
+def test_pipelined_host_steps_back_to_back(oracle, gate, state_bf16):
+    """Consecutive pipelined calls without a synchronisation in between chain onto each other (the inputs of a
+    call are brought in while the call before it is still computing and copying out): every token has its own
+    pinned inputs and its own output array, and everything is compared once at the end."""
+    kw = dict(r=0, smooth=0, state_bf16=1) if state_bf16 else dict(r=2)
+    wl = synth.Workload("hb", 40, 4, 2, W=4, gate=gate, seed=760, **kw)
+    osh, lsh = gu.shapes(wl)
+    ost = OState(osh)
+    S0 = synth.dense_states(wl, 12)
+    oracle.quantize_state(osh, S0, ost)
+    st = lq.State(lsh)
+    lq.quantize_state(lsh, gu.dev(S0), st)
+    stage = torch.empty((lq.decode_stage_bytes(lsh),), dtype=torch.uint8, device="cuda")
+    steps = 11
+    toks = [synth.token_inputs(wl, t) for t in range(steps)]
+    pins = [{k: torch.from_numpy(v.view(np.int16)).pin_memory() for k, v in tok.items()} for tok in toks]
+    outs = [torch.full((40, 4, 128), float("nan"), dtype=torch.float32).pin_memory() for _ in range(steps)]
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        for t in range(steps - 1):           # (the last token is the one the unpipelined call below takes)
+            d = pins[t]
+            lq.decode_step_host_pipelined(lsh, st, d["q"], d["k"], d["v"], d["beta"], d["alpha"], outs[t], stage, side)
+            if t == 5:                       # an unpipelined call in between breaks the chain and must still be ordered
+                t2 = steps - 1
+                d = pins[t2]
+                lq.decode_step_host(lsh, st, d["q"], d["k"], d["v"], d["beta"], d["alpha"], outs[t2], stage, side)
+    side.synchronize()
+    order = list(range(6)) + [steps - 1] + list(range(6, steps - 1))
+    for t in order:
+        want = oracle.decode_step(osh, ost, **toks[t])
+        _close(outs[t].numpy(), want, f"back-to-back host step {t}")
+    gu.assert_state_parity(st, ost, wl.r, "back-to-back pipelined chain")
+    assert lq.check_device() == 0
+
+
 # ---- per-window BF16 (the -w baseline): bfloat16 boundary state, no scale, smoothing or compensators ----
 
 def _bf16w(name, batch, heads_v, heads_qk, **kw):
