@@ -78,6 +78,21 @@ __device__ __forceinline__ void stage_issue(const Params &p, const BoundarySmem 
     cp_async16(sm.ckh + 8 * e, hb + HB_COMP_K + 16 * e);      // (cuh follows ckh in the buffer as in the block)
 }
 
+// M += x y^T on the register tile, two columns per instruction (fma.rn.f32x2 is two independent round-to-nearest
+// FMAs, so the values are those of fmaf; what it halves is the issue slots of the phases that are bound by them).
+__device__ __forceinline__ void rank1_update(float (&M)[8][8], const float (&x)[8], const float (&y)[8]) {
+#pragma unroll
+  for (int a = 0; a < 8; a++) {
+    const float2 xa = make_float2(x[a], x[a]);
+#pragma unroll
+    for (int b = 0; b < 8; b += 2) {
+      const float2 m = __ffma2_rn(xa, make_float2(y[b], y[b + 1]), make_float2(M[a][b], M[a][b + 1]));
+      M[a][b] = m.x;
+      M[a][b + 1] = m.y;
+    }
+  }
+}
+
 // Eq. 7 for the tile of thread t: M = Gamma_{1:n}[C (Z/127) B + Kc Uc^T] + sum_j Gamma_{j+1:n} kt_j u_j^T,
 // evaluated per element as  base = c_i*(Z_ij*s_j) with s_j the stored code step; base = fma(kc_hi, uc_hj, base) for h = 0..r-1;
 // x = gamma_i*base; x = fma(kd_ji, u_jj, x) for j = 0..n-1.  No sum crosses threads.
@@ -148,10 +163,7 @@ __device__ __forceinline__ void reconstruct_tile(const Params &p, const Boundary
     float kc[8], uc[8];
     load8(sm.ck + h * D + 8 * t.ty, kc);
     load8(sm.cu + h * D + 8 * t.tx, uc);
-#pragma unroll
-    for (int a = 0; a < 8; a++)
-#pragma unroll
-      for (int b = 0; b < 8; b++) M[a][b] = fmaf(kc[a], uc[b], M[a][b]);
+    rank1_update(M, kc, uc);
   }
 #pragma unroll
   for (int a = 0; a < 8; a++)
@@ -161,10 +173,7 @@ __device__ __forceinline__ void reconstruct_tile(const Params &p, const Boundary
     float kj[8], uj[8];
     load8(sm.kd + j * D + 8 * t.ty, kj);
     load8(sm.bu + j * D + 8 * t.tx, uj);
-#pragma unroll
-    for (int a = 0; a < 8; a++)
-#pragma unroll
-      for (int b = 0; b < 8; b++) M[a][b] = fmaf(kj[a], uj[b], M[a][b]);
+    rank1_update(M, kj, uj);
   }
   LQ_BTICK(3);
 }
@@ -249,10 +258,10 @@ __device__ __forceinline__ void quantize_tile(const Params &p, const BoundarySme
                             ub[6] | (uint32_t)ub[7] << 16);
       *reinterpret_cast<uint4 *>(p.comp_u(bh) + h * D + 8 * t.tx) = pu;
     }
+    float nk[8];
 #pragma unroll
-    for (int a = 0; a < 8; a++)
-#pragma unroll
-      for (int b = 0; b < 8; b++) M[a][b] = fmaf(-kf[a], uf[b], M[a][b]);
+    for (int a = 0; a < 8; a++) nk[a] = -kf[a];
+    rank1_update(M, nk, uf);                                  // M -= k u^T with the stored values
   }
   LQ_BTICK(4);
   // a vanished component means nothing is left to fit: this and all later compensators are zero
