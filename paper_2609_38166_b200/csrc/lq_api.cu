@@ -115,7 +115,7 @@ __global__ void __launch_bounds__(256, 2) boundary_kernel(const Params p, const 
 // Baseline: Eq. 1 on a dense state that is read and written in full every token.
 // ---------------------------------------------------------------------------------------------
 template <int GATE, bool BF16>
-__global__ void __launch_bounds__(256, BF16 ? 3 : 2) ref_kernel(const Params p) {
+__global__ void __launch_bounds__(256, (BF16 || GATE == LQ_GATE_SCALAR) ? 3 : 2) ref_kernel(const Params p) {
   __shared__ __align__(16) float kt_s[D], q_s[D], bv_s[D], a_s[D], col_s[D], part_s[8 * D];
   const Tile t;
   const size_t bh = blockIdx.x;
