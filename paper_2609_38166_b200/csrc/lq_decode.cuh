@@ -93,6 +93,23 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t
                "l"(src), "r"(bytes), "r"(bar)
                : "memory");
 }
+// The same with an L2 eviction priority for the lines the copy brings in.
+__device__ __forceinline__ void bulk_g2s_hint(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;\n" ::"r"(dst),
+      "l"(src), "r"(bytes), "r"(bar), "l"(policy)
+      : "memory");
+}
+__device__ __forceinline__ uint64_t l2_stream_policy() {
+  uint64_t policy;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;\n" : "=l"(policy));
+  return policy;
+}
+__device__ __forceinline__ uint64_t l2_keep_policy() {
+  uint64_t policy;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;\n" : "=l"(policy));
+  return policy;
+}
 // Bounded wait for phase `parity`; false if the limit ran out (the caller then reports and bails out).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
   for (int spin = 0; spin < (1 << 20); spin++) {
@@ -244,17 +261,24 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
   // The regions the copies overwrite were only READ through ordinary loads, whose values have been used
   // before the call; the warps write only their scratch regions.  So nothing written by the generic proxy is
   // at stake and no cross-proxy fence is needed (it costs over a thousand cycles here).
-  auto request_head = [&](unsigned bh) {
+  // A head at its last free record (n == W - 1) goes through the window boundary right after this kernel, which
+  // reads the same head block and records again: its lines are asked to stay in the L2 until then.
+  const uint64_t keep = l2_keep_policy(), stream = l2_stream_policy();
+  auto request_head = [&](unsigned bh, int n) {
     if (lane == 0) {
       mbar_expect_tx(barA, head_bytes(r));
-      bulk_g2s(slot_a + L.head, p.head(bh), head_bytes(r), barA);
+      if (n == W - 1) bulk_g2s_hint(slot_a + L.head, p.head(bh), head_bytes(r), barA, keep);
+      else bulk_g2s_hint(slot_a + L.head, p.head(bh), head_bytes(r), barA, stream);
     }
   };
   auto request_records = [&](unsigned bh, int n) {
     if (lane == 0) {
       const uint32_t rb = static_cast<uint32_t>(sizeof(rec_t)) * RF * n;
       mbar_expect_tx(barR, rb);              // with no records the phase completes at once
-      if (n > 0) bulk_g2s(slot_a + L.rec, p.record<rec_t>(bh, 0, DIAG), rb, barR);
+      if (n > 0) {
+        if (n == W - 1) bulk_g2s_hint(slot_a + L.rec, p.record<rec_t>(bh, 0, DIAG), rb, barR, keep);
+        else bulk_g2s_hint(slot_a + L.rec, p.record<rec_t>(bh, 0, DIAG), rb, barR, stream);
+      }
     }
   };
   // Bounded wait for one of the two.  A copy that never lands must not hang the GPU: when the limit runs out the
@@ -295,7 +319,7 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
     const int n0 = __shfl_sync(FULL, sc_n, 0) & 0xFFFF;
     if (first < nh && wanted(n0)) {
       load_token<GATE>(p, hd, group, lane, role, nxt);
-      if (role == 0) request_head(first);
+      if (role == 0) request_head(first, n0);
       else request_records(first, n0);
     }
   }
@@ -319,7 +343,7 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
     if (!active) {                           // nothing was requested for this head; keep the pipeline going
       if (next_active) {
         load_token<GATE>(p, hd1, group, lane, role, nxt);
-        if (role == 0) request_head(bh_next);
+        if (role == 0) request_head(bh_next, n_next);
         else request_records(bh_next, n_next);
       }
       continue;
@@ -639,7 +663,7 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
           for (int e = 0; e < 4; e++) { rk[e] = fmaf(uc[e], pkh, rk[e]); rq[e] = fmaf(uc[e], pqh, rq[e]); }
         }
         __syncwarp();                        // nobody reads the head block any more (the dot warp finished with
-        if (next_active) request_head(bh_next);   // it before barrier 3): the next head's may land
+        if (next_active) request_head(bh_next, n_next);   // it before barrier 3): the next head's may land
         named_wait(bar0 + 1);                       // the record terms are complete
         {
           const float4 tk = *reinterpret_cast<const float4 *>(y + 4 * lane);
