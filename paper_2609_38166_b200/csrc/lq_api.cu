@@ -125,7 +125,7 @@ __global__ void __launch_bounds__(256, (BF16 || GATE == LQ_GATE_SCALAR) ? 3 : 2)
     const uint16_t *S = p.S16 + bh * (size_t)(D * D);
 #pragma unroll
     for (int a = 0; a < 8; a++) {
-      const uint4 w = *reinterpret_cast<const uint4 *>(S + (8 * t.ty + a) * D + 8 * t.tx);
+      const uint4 w = __ldcs(reinterpret_cast<const uint4 *>(S + (8 * t.ty + a) * D + 8 * t.tx));   // streamed: read once
       const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
       for (int e = 0; e < 4; e++) {
@@ -136,7 +136,7 @@ __global__ void __launch_bounds__(256, (BF16 || GATE == LQ_GATE_SCALAR) ? 3 : 2)
   } else {
     const float *S = p.S + bh * (size_t)(D * D);
 #pragma unroll
-    for (int a = 0; a < 8; a++) load8(S + (8 * t.ty + a) * D + 8 * t.tx, M[a]);
+    for (int a = 0; a < 8; a++) load8(S + (8 * t.ty + a) * D + 8 * t.tx, M[a]);   // (streaming hints slow this one down)
   }
   if (t.tid < D) {
     const int group = p.heads_v / p.heads_qk;
@@ -176,7 +176,7 @@ __global__ void __launch_bounds__(256, (BF16 || GATE == LQ_GATE_SCALAR) ? 3 : 2)
 #pragma unroll
       for (int e = 0; e < 4; e++)
         ws[e] = (uint32_t)to_bf16_bits(M[a][2 * e]) | ((uint32_t)to_bf16_bits(M[a][2 * e + 1]) << 16);
-      *reinterpret_cast<uint4 *>(S + (8 * t.ty + a) * D + 8 * t.tx) = make_uint4(ws[0], ws[1], ws[2], ws[3]);
+      __stcs(reinterpret_cast<uint4 *>(S + (8 * t.ty + a) * D + 8 * t.tx), make_uint4(ws[0], ws[1], ws[2], ws[3]));
     }
   } else {
     float *S = p.S + bh * (size_t)(D * D);

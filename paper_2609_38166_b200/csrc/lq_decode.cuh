@@ -100,16 +100,6 @@ __device__ __forceinline__ void bulk_g2s_hint(uint32_t dst, const void *src, uin
       "l"(src), "r"(bytes), "r"(bar), "l"(policy)
       : "memory");
 }
-__device__ __forceinline__ uint64_t l2_stream_policy() {
-  uint64_t policy;
-  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;\n" : "=l"(policy));
-  return policy;
-}
-__device__ __forceinline__ uint64_t l2_keep_policy() {
-  uint64_t policy;
-  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;\n" : "=l"(policy));
-  return policy;
-}
 // Bounded wait for phase `parity`; false if the limit ran out (the caller then reports and bails out).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
   for (int spin = 0; spin < (1 << 20); spin++) {
