@@ -50,7 +50,7 @@ def metric_name(wl) -> str:
 
 # DRAM bytes per launch from the ncu captures summarised under profiles/ (dram__bytes_read.sum +
 # dram__bytes_write.sum of one full-batch launch of the gdn_b256 workload, W = 16), or None when not captured.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"decode_kernel": 237.9e6, "boundary_kernel": 18.4e6}
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"decode_kernel": 235.0e6, "boundary_kernel": 18.4e6}
 
 
 def record_bytes(diag: bool, rec16: int) -> int:
