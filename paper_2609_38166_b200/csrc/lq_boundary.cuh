@@ -49,33 +49,26 @@ struct BoundarySmem {
 
 // Issue the asynchronous copies that bring head bh (its codes, scales, compensators and n records) into the
 // staging buffer of sm.  The caller commits the group and later waits for it.
-template <int GATE, bool R16, bool HINT = true>
+template <int GATE, bool R16>
 __device__ __forceinline__ void stage_issue(const Params &p, const BoundarySmem &sm, const Tile &t, size_t bh, int n) {
   constexpr bool DIAG = GATE == LQ_GATE_DIAG;
   constexpr int RF = record_floats(DIAG);
   const int r = p.r;
-  // HINT: the lines are read here for the last time before they are rewritten or dropped, and are marked evict-first
-  // in the L2.  (Not in the fused step kernel, which takes the plain copies.)
-  const uint64_t once = HINT ? l2_stream_policy() : 0;
-  auto copy16 = [&](void *dst, const void *src) {
-    if (HINT) cp_async16_hint(dst, src, once);
-    else cp_async16(dst, src);
-  };
   const uint8_t *hb = p.head(bh);
   for (int e = t.tid; e < D * D / 16; e += 256) {             // codes: 1024 chunks of 16 bytes
     const int v = e >> 3, q = e & 7;
-    copy16(sm.zt + v * D + 16 * (q ^ ((v >> 3) & 7)), hb + HB_CODES + 16 * e);
+    cp_async16(sm.zt + v * D + 16 * (q ^ ((v >> 3) & 7)), hb + HB_CODES + 16 * e);
   }
   if (R16) {                                                  // the n rows are one contiguous piece of fp16 values
     const __half *rec = p.record<__half>(bh, 0, DIAG);
-    for (int e = t.tid; e < n * (RF / 8); e += 256) copy16(sm.raw + 8 * e, rec + 8 * e);
+    for (int e = t.tid; e < n * (RF / 8); e += 256) cp_async16(sm.raw + 8 * e, rec + 8 * e);
   } else {
     const float *rec = p.record<float>(bh, 0, DIAG);
     for (int e = t.tid; e < n * (D / 4); e += 256) {
       const int j = e / (D / 4), q4 = 4 * (e % (D / 4));
-      copy16(sm.kd + j * D + q4, rec + j * RF + REC_KT + q4);
-      copy16(sm.bu + j * D + q4, rec + j * RF + REC_U + q4);
-      if (DIAG) copy16(sm.ba + j * D + q4, rec + j * RF + REC_A + q4);
+      cp_async16(sm.kd + j * D + q4, rec + j * RF + REC_KT + q4);
+      cp_async16(sm.bu + j * D + q4, rec + j * RF + REC_U + q4);
+      if (DIAG) cp_async16(sm.ba + j * D + q4, rec + j * RF + REC_A + q4);
     }
   }
   if (!DIAG && t.tid < n) cp_async4(sm.ba + t.tid, p.decays + bh * (size_t)p.W + t.tid);

@@ -77,11 +77,6 @@ __device__ __forceinline__ void cp_async16(void *smem, const void *gmem) {
   unsigned s = static_cast<unsigned>(__cvta_generic_to_shared(smem));
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem) : "memory");
 }
-// the same with an L2 eviction priority for the line it reads (a policy made by one of the functions below)
-__device__ __forceinline__ void cp_async16_hint(void *smem, const void *gmem, uint64_t policy) {
-  unsigned s = static_cast<unsigned>(__cvta_generic_to_shared(smem));
-  asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;\n" ::"r"(s), "l"(gmem), "l"(policy) : "memory");
-}
 // L2 eviction priorities: lines that will not be read again soon / lines another kernel reads next
 __device__ __forceinline__ uint64_t l2_stream_policy() {
   uint64_t policy;

@@ -37,7 +37,7 @@ __device__ __forceinline__ void fused_boundary_head(const Params &p, float *smem
   const BoundarySmem sm(smem, p.W, p.r, DIAG, R16, 0);
   const int b = static_cast<int>(bh / p.heads_v);
   float M[8][8];
-  stage_issue<GATE, R16, false>(p, sm, t, bh, n);
+  stage_issue<GATE, R16>(p, sm, t, bh, n);
   cp_async_commit();
   cp_async_wait_all();
   // (the 4-byte copies of the scalar gate's decays go through the L1, which may hold an older copy of the line)
