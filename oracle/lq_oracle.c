@@ -32,17 +32,25 @@
  * rounded, the others folded in with fmaf), and the two halves are added; the
  * block results are then added as a balanced binary tree over the block index
  * (neighbours first).  (Two interleaved chains per block are what a two-wide
- * fp32 fused multiply-add gives.)  Building the file
- * with -DLQO_WIDE replaces this by a plain left-to-right sum in binary64,
- * rounded once; comparing the two builds measures how much of any
- * disagreement is attributable to fp32 summation order.
+ * fp32 fused multiply-add gives.)  Two other builds of this file exist to
+ * measure what that choice and the fixed-point readout are worth:
+ *   -DLQO_WIDE   every such sum is taken left to right in binary64 and
+ *                rounded once (the fixed-point readout is kept);
+ *   -DLQO_PLAIN  the same, and the readout is the plain definition as well:
+ *                sum_i Z_ij x_i with x in binary32 as computed, no fixed-point
+ *                grid, accumulated left to right in binary64 together with
+ *                the compensator and record terms (records oldest first),
+ *                rounded once.  Same constants, same start vectors.
+ * A result of the defining build that differs from the PLAIN build's does
+ * so because of summation order and the fixed-point grid, nothing else.
  *
  * Parity status of the pieces (what pins each is listed in the tests):
  *   reference recurrence, windowed decode, reconstruction, quantizer,
  *   smoothing, rank-r fit as a Frobenius minimiser        : pinned
- *   the constants n_iter, the all-equal start vector, the 1e-30 zero guard,
- *   the 1e-6 smoothing floor, the summation tree, the 30-bit fixed-point
- *   grid of the readout vector                             : parity unpinned
+ *   the constants n_iter, the start vectors of the power iteration, the 1e-30
+ *   and 1e-6 guards of its orthonormalisation, the 1e-6 smoothing floor, the
+ *   summation tree, the 30-bit fixed-point grid of the readout vector,
+ *   the grouping of the readout's terms                    : parity unpinned
  *   (the paper fixes none of them; they are this build's definition).
  */
 #include <math.h>
@@ -52,6 +60,10 @@
 
 #ifdef _OPENMP
 #include <omp.h>
+#endif
+
+#if defined(LQO_PLAIN) && !defined(LQO_WIDE)
+#define LQO_WIDE
 #endif
 
 enum { LQO_GATE_SCALAR = 0, LQO_GATE_DIAG = 1 };
@@ -366,58 +378,114 @@ static void head_reconstruct(const lqo_shape *sh, const head_view *hv, int n, fl
 
 /* ------------------------------------------------------------------ */
 /* Window-boundary quantization of a dense state M (destroyed):        */
-/*   r Compensator Tokens, Eqs. 5-6, each the leading singular pair of  */
-/*   what is left, found by power iteration and removed with the values */
-/*   that are actually stored (fp16);                                   */
+/*   r Compensator Tokens, Eqs. 5-6: K~ U~^T is a rank-r fit of M in    */
+/*   the Frobenius norm, found by power iteration on all r vectors at   */
+/*   once and removed with the values that are actually stored (fp16);  */
 /*   smoothing scales c, Sec. 3.4 (square root of the row mean |.|);    */
 /*   per-value-channel symmetric 8-bit codes, Appendix B.3.             */
-/* The paper does not say where the power iteration starts.  Here the   */
-/* iteration for component h starts from the value side u of the        */
-/* (h+1)-th newest buffered record, scaled to unit length (the newest   */
-/* records dominate the state that is being fitted); where there is no  */
-/* such record, or it is (numerically) zero, from the vector with all   */
-/* entries equal.  `starts` holds `nstarts` rows of d_v floats, oldest  */
-/* first (the u part of the record buffer), or is NULL.                 */
 /* ------------------------------------------------------------------ */
-static void head_quantize(const lqo_shape *sh, float *M, const head_view *hv, const float *starts, int nstarts) {
-  int K = sh->d_k, V = sh->d_v;
-  float *w = (float *)malloc(sizeof(float) * V), *t = (float *)malloc(sizeof(float) * K);
-  float *col = (float *)malloc(sizeof(float) * K);
-  float *kf = (float *)malloc(sizeof(float) * K), *uf = (float *)malloc(sizeof(float) * V);
 
-  for (int h = 0; h < sh->r; h++) {
-    int vanished = 0;
-    for (int j = 0; j < V; j++) w[j] = 1.0f / sqrtf((float)V);
-    if (starts && h < nstarts) {
-      const float *u = starts + (size_t)(nstarts - 1 - h) * V;
-      float nu0 = lqo_csum_dot(u, u, V);
-      if (nu0 >= 1e-30f) {
-        float s0 = 1.0f / sqrtf(nu0);
-        for (int j = 0; j < V; j++) w[j] = u[j] * s0;
+/* Start vector h of the power iteration when no buffered record supplies one: entry j is -1 where j and h
+ * share an odd number of set bits, else +1 (the Walsh functions: h = 0 is the all-equal vector, different h
+ * are orthogonal).  Data-independent, so that the fit has one result per input. */
+static float walsh_entry(int h, int j) {
+  int x = h & j, odd = 0;
+  while (x) { odd ^= 1; x &= x - 1; }
+  return odd ? -1.0f : 1.0f;
+}
+
+/* Orthonormal basis Q of the span of the r vectors X[0..r-1] (each of length len), taken in order:
+ * q_h = (x_h - sum_{j<h} L_hj q_j) / L_hh with L the Cholesky factor of the Gram matrix X^T X.  One pass of
+ * dot products serves all r vectors.  A vector that is zero (squared length below 1e-30), or that the vectors
+ * before it span already (what is left of its squared length is not above 1e-6 of it: fp32 cannot tell such a
+ * remainder from rounding noise), gives q_h = 0 and alive[h] = 0. */
+static void orthonormalize(const float *X, int len, int r, float *Q, int *alive) {
+  float *G = (float *)malloc(sizeof(float) * (size_t)r * r), *L = (float *)calloc((size_t)r * r, sizeof(float));
+  float *inv = (float *)malloc(sizeof(float) * (size_t)r);
+  for (int a = 0; a < r; a++)
+    for (int b = 0; b <= a; b++) G[a * r + b] = lqo_csum_dot(X + (size_t)a * len, X + (size_t)b * len, len);
+  for (int h = 0; h < r; h++) {
+    for (int j = 0; j < h; j++) {
+      float s = G[h * r + j];
+      for (int m = 0; m < j; m++) s = fmaf(-L[h * r + m], L[j * r + m], s);
+      L[h * r + j] = s * inv[j];                          /* inv[j] = 0 for a vector that was dropped */
+    }
+    float d = G[h * r + h];
+    for (int m = 0; m < h; m++) d = fmaf(-L[h * r + m], L[h * r + m], d);
+    alive[h] = G[h * r + h] >= 1e-30f && d > 1e-6f * G[h * r + h];
+    inv[h] = alive[h] ? 1.0f / sqrtf(d) : 0.0f;
+  }
+  for (int i = 0; i < len; i++)
+    for (int h = 0; h < r; h++) {
+      float x = X[(size_t)h * len + i];
+      for (int j = 0; j < h; j++) x = fmaf(-L[h * r + j], Q[(size_t)j * len + i], x);
+      Q[(size_t)h * len + i] = x * inv[h];
+    }
+  free(G); free(L); free(inv);
+}
+
+/* The paper says the compensators are "fitted with power iteration" and no more.  Here all r vectors are iterated
+ * together (power iteration on a subspace): T = M W, orthonormalize; W = M^T T, orthonormalize; ... n_iter
+ * times, ending on the key side.  The columns of W start from the value sides u of the newest buffered records
+ * (column h from the (h+1)-th newest: they dominate the state that is being fitted), from Walsh vectors
+ * where there is no such record.  The key sides are then rounded to fp16, and value side h is the least-squares
+ * answer for what is left after components 0..h-1 as stored:
+ *   u_h = (M - sum_{a<h} k_a u_a^T)^T k_h = M^T k_h - sum_{a<h} u_a (k_a^T k_h),
+ * rounded to fp16 in turn.  `starts` holds `nstarts` rows of d_v floats, oldest first (the u part of the record
+ * buffer), or is NULL. */
+static void head_quantize(const lqo_shape *sh, float *M, const head_view *hv, const float *starts, int nstarts) {
+  int K = sh->d_k, V = sh->d_v, r = sh->r;
+  float *col = (float *)malloc(sizeof(float) * K);
+
+  if (r > 0) {
+    float *Wv = (float *)malloc(sizeof(float) * (size_t)r * V), *Xv = (float *)malloc(sizeof(float) * (size_t)r * V);
+    float *T = (float *)malloc(sizeof(float) * (size_t)r * K), *Q = (float *)malloc(sizeof(float) * (size_t)r * K);
+    float *kf = (float *)malloc(sizeof(float) * (size_t)r * K), *uf = (float *)malloc(sizeof(float) * (size_t)r * V);
+    float *g = (float *)malloc(sizeof(float) * (size_t)r * r);
+    int *alive = (int *)malloc(sizeof(int) * (size_t)r);
+    for (int h = 0; h < r; h++)
+      for (int j = 0; j < V; j++)
+        Wv[(size_t)h * V + j] = (starts && h < nstarts) ? starts[(size_t)(nstarts - 1 - h) * V + j] : walsh_entry(h, j);
+    for (int it = 0; it < sh->n_iter; it++) {
+      for (int h = 0; h < r; h++)
+        for (int i = 0; i < K; i++) T[(size_t)h * K + i] = lqo_csum_dot(M + (size_t)i * V, Wv + (size_t)h * V, V);   /* T = M W */
+      orthonormalize(T, K, r, Q, alive);
+      if (it + 1 < sh->n_iter) {
+        for (int j = 0; j < V; j++) {
+          column_of(M, K, V, j, col);
+          for (int h = 0; h < r; h++) Xv[(size_t)h * V + j] = lqo_csum_dot(col, Q + (size_t)h * K, K);                /* W = M^T T */
+        }
+        orthonormalize(Xv, V, r, Wv, alive);
       }
     }
-    for (int it = 0; it < sh->n_iter; it++) {
-      for (int i = 0; i < K; i++) t[i] = lqo_csum_dot(M + (size_t)i * V, w, V);      /* t = M w      */
-      float nu = lqo_csum_dot(t, t, K);
-      if (nu < 1e-30f) { vanished = 1; break; }
-      float rinv = 1.0f / sqrtf(nu);
-      for (int i = 0; i < K; i++) t[i] = t[i] * rinv;                                   /* unit length  */
-      if (it + 1 < sh->n_iter)
-        for (int j = 0; j < V; j++) { column_of(M, K, V, j, col); w[j] = lqo_csum_dot(col, t, K); } /* w = M^T t */
-    }
-    for (int i = 0; i < K; i++) {
-      uint16_t bits = vanished ? 0 : lqo_f32_to_f16(clamp_f16_range(t[i]));
-      hv->ck[(size_t)h * K + i] = bits;
-      kf[i] = lqo_f16_to_f32(bits);
-    }
+    /* key sides as stored */
+    for (int h = 0; h < r; h++)
+      for (int i = 0; i < K; i++) {
+        uint16_t bits = alive[h] ? lqo_f32_to_f16(clamp_f16_range(Q[(size_t)h * K + i])) : 0;
+        hv->ck[(size_t)h * K + i] = bits;
+        kf[(size_t)h * K + i] = lqo_f16_to_f32(bits);
+      }
+    for (int a = 0; a < r; a++)
+      for (int b = a + 1; b < r; b++) g[a * r + b] = lqo_csum_dot(kf + (size_t)a * K, kf + (size_t)b * K, K);
+    /* value sides */
     for (int j = 0; j < V; j++) {
-      uint16_t bits = 0;
-      if (!vanished) { column_of(M, K, V, j, col); bits = lqo_f32_to_f16(clamp_f16_range(lqo_csum_dot(col, kf, K))); }
-      hv->cu[(size_t)h * V + j] = bits;
-      uf[j] = lqo_f16_to_f32(bits);
+      column_of(M, K, V, j, col);
+      for (int h = 0; h < r; h++) {
+        float x = lqo_csum_dot(col, kf + (size_t)h * K, K);
+        for (int a = 0; a < h; a++) x = fmaf(-uf[(size_t)a * V + j], g[a * r + h], x);
+        uint16_t bits = alive[h] ? lqo_f32_to_f16(clamp_f16_range(x)) : 0;   /* a dropped component is all zero bits */
+        hv->cu[(size_t)h * V + j] = bits;
+        uf[(size_t)h * V + j] = lqo_f16_to_f32(bits);
+      }
     }
+    /* the residual R = M - K~ U~^T with the stored values */
     for (int i = 0; i < K; i++)
-      for (int j = 0; j < V; j++) M[(size_t)i * V + j] = fmaf(-kf[i], uf[j], M[(size_t)i * V + j]);
+      for (int j = 0; j < V; j++) {
+        float x = M[(size_t)i * V + j];
+        for (int h = 0; h < r; h++) x = fmaf(-kf[(size_t)h * K + i], uf[(size_t)h * V + j], x);
+        M[(size_t)i * V + j] = x;
+      }
+    free(Wv); free(Xv); free(T); free(Q); free(kf); free(uf); free(g); free(alive);
   }
 
   /* M is now the residual R.  Smooth the key rows, then quantize each value channel. */
@@ -442,7 +510,7 @@ static void head_quantize(const lqo_shape *sh, float *M, const head_view *hv, co
       hv->Z[(size_t)i * V + j] = (int8_t)z;
     }
   }
-  free(w); free(t); free(col); free(kf); free(uf);
+  free(col);
 }
 
 /* the boundary state without the 8-bit quantizer: the dense state itself, or (per-window BF16) each element
@@ -517,6 +585,28 @@ static void head_decode(const lqo_shape *sh, const head_view *hv, int n, const t
       rk = lqo_csum_dot(col, xk, K);
       rq = lqo_csum_dot(col, xq, K);
     } else {
+#ifdef LQO_PLAIN
+      /* Eq. 10 as it stands: (B/127) Z^T (C Gamma x) + Uc (Kc^T Gamma x) + sum_j u_j (kt_j^T Gamma x), one sum */
+      double ak = 0.0, aq = 0.0;
+      for (int i = 0; i < K; i++) {
+        ak += (double)hv->Z[(size_t)i * V + j] * (double)xk[i];
+        aq += (double)hv->Z[(size_t)i * V + j] * (double)xq[i];
+      }
+      ak *= (double)hv->B[j];
+      aq *= (double)hv->B[j];
+      for (int h = 0; h < r; h++) {
+        double uc = (double)lqo_f16_to_f32(hv->cu[(size_t)h * V + j]);
+        ak += uc * (double)ptk[h];
+        aq += uc * (double)ptq[h];
+      }
+      for (int jj = 0; jj < n; jj++) {
+        ak += (double)hv->bu[(size_t)jj * V + j] * (double)pk[jj];
+        aq += (double)hv->bu[(size_t)jj * V + j] * (double)pq[jj];
+      }
+      rk = (float)ak;
+      rq = (float)aq;
+      (void)Xk; (void)Xq; (void)back_k; (void)back_q;
+#else
       int64_t tk = 0, tq = 0;
       for (int i = 0; i < K; i++) {
         tk += (int64_t)hv->Z[(size_t)i * V + j] * Xk[i];
@@ -530,15 +620,21 @@ static void head_decode(const lqo_shape *sh, const head_view *hv, int n, const t
         rk = fmaf(uc, ptk[h], rk);
         rq = fmaf(uc, ptq[h], rq);
       }
+#endif
     }
-    /* the records' terms: their own sum, from the newest record back, added as one number */
-    float sk = 0.0f, sq = 0.0f;
-    for (int jj = n - 1; jj >= 0; jj--) {
-      sk = fmaf(hv->bu[(size_t)jj * V + j], pk[jj], sk);
-      sq = fmaf(hv->bu[(size_t)jj * V + j], pq[jj], sq);
+#ifdef LQO_PLAIN
+    if (hv->S0)
+#endif
+    {
+      /* the records' terms: their own sum, from the newest record back, added as one number */
+      float sk = 0.0f, sq = 0.0f;
+      for (int jj = n - 1; jj >= 0; jj--) {
+        sk = fmaf(hv->bu[(size_t)jj * V + j], pk[jj], sk);
+        sq = fmaf(hv->bu[(size_t)jj * V + j], pq[jj], sq);
+      }
+      rk = rk + sk;
+      rq = rq + sq;
     }
-    rk = rk + sk;
-    rq = rq + sq;
     u[j] = sh->delta ? t->v[j] - rk : t->v[j];   /* Eq. 3: u = v - S_{l-1}^T b, b = alpha (.) k or 0 */
     o[j] = fmaf(u[j], ktq, rq);          /* o = S_{l-1}^T (alpha (.) q) + u (kt^T q) */
   }

@@ -3,9 +3,11 @@
 Test infrastructure only: the tests, the smoke check and the benchmark's CPU
 baseline leg use it; the product path never imports it.  It compiles the C file
 with gcc on first use (``-O2 -ffp-contract=off -fopenmp``) and passes numpy
-arrays through ctypes.  Two builds exist: the defining one (fp32, fixed
-summation tree) and a "wide" one whose sums run left to right in binary64,
-used to measure what is attributable to fp32 summation order.
+arrays through ctypes.  Three builds exist: the defining one (fp32, fixed
+summation tree, fixed-point readout), a "wide" one whose sums run left to right
+in binary64, and a "plain" one that in addition takes the readout as the plain
+definition (no fixed-point grid); the last two measure what is attributable to
+fp32 summation order and to the grid.
 """
 from __future__ import annotations
 
@@ -25,7 +27,8 @@ GATE_DIAG = 1    # Kimi Delta Attention
 
 def build(force: bool = False) -> None:
     """Compile both oracle builds next to the source (no-op when up to date)."""
-    for name, extra in (("liblq_oracle.so", []), ("liblq_oracle_wide.so", ["-DLQO_WIDE"])):
+    for name, extra in (("liblq_oracle.so", []), ("liblq_oracle_wide.so", ["-DLQO_WIDE"]),
+                        ("liblq_oracle_plain.so", ["-DLQO_PLAIN"])):
         out = os.path.join(_HERE, name)
         if not force and os.path.exists(out) and os.path.getmtime(out) >= os.path.getmtime(_SRC):
             continue
@@ -114,9 +117,10 @@ def _chk(a: np.ndarray, dtype, shape=None) -> np.ndarray:
 
 
 class Oracle:
-    def __init__(self, wide: bool = False):
+    def __init__(self, wide: bool = False, plain: bool = False):
         build()
-        self.lib = C.CDLL(os.path.join(_HERE, "liblq_oracle_wide.so" if wide else "liblq_oracle.so"))
+        name = "liblq_oracle_plain.so" if plain else "liblq_oracle_wide.so" if wide else "liblq_oracle.so"
+        self.lib = C.CDLL(os.path.join(_HERE, name))
         L = self.lib
         L.lqo_csum_dot.restype = C.c_float
         L.lqo_csum_dot.argtypes = [C.c_void_p, C.c_void_p, C.c_int]

@@ -22,3 +22,9 @@ def oracle():
 def oracle_wide():
     from oracle.lq_oracle import Oracle
     return Oracle(wide=True)
+
+
+@pytest.fixture(scope="session")
+def oracle_plain():
+    from oracle.lq_oracle import Oracle
+    return Oracle(plain=True)

@@ -104,9 +104,12 @@ def test_recall_special_case_holds_with_quantization_on(oracle, gate):
 
 @pytest.mark.parametrize("gate", GATES)
 @pytest.mark.parametrize("dims", [(4, 4, 3, 1), (4, 4, 2, 2), (8, 16, 3, 2), (5, 3, 4, 1)])
-def test_brute_force_on_tiny_states(oracle, gate, dims):
+@pytest.mark.parametrize("build", ["defining", "plain"])
+def test_brute_force_on_tiny_states(oracle, oracle_plain, build, gate, dims):
     """Materialise the state densely before every token (Eq. 7 written out in float64 from the stored arrays),
-    apply the native update, and compare the token's output and the record it appends."""
+    apply the native update, and compare the token's output and the record it appends.  Both the defining build
+    (fixed summation tree, fixed-point readout) and the plain one (binary64 sums, no grid) must pass."""
+    oracle = oracle_plain if build == "plain" else oracle
     K, V, W, r = dims
     wl = synth.Workload("t", 2, 2, 2, K, V, W=W, r=r, gate=gate, seed=15)
     sh = _shape(wl)
@@ -195,6 +198,73 @@ def test_boundary_term_is_exact_up_to_the_fixed_point_grid(oracle):
             got = v - st.buf_u[b, h, 0].astype(np.float64)
             grid = 2.0 ** -29 * 2 * np.abs(x).max() * np.abs(Z).sum(axis=0) * s
             assert np.all(np.abs(got - exact) <= grid + 3 * 2.0 ** -24 * (np.abs(exact) + np.abs(v)))
+
+
+def _grid_probe(oracle, tail):
+    """u of one token against a hand-made state: codes Z[1][j] = j - 64 (else 0), step 1, c = 1, alpha = beta = 1,
+    v = 0 and key (1, tail, 0, ...): u_j = -(j - 64) * tail-as-the-readout-sees-it."""
+    sh = Shape(1, 1, 1, 128, 128, 4, 0, 1, synth.GATE_SCALAR, 0)
+    st = State(sh)
+    st.codes[0, 0, 1, :] = np.arange(128) - 64
+    st.col_scale[...] = 1.0
+    k = np.zeros((1, 1, 128), np.float32); k[0, 0, 0] = 1.0; k[0, 0, 1] = tail
+    kb = synth.f32_to_bf16_bits(k)
+    assert np.array_equal(synth.bf16_bits_to_f32(kb), k)          # the probe values are bfloat16 numbers
+    one = synth.f32_to_bf16_bits(np.ones((1, 1), np.float32))
+    zero_v = synth.f32_to_bf16_bits(np.zeros((1, 1, 128), np.float32))
+    oracle.decode_step(sh, st, kb, kb, zero_v, one, one)
+    return -st.buf_u[0, 0, 0].astype(np.float64) / (np.arange(128) - 64 + 1e-300)
+
+
+def test_fixed_point_grid_is_thirty_bits_below_the_bound(oracle, oracle_plain):
+    """The readout vector is rounded to multiples of 2^(e-29), 2^e <= max|x| < 2^(e+1), ties to even.  With
+    max|x| = 1 a second entry of 2^-29 must pass through exactly (a 28-bit grid would lose it), 2^-30 is a tie
+    that goes to zero and 3 * 2^-30 a tie that goes to 2^-28 (a finer grid would keep both).  The plain build
+    has no grid and returns all three as they are."""
+    for tail, on_grid in ((2.0 ** -29, 2.0 ** -29), (2.0 ** -30, 0.0), (3 * 2.0 ** -30, 2.0 ** -28)):
+        seen = _grid_probe(oracle, tail)
+        seen_plain = _grid_probe(oracle_plain, tail)
+        keep = np.arange(128) != 64
+        assert np.all(seen[keep] == on_grid), (tail, seen[:3])
+        assert np.all(seen_plain[keep] == tail), (tail, seen_plain[:3])
+
+
+@pytest.mark.parametrize("gate", GATES)
+def test_defining_build_agrees_with_the_plain_definition_along_a_chain(oracle, oracle_plain, gate):
+    """What the fixed summation tree and the fixed-point readout cost against the plain definition, measured
+    on the CPU with both builds started from the same state at every token (so that differences do not
+    compound): outputs and records within 1e-3 relative / 1e-5 absolute; after a boundary, heads whose fp16
+    compensators came out identical differ by at most one code step on at most 0.01 % of the entries."""
+    wl = synth.Workload("t", 2, 4, 2, 128, 128, W=8, r=4, gate=gate, seed=71)
+    sh = _shape(wl)
+    st = State(sh)
+    oracle.quantize_state(sh, synth.dense_states(wl, 3), st)
+    same_heads = diff_entries = entries = 0
+    for step in range(3 * wl.W):
+        tok = synth.token_inputs(wl, step)
+        st_p = State(sh)
+        for name in ("codes", "col_scale", "row_smooth", "comp_k", "comp_u", "buf_k", "buf_u", "buf_a", "win_pos"):
+            getattr(st_p, name)[...] = getattr(st, name)
+        o = oracle.decode_step(sh, st, **tok)
+        o_p = oracle_plain.decode_step(sh, st_p, **tok)
+        assert np.allclose(o, o_p, rtol=1e-3, atol=1e-5), step
+        assert np.array_equal(st.win_pos, st_p.win_pos)
+        if st.win_pos[0] != 0:
+            n = st.win_pos[0] - 1
+            assert np.allclose(st.buf_u[:, :, n], st_p.buf_u[:, :, n], rtol=1e-3, atol=1e-5)
+            continue
+        for b in range(wl.batch):
+            for h in range(wl.heads_v):
+                if not (np.array_equal(st.comp_k[b, h], st_p.comp_k[b, h]) and
+                        np.array_equal(st.comp_u[b, h], st_p.comp_u[b, h])):
+                    continue
+                same_heads += 1
+                d = np.abs(st.codes[b, h].astype(int) - st_p.codes[b, h].astype(int))
+                assert d.max() <= 1
+                diff_entries += int((d > 0).sum()); entries += d.size
+                assert np.allclose(st.col_scale[b, h], st_p.col_scale[b, h], rtol=1e-3, atol=1e-5)
+                assert np.allclose(st.row_smooth[b, h], st_p.row_smooth[b, h], rtol=1e-3, atol=1e-5)
+    assert same_heads > 0 and diff_entries <= 1e-4 * entries, (same_heads, diff_entries, entries)
 
 
 @pytest.mark.parametrize("gate", GATES)
