@@ -23,10 +23,12 @@
  *  - Errors are reported through the return value; nothing aborts or throws.
  *    Argument errors are detected before anything is enqueued.
  *  - Arithmetic is IEEE binary32.  Sums over a channel index are taken in a
- *    fixed order (blocks of eight consecutive terms accumulated left to right
- *    with fused multiply-add, block results combined as a balanced binary
- *    tree over the block index), so results do not depend on the launch
- *    configuration and are reproducible bit for bit.
+ *    fixed order (blocks of eight consecutive terms; inside a block the
+ *    even-numbered and the odd-numbered terms are two chains of fused
+ *    multiply-adds that are added at the end; block results combined as a
+ *    balanced binary tree over the block index, neighbours first), and the
+ *    code-matrix term of the readout is an exact integer sum, so results do
+ *    not depend on the launch configuration and are reproducible bit for bit.
  *  - Supported shapes: d_k = d_v = 128, 1 <= W <= 64, 0 <= r <= 16,
  *    n_iter >= 1, heads_v a multiple of heads_qk.  Anything else returns
  *    LQ_ERR_UNSUPPORTED.
@@ -65,10 +67,11 @@ typedef struct {
   int d_k, d_v; /* state is d_k x d_v                                             */
   int W;        /* window length (the paper's p)                                  */
   int r;        /* Compensator Tokens per state                                   */
-  int n_iter;   /* power-iteration steps per Compensator Token at a boundary (2 is  */
-                /* the default of the binding); compensator h starts from the u of  */
-                /* the (h+1)-th newest buffered record, scaled to unit length, or   */
-                /* from the all-equal unit vector where there is no such record     */
+  int n_iter;   /* rounds of the power iteration at a boundary (1 is the default of */
+                /* the binding).  All r vectors are iterated together: T = S W,     */
+                /* orthonormalise, W = S^T T, orthonormalise, ...; column h of W    */
+                /* starts from the u of the (h+1)-th newest buffered record, or     */
+                /* from Walsh function h where there is no such record              */
   int gate;     /* lq_gate                                                        */
   int smooth;   /* 1: residual smoothing (Sec. 3.4); 0: c = 1 (ablation)          */
   int delta;    /* 1: delta rule, the correction reads the state back with          */

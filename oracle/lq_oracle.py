@@ -57,7 +57,7 @@ class Shape:
     d_v: int
     W: int
     r: int = 4
-    n_iter: int = 2
+    n_iter: int = 1
     gate: int = GATE_SCALAR
     smooth: int = 1
     delta: int = 1

@@ -1,6 +1,6 @@
 // Window-boundary work on one 128x128 state held as 8x8 register tiles by a CTA of 256 threads:
 // reconstruction of the dense state from the window representation (Eq. 7) and its quantization
-// (Compensator-Token fit by power iteration with deflation, Eqs. 5-6; residual smoothing, Sec. 3.4;
+// (Compensator-Token fit by power iteration on all r vectors at once, Eqs. 5-6; residual smoothing, Sec. 3.4;
 // per-value-channel symmetric 8-bit codes, Appendix B.3).
 #pragma once
 #include "lq_common.cuh"
@@ -14,10 +14,12 @@ struct BoundarySmem {
   // fixed part
   float *ck;     // [r][128]  compensator keys widened to fp32
   float *cu;     // [r][128]  compensator values widened to fp32
-  float *vec;    // [128]     row-sum results (t of the power iteration, row mean-abs)
-  float *colv;   // [128]     column-sum results
-  float *part;   // [8][128]  per-warp column partial sums
+  float *vec;    // [128]     row-sum results (row mean-abs)
+  float *colv;   // [128]     1 / c
+  float *part;   // [8][2][128] per-warp column partial sums of two vectors (column maxima: [8][128])
   float *gam;    // [128]     Gamma_{1:n}
+  float *gram;   // [16][16]  Gram matrix of the vectors being orthonormalised (lower triangle), later K^T K
+  float *chol;   // [16][16]  its Cholesky factor L (strictly lower triangle), then [16] 1 / L_hh, [16] alive flags
   // staging buffer `buf`
   float *kd;     // [W][128]  buffered write keys, turned in place into Gamma_{j+1:n} kt_j
   float *bu;     // [W][128]  buffered corrections u_j
@@ -28,12 +30,15 @@ struct BoundarySmem {
   uint16_t *cuh; // [r][128]  compensator values as stored
   uint8_t *zt;   // [128][128] codes Z^T, 16-byte chunk q of row v stored at chunk q ^ ((v >> 3) & 7)
   __half *raw;   // fp16 records only: [W] rows as stored (kt | u | (alpha)), widened into kd, bu by the decay scan
-  __host__ __device__ static constexpr int fixed_floats(int r) { return 2 * r * D + 11 * D; }
+  __host__ __device__ static constexpr int fixed_floats(int r) {
+    return 2 * r * D + 19 * D + 2 * MAX_R * MAX_R + 2 * MAX_R;
+  }
   __host__ __device__ static constexpr int stage_floats(int W, int r, bool diag, bool rec16) {
     return 2 * W * D + (diag ? W * D : MAX_W) + 2 * D + r * D + D * D / 4 + (rec16 ? W * record_floats(diag) / 2 : 0);
   }
   __device__ __forceinline__ BoundarySmem(float *base, int W, int r, bool diag, bool rec16, int buf) {
-    ck = base; cu = ck + r * D; vec = cu + r * D; colv = vec + D; part = colv + D; gam = part + 8 * D;
+    ck = base; cu = ck + r * D; vec = cu + r * D; colv = vec + D; part = colv + D; gam = part + 16 * D;
+    gram = gam + D; chol = gram + MAX_R * MAX_R;
     kd = base + fixed_floats(r) + buf * stage_floats(W, r, diag, rec16);
     bu = kd + W * D; ba = bu + W * D; cs = ba + (diag ? W * D : MAX_W); ss = cs + D;
     ckh = reinterpret_cast<uint16_t *>(ss + D); cuh = ckh + r * D;
@@ -178,97 +183,229 @@ __device__ __forceinline__ void reconstruct_tile(const Params &p, const Boundary
   LQ_BTICK(3);
 }
 
+// ---- pieces of the Compensator-Token fit: power iteration on all r vectors at once ----
+
+// Entry j of start vector h where no buffered record supplies one: -1 where h and j share an odd number of bits
+__device__ __forceinline__ float walsh_entry(int h, int j) { return (__popc(h & j) & 1) ? -1.0f : 1.0f; }
+
+// Lower triangle of the Gram matrix of the nv vectors X[0..nv-1] (rows of 128 floats in shared memory), one dot
+// product per half-warp and trip.  Barrier before (X complete) and after (G complete) are the caller's.
+__device__ __forceinline__ void gram_lower(const float *X, int nv, float *G, const Tile &t, bool with_diagonal) {
+  const int hw = t.tid >> 4, c = t.lane & 15;
+  const int npairs = with_diagonal ? nv * (nv + 1) / 2 : nv * (nv - 1) / 2;
+  for (int base = 0; base < npairs; base += 16) {            // the same trip count for every thread of the CTA
+    const int idx = base + hw;
+    const int ii = idx < npairs ? idx : 0;
+    int a = 0;                                               // ii = a (a + 1) / 2 + b with b <= a, without a loop
+#pragma unroll
+    for (int e = 1; e < MAX_R; e++) a += ii >= e * (e + 1) / 2;
+    int b = ii - a * (a + 1) / 2;
+    if (!with_diagonal) a += 1;                              // pairs b < a only
+    const float d = dot128_shared(X + a * D, X + b * D, c);
+    if (idx < npairs && c == 0) G[a * MAX_R + b] = d;
+  }
+}
+
+// Cholesky factor of the Gram matrix, by one thread: L (strictly lower part), inv[h] = 1 / L_hh, alive[h].
+// A vector whose squared length is below 1e-30, or of which the vectors before it leave no more than 1e-6 of its
+// squared length, is dropped: inv = 0, which makes its orthonormalised vector and all its L entries zero.
+// Up to four vectors are handled in registers (all loads first, then arithmetic only); more go through shared memory.
+__device__ __forceinline__ void cholesky_lower(const float *G, int nv, float *L) {
+  float *inv = L + MAX_R * MAX_R, *alive = inv + MAX_R;
+  if (nv <= 4) {
+    float g[4][4], l[4][4], iv[4];
+#pragma unroll
+    for (int h = 0; h < 4; h++)
+#pragma unroll
+      for (int j = 0; j <= h; j++) g[h][j] = h < nv ? G[h * MAX_R + j] : 0.0f;
+#pragma unroll
+    for (int h = 0; h < 4; h++) {
+#pragma unroll
+      for (int j = 0; j < h; j++) {
+        float sacc = g[h][j];
+#pragma unroll
+        for (int m = 0; m < j; m++) sacc = fmaf(-l[h][m], l[j][m], sacc);
+        l[h][j] = sacc * iv[j];
+      }
+      float d = g[h][h];
+#pragma unroll
+      for (int m = 0; m < h; m++) d = fmaf(-l[h][m], l[h][m], d);
+      const bool ok = g[h][h] >= 1e-30f && d > 1e-6f * g[h][h];
+      iv[h] = ok ? 1.0f / sqrtf(d) : 0.0f;
+      if (h < nv) {
+#pragma unroll
+        for (int j = 0; j < h; j++) L[h * MAX_R + j] = l[h][j];
+        inv[h] = iv[h];
+        alive[h] = ok ? 1.0f : 0.0f;
+      }
+    }
+    return;
+  }
+  for (int h = 0; h < nv; h++) {
+    for (int j = 0; j < h; j++) {
+      float sacc = G[h * MAX_R + j];
+      for (int m = 0; m < j; m++) sacc = fmaf(-L[h * MAX_R + m], L[j * MAX_R + m], sacc);
+      L[h * MAX_R + j] = sacc * inv[j];
+    }
+    const float ghh = G[h * MAX_R + h];
+    float d = ghh;
+    for (int m = 0; m < h; m++) d = fmaf(-L[h * MAX_R + m], L[h * MAX_R + m], d);
+    const bool ok = ghh >= 1e-30f && d > 1e-6f * ghh;
+    inv[h] = ok ? 1.0f / sqrtf(d) : 0.0f;
+    alive[h] = ok ? 1.0f : 0.0f;
+  }
+}
+
+// Orthonormalise the nv vectors X (rows of 128 floats in shared memory) in place, in order:
+// q_h = (x_h - sum_{j<h} L_hj q_j) / L_hh, one thread per element index (it reads back the q_j it wrote).
+// With FINAL the results are then rounded to fp16 (what is stored as compensator keys), written to comp_k of
+// head bh and kept in X as the stored values.  Begins and ends with a barrier.
+template <bool FINAL>
+__device__ __forceinline__ void orthonormalize(const Params &p, const BoundarySmem &sm, const Tile &t, float *X,
+                                               int nv, size_t bh) {
+  __syncthreads();
+  gram_lower(X, nv, sm.gram, t, true);
+  __syncthreads();
+  if (t.tid == 0) cholesky_lower(sm.gram, nv, sm.chol);
+  __syncthreads();
+  if (t.tid < D) {
+    const float *L = sm.chol, *inv = L + MAX_R * MAX_R, *alive = inv + MAX_R;
+    const int i = t.tid;
+    for (int h = 0; h < nv; h++) {
+      float x = X[h * D + i];
+      for (int j = 0; j < h; j++) x = fmaf(-L[h * MAX_R + j], X[j * D + i], x);
+      X[h * D + i] = x * inv[h];
+    }
+    if (FINAL) {
+      for (int h = 0; h < nv; h++) {
+        const uint16_t bits = alive[h] != 0.0f ? to_f16_bits_sat(X[h * D + i]) : static_cast<uint16_t>(0);
+        p.comp_k(bh)[h * D + i] = bits;
+        X[h * D + i] = f16_bits(bits);
+      }
+    }
+  }
+  __syncthreads();
+}
+
+// T[h] = M w_h for the nv vectors w_h (two at a time), into Tm (rows of 128 floats).  `wsrc(h, w)` loads the eight
+// entries of w_h for this thread's columns.  No barrier inside.
+template <typename WSrc>
+__device__ __forceinline__ void rows_times_vectors(const float (&M)[8][8], const Tile &t, int nv, float *Tm, WSrc wsrc) {
+  for (int h0 = 0; h0 < nv; h0 += 2) {
+    const bool two = h0 + 1 < nv;
+    float w0[8], w1[8], pr0[8], pr1[8];
+    wsrc(h0, w0);
+    wsrc(two ? h0 + 1 : h0, w1);
+    row_blocks(M, w0, pr0);
+    row_blocks(M, w1, pr1);
+    int sel;
+    const float t0 = row_tree(pr0, t.lane, sel);
+    const float t1 = row_tree(pr1, t.lane, sel);
+    if (t.tx < 8) {
+      Tm[h0 * D + 8 * t.ty + sel] = t0;
+      if (two) Tm[(h0 + 1) * D + 8 * t.ty + sel] = t1;
+    }
+  }
+}
+
+// Out[h] = M^T x_h for the nv vectors x_h in Xm (rows of 128 floats in shared memory), two at a time.
+// Column sums in the fixed order: this thread's eight rows, its neighbour in the warp (lane ^ 16), then the
+// eight warps as a balanced tree.  Begins after a barrier of the caller (Xm complete); ends with a barrier.
+__device__ __forceinline__ void columns_times_vectors(const float (&M)[8][8], const BoundarySmem &sm, const Tile &t,
+                                                      int nv, const float *Xm, float *Out) {
+  const bool up = t.lane & 16;
+  for (int h0 = 0; h0 < nv; h0 += 2) {
+    const bool two = h0 + 1 < nv;
+    float x0[8], x1[8], pc0[8], pc1[8];
+    load8(Xm + h0 * D + 8 * t.ty, x0);
+    load8(Xm + (two ? h0 + 1 : h0) * D + 8 * t.ty, x1);
+    col_blocks(M, x0, pc0);
+    col_blocks(M, x1, pc1);
+    float r0[4], r1[4];
+#pragma unroll
+    for (int e = 0; e < 4; e++) {
+      const float keep0 = up ? pc0[e + 4] : pc0[e], send0 = up ? pc0[e] : pc0[e + 4];
+      const float keep1 = up ? pc1[e + 4] : pc1[e], send1 = up ? pc1[e] : pc1[e + 4];
+      r0[e] = keep0 + __shfl_xor_sync(FULL, send0, 16);
+      r1[e] = keep1 + __shfl_xor_sync(FULL, send1, 16);
+    }
+    if (h0 > 0) __syncthreads();                              // the previous pair's partial sums have been read
+    float *part = sm.part + t.warp * 2 * D + 8 * t.tx + (up ? 4 : 0);
+    *reinterpret_cast<float4 *>(part) = make_float4(r0[0], r0[1], r0[2], r0[3]);
+    *reinterpret_cast<float4 *>(part + D) = make_float4(r1[0], r1[1], r1[2], r1[3]);
+    __syncthreads();
+    {
+      const int v = t.tid >> 7, col = t.tid & (D - 1);
+      const float *c = sm.part + v * D + col;
+      const float sum = ((c[0] + c[2 * D]) + (c[4 * D] + c[6 * D])) + ((c[8 * D] + c[10 * D]) + (c[12 * D] + c[14 * D]));
+      if (v == 0 || two) Out[(h0 + v) * D + col] = sum;
+    }
+  }
+  __syncthreads();
+}
+
 // Quantize the dense state held in M (destroyed) and write codes, scales and compensators of head bh.
-// Uses sm.vec and sm.part; begins with a barrier so that it may follow any other use of shared memory.
-// The power iteration of compensator h starts from the value side u of the (h+1)-th newest of the n records in
-// sm.bu, scaled to unit length; from the all-equal unit vector where there is no such record or it is zero.
+// Uses the fixed part of shared memory (ck, cu, vec, colv, part, gram, chol); begins with a barrier so that it
+// may follow any other use of it.
+// Compensator Tokens (Eqs. 5-6): power iteration on all r vectors at once.  T = M W, orthonormalise, W = M^T T,
+// orthonormalise, ... n_iter times, ending on the key side; column h of W starts from the value side u of the
+// (h+1)-th newest of the n records in sm.bu, from a Walsh vector where there is no such record.  The keys are
+// rounded to fp16; value side h is M^T k_h - sum_{a<h} u_a (k_a^T k_h) with the stored values (the least-squares
+// answer for what components 0..h-1 leave), rounded to fp16 in turn; then M -= K U^T with the stored values.
 __device__ __forceinline__ void quantize_tile(const Params &p, const BoundarySmem &sm, const Tile &t, size_t bh,
                                               int n, float (&M)[8][8]) {
   const int r = p.r;
   __syncthreads();
-  // The scales 1 / |u| of all start vectors at once, one per group of sixteen lanes (they depend on the records
-  // only; taken one by one inside the loop each would cost a reduction and a reciprocal square root of latency).
-  // 0 marks "no such record, or a zero one": start from the all-equal vector.  Kept in sm.gam, which is free now.
-  float *start_scale = sm.gam;
-  {
-    // (every thread takes part in the warp-wide reduction, whatever r and n: groups without a record of
-    // their own reduce record 0 and drop the result)
-    const int g16 = t.tid >> 4;                               // r <= 16 = the number of groups
-    const bool mine = g16 < r && g16 < n;
-    const float *u = sm.bu + (mine ? n - 1 - g16 : 0) * D;
-    const float nu0 = dot128_shared(u, u, t.lane & 15);
-    const float s0 = mine && nu0 >= 1e-30f ? 1.0f / sqrtf(nu0) : 0.0f;
-    if (g16 < r && (t.lane & 15) == 0) start_scale[g16] = s0;
-  }
-  __syncthreads();
-  int h = 0;
-  for (; h < r; h++) {
-    float w[8], tn[8];
-    const float w0 = 1.0f / sqrtf(static_cast<float>(D));
-#pragma unroll
-    for (int b = 0; b < 8; b++) w[b] = w0;
-    {
-      const float s0 = start_scale[h];
-      if (s0 != 0.0f) {
-        load8(sm.bu + (n - 1 - h) * D + 8 * t.tx, w);
-#pragma unroll
-        for (int b = 0; b < 8; b++) w[b] = w[b] * s0;
-      }
-    }
-    bool vanished = false;
+  if (r > 0) {
+    float *Tm = sm.ck, *Wm = sm.cu;                           // [r][128] each; the old compensators are done with
     for (int it = 0; it < p.n_iter; it++) {
-      float pr[8];
-      row_blocks(M, w, pr);                                   // t = M w
-      int sel;
-      const float tv = row_tree(pr, t.lane, sel);
-      if (t.tx < 8) sm.vec[8 * t.ty + sel] = tv;
-      __syncthreads();
-      const float nu = dot128_shared(sm.vec, sm.vec, t.lane & 15);
-      if (nu < 1e-30f) { vanished = true; break; }            // same value in every thread
-      const float rinv = 1.0f / sqrtf(nu);
-      load8(sm.vec + 8 * t.ty, tn);
+      if (it == 0) {
+        rows_times_vectors(M, t, r, Tm, [&](int h, float (&w)[8]) {
+          if (h < n) {
+            load8(sm.bu + (n - 1 - h) * D + 8 * t.tx, w);
+          } else {
 #pragma unroll
-      for (int a = 0; a < 8; a++) tn[a] = tn[a] * rinv;
+            for (int b = 0; b < 8; b++) w[b] = walsh_entry(h, 8 * t.tx + b);
+          }
+        });
+      } else {
+        rows_times_vectors(M, t, r, Tm, [&](int h, float (&w)[8]) { load8(Wm + h * D + 8 * t.tx, w); });
+      }
+      LQ_BTICK(10);
       if (it + 1 < p.n_iter) {
-        float pc[8];
-        col_blocks(M, tn, pc);                                // w = M^T t
-        col_tree(pc, sm.part, sm.colv, t, w);
+        orthonormalize<false>(p, sm, t, Tm, r, bh);
+        columns_times_vectors(M, sm, t, r, Tm, Wm);
+        orthonormalize<false>(p, sm, t, Wm, r, bh);
       }
     }
-    if (vanished) break;
-    // store the key side in fp16 and continue with the stored values
-    float kf[8], uf[8];
-    uint16_t kb[8], ub[8];
-#pragma unroll
-    for (int a = 0; a < 8; a++) { kb[a] = to_f16_bits_sat(tn[a]); kf[a] = f16_bits(kb[a]); }
-    {
-      float pc[8], uraw[8];
-      col_blocks(M, kf, pc);                                  // value side = M^T k
-      col_tree(pc, sm.part, sm.colv, t, uraw);
-#pragma unroll
-      for (int b = 0; b < 8; b++) { ub[b] = to_f16_bits_sat(uraw[b]); uf[b] = f16_bits(ub[b]); }
+    orthonormalize<true>(p, sm, t, Tm, r, bh);                // Tm now holds the keys as stored
+    LQ_BTICK(11);
+    gram_lower(Tm, r, sm.gram, t, false);                     // k_a^T k_h, a < h, in gram[h][a]
+    columns_times_vectors(M, sm, t, r, Tm, Wm);               // M^T k_h (its barriers also publish gram)
+    LQ_BTICK(13);
+    if (t.tid < D) {
+      const float *alive = sm.chol + MAX_R * MAX_R + MAX_R;
+      const int j = t.tid;
+      for (int h = 0; h < r; h++) {                           // (reads back the stored values u_a it wrote)
+        float x = Wm[h * D + j];
+        for (int a = 0; a < h; a++) x = fmaf(-Wm[a * D + j], sm.gram[h * MAX_R + a], x);
+        const uint16_t bits = alive[h] != 0.0f ? to_f16_bits_sat(x) : static_cast<uint16_t>(0);
+        p.comp_u(bh)[h * D + j] = bits;
+        Wm[h * D + j] = f16_bits(bits);
+      }
     }
-    if (t.tx == 0) {
-      uint4 pk = make_uint4(kb[0] | (uint32_t)kb[1] << 16, kb[2] | (uint32_t)kb[3] << 16, kb[4] | (uint32_t)kb[5] << 16,
-                            kb[6] | (uint32_t)kb[7] << 16);
-      *reinterpret_cast<uint4 *>(p.comp_k(bh) + h * D + 8 * t.ty) = pk;
-    }
-    if (t.ty == 0) {
-      uint4 pu = make_uint4(ub[0] | (uint32_t)ub[1] << 16, ub[2] | (uint32_t)ub[3] << 16, ub[4] | (uint32_t)ub[5] << 16,
-                            ub[6] | (uint32_t)ub[7] << 16);
-      *reinterpret_cast<uint4 *>(p.comp_u(bh) + h * D + 8 * t.tx) = pu;
-    }
-    float nk[8];
+    __syncthreads();
+    LQ_BTICK(14);
+    for (int h = 0; h < r; h++) {                             // M -= k u^T with the stored values
+      float kf[8], uf[8], nk[8];
+      load8(Tm + h * D + 8 * t.ty, kf);
+      load8(Wm + h * D + 8 * t.tx, uf);
 #pragma unroll
-    for (int a = 0; a < 8; a++) nk[a] = -kf[a];
-    rank1_update(M, nk, uf);                                  // M -= k u^T with the stored values
+      for (int a = 0; a < 8; a++) nk[a] = -kf[a];
+      rank1_update(M, nk, uf);
+    }
   }
   LQ_BTICK(4);
-  // a vanished component means nothing is left to fit: this and all later compensators are zero
-  for (; h < r; h++) {
-    if (t.tx == 0) *reinterpret_cast<uint4 *>(p.comp_k(bh) + h * D + 8 * t.ty) = make_uint4(0, 0, 0, 0);
-    if (t.ty == 0) *reinterpret_cast<uint4 *>(p.comp_u(bh) + h * D + 8 * t.tx) = make_uint4(0, 0, 0, 0);
-  }
 
   // residual smoothing: c_i = max(sqrt(mean_j |R_ij|), 1e-6)
   float c[8];

@@ -43,7 +43,7 @@ class Workload:
     d_v: int = 128
     W: int = 16
     r: int = 4
-    n_iter: int = 2
+    n_iter: int = 1
     gate: int = GATE_SCALAR
     smooth: int = 1
     delta: int = 1                  # 1: delta rule (GDN, KDA); 0: no read-back, u = v (Mamba2, GLA, ...)
