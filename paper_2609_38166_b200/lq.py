@@ -241,9 +241,10 @@ def quantize_state(sh: Shape, S, st: State, stream=None, b0: int = 0, nb: Option
     _check(lib().lq_quantize_state(C.byref(s), _ptr(S, b0), C.byref(cs), _stream(stream)), "lq_quantize_state")
 
 
-def dequantize_state(sh: Shape, st: State, S, stream=None):
-    s = sh.c()
-    cs = st.c()
+def dequantize_state(sh: Shape, st: State, S, stream=None, b0: int = 0, nb: Optional[int] = None):
+    """lq_dequantize_state on sequences [b0, b0+nb) of the state; ``S`` receives exactly those sequences."""
+    s = _sub(sh, b0, nb).c()
+    cs = st.c(b0)
     _check(lib().lq_dequantize_state(C.byref(s), C.byref(cs), _ptr(S), _stream(stream)), "lq_dequantize_state")
 
 
