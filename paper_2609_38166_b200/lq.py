@@ -100,15 +100,24 @@ class State:
     ``decays`` (scalar gate) and ``win_pos``.  The named pieces (codes, col_scale, row_smooth, comp_k,
     comp_u, buf_k, buf_u, buf_a) are strided views into those tensors."""
 
-    def __init__(self, sh: Shape, device="cuda"):
+    def __init__(self, sh: Shape, device="cuda", storage=None):
+        """``storage``: optionally the four tensors (heads, records, decays, win_pos) to use instead of fresh
+        ones - contiguous, of the shapes and dtypes below (callers that place the state in memory of their own)."""
         B, H, K, V, W, r = sh.batch, sh.heads_v, sh.d_k, sh.d_v, sh.W, sh.r
         self.shape = sh
         hb, rf = head_bytes(sh), record_floats(sh)
         assert hb > 0 and rf > 0, "shape not supported by the library"
-        self.heads = torch.zeros((B, H, hb), dtype=torch.uint8, device=device)
-        self.records = torch.zeros((B, H, W, rf), dtype=torch.float16 if sh.rec16 else torch.float32, device=device)
-        self.decays = torch.zeros((B, H, W), dtype=torch.float32, device=device)
-        self.win_pos = torch.zeros((B,), dtype=torch.int32, device=device)
+        rec_dtype = torch.float16 if sh.rec16 else torch.float32
+        if storage is None:
+            self.heads = torch.zeros((B, H, hb), dtype=torch.uint8, device=device)
+            self.records = torch.zeros((B, H, W, rf), dtype=rec_dtype, device=device)
+            self.decays = torch.zeros((B, H, W), dtype=torch.float32, device=device)
+            self.win_pos = torch.zeros((B,), dtype=torch.int32, device=device)
+        else:
+            self.heads, self.records, self.decays, self.win_pos = storage
+            for t, shape, dt in ((self.heads, (B, H, hb), torch.uint8), (self.records, (B, H, W, rf), rec_dtype),
+                                 (self.decays, (B, H, W), torch.float32), (self.win_pos, (B,), torch.int32)):
+                assert tuple(t.shape) == shape and t.dtype == dt and t.is_contiguous(), (tuple(t.shape), shape, t.dtype, dt)
         if sh.state_bf16:                    # per-window BF16: the head block is S^T in bfloat16, nothing else
             assert hb == 2 * K * V
             self.state16 = self.heads.view(torch.bfloat16).unflatten(-1, (V, K))
@@ -122,7 +131,8 @@ class State:
         self.comp_k = self.heads[..., o:o + 2 * r * K].view(torch.float16).unflatten(-1, (r, K)); o += 2 * r * K
         self.comp_u = self.heads[..., o:o + 2 * r * V].view(torch.float16).unflatten(-1, (r, V)); o += 2 * r * V
         assert o == hb
-        self.row_smooth.fill_(1.0)
+        if storage is None:
+            self.row_smooth.fill_(1.0)
         self._record_views(sh)
 
     def _record_views(self, sh: Shape) -> None:
