@@ -21,7 +21,8 @@
  *    structs themselves are read on the host during the call only.
  *  - bf16 and fp16 values travel as their 16-bit patterns (uint16_t).
  *  - Errors are reported through the return value; nothing aborts or throws.
- *    Argument errors are detected before anything is enqueued.
+ *    Argument errors are detected before anything is enqueued (the host-buffer
+ *    entry points included).
  *  - Arithmetic is IEEE binary32.  Sums over a channel index are taken in a
  *    fixed order (blocks of eight consecutive terms; inside a block the
  *    even-numbered and the odd-numbered terms are two chains of fused
@@ -259,10 +260,25 @@ lq_status lq_ref_decode_step_bf16(const lq_shape *shape, uint16_t *S, const uint
 
 /*
  * Device-side error flags of the current device (0 = none), written to *flags (a host pointer).  Waits inside
- * the kernels are bounded; bit 0 is set when a decode warp gave up waiting for its asynchronous copies, in
- * which case the outputs of that launch are not valid.  The call synchronises the device.
+ * the kernels are bounded; bit 0 is set when a decode warp gave up waiting for its asynchronous copies.  After
+ * that, neither the outputs of that launch NOR THE STATE it worked on are valid (records may be missing or
+ * half written): restore the state from a checkpoint.  Bits 1 and 2 belong to the optional fused step kernel
+ * (gave up waiting for decode work / more heads than it can track), bit 3 to lq_selftest_bounded_wait.
+ * The flags stay set until lq_clear_device_flags is called.  Both calls synchronise the device.
  */
 lq_status lq_check_device(int *flags);
+lq_status lq_clear_device_flags(void);
+
+/*
+ * Self test of the give-up path of the bounded waits (no passage of the paper): launches one warp that
+ * waits, with a limit of 64 polls, on a barrier nothing completes.  The wait returns "gave up", the warp sets
+ * bit 3 of the error flags and exits; the context stays usable.  Read the flag with lq_check_device and clear
+ * it with lq_clear_device_flags.
+ */
+lq_status lq_selftest_bounded_wait(lq_stream stream);
+
+/* LQ_STATIC_STAGE_BYTES as the loaded library was built with (for bindings that cannot read the macro). */
+uint64_t lq_static_stage_bytes(void);
 
 /* Kernels one lq_decode_step call launches for `shape` (used to report launch counts). */
 int lq_decode_launches(const lq_shape *shape);

@@ -544,6 +544,7 @@ static lq_status host_step_impl(const lq_shape *shape, const lq_state *state, co
                                 void *stage, lq_stream stream, bool direct_ok) {
   lq_status rc = check_shape(shape);
   if (rc != LQ_OK) return rc;
+  if ((rc = check_state(shape, state, true)) != LQ_OK) return rc;     // nothing is enqueued before every argument is checked
   if (!q_h || !k_h || !v_h || !beta_h || !alpha_h || !o_h || !stage) return LQ_ERR_NULL;
   if (!aligned16(stage)) return LQ_ERR_ALIGN;
   const uint64_t B = shape->batch, Hv = shape->heads_v, Hqk = shape->heads_qk, K = shape->d_k, V = shape->d_v;
@@ -818,6 +819,7 @@ lq_status lq_decode_step_host_static(const lq_shape *shape, const lq_state *stat
   if (rc != LQ_OK) return rc;
   const uint64_t need = lq_decode_stage_bytes(shape);
   if (need > LQ_STATIC_STAGE_BYTES) return LQ_ERR_TOO_LARGE;
+  if ((rc = check_state(shape, state, true)) != LQ_OK) return rc;     // before the clearing below is enqueued
   if (!q_h || !k_h || !v_h || !beta_h || !alpha_h || !o_h) return LQ_ERR_NULL;
   void *stage = nullptr;
   if ((rc = static_stage_address(&stage)) != LQ_OK) return rc;
@@ -911,6 +913,39 @@ lq_status lq_check_device(int *flags) {
   return LQ_OK;
 }
 
+lq_status lq_clear_device_flags(void) {
+  const int zero = 0;
+  if (cudaMemcpyToSymbol(g_device_error, &zero, sizeof(int)) != cudaSuccess) {
+    cudaGetLastError();
+    return LQ_ERR_CUDA;
+  }
+  return LQ_OK;
+}
+
+uint64_t lq_static_stage_bytes(void) { return LQ_STATIC_STAGE_BYTES; }
+
+}  // extern "C"
+
+// One warp waits, with a limit of a few dozen polls, on a barrier that nothing will ever complete: the wait
+// must come back with "gave up", which is reported like in the decode kernel (error flag, bit 3 here).
+namespace {
+__global__ void bounded_wait_probe_kernel() {
+  __shared__ __align__(8) unsigned long long bar;
+  const uint32_t b = lq::smem_addr(&bar);
+  if (threadIdx.x == 0) lq::mbar_init(b, 1);
+  __syncwarp();
+  const bool done = lq::mbar_wait<64>(b, 0);
+  if (!done && threadIdx.x == 0) atomicOr(&lq::g_device_error, 8);
+}
+}  // namespace
+
+extern "C" {
+
+lq_status lq_selftest_bounded_wait(lq_stream stream) {
+  bounded_wait_probe_kernel<<<1, 32, 0, reinterpret_cast<cudaStream_t>(stream)>>>();
+  return cudaGetLastError() == cudaSuccess ? LQ_OK : LQ_ERR_CUDA;
+}
+
 #ifdef LQ_TIMING
 // development aid: copies the phase counters to host memory and clears them
 int lq_debug_phase_cycles(unsigned long long *out) {
@@ -935,6 +970,6 @@ const char *lq_status_string(lq_status status) {
   return "unknown status";
 }
 
-int lq_version(void) { return 4; }
+int lq_version(void) { return 5; }
 
 }  // extern "C"

@@ -36,7 +36,8 @@
 
 namespace lq {
 
-// Set when a bounded wait gave up (bit 0: a decode warp's wait for one of its bulk copies).  Never cleared by kernels.
+// Set when a bounded wait gave up (bit 0: a decode warp's wait for one of its bulk copies; bits 1, 2: the fused step
+// kernel's waits; bit 3: the wait of lq_selftest_bounded_wait).  Never cleared by kernels: lq_clear_device_flags.
 __device__ int g_device_error = 0;
 
 // ---- shared-memory slot of one CTA ----
@@ -100,9 +101,10 @@ __device__ __forceinline__ void bulk_g2s_hint(uint32_t dst, const void *src, uin
       "l"(src), "r"(bytes), "r"(bar), "l"(policy)
       : "memory");
 }
-// Bounded wait for phase `parity`; false if the limit ran out (the caller then reports and bails out).
+// Bounded wait for phase `parity`; false if the limit of LIMIT polls ran out (the caller then reports and bails out).
+template <int LIMIT = (1 << 20)>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (int spin = 0; spin < (1 << 20); spin++) {
+  for (int spin = 0; spin < LIMIT; spin++) {
     uint32_t done;
     asm volatile(
         "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"

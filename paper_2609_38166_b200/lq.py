@@ -22,7 +22,8 @@ _lib = None
 EXPORTS = ["lq_decode_step", "lq_decode_step_profiled", "lq_decode_step_host", "lq_decode_step_host_pipelined", "lq_decode_step_host_static", "lq_decode_stage_bytes", "lq_head_bytes", "lq_record_floats",
            "lq_window_flush",
            "lq_quantize_state", "lq_dequantize_state", "lq_ref_decode_step_f32", "lq_ref_decode_step_bf16",
-           "lq_decode_launches", "lq_check_device", "lq_status_string", "lq_version"]
+           "lq_decode_launches", "lq_check_device", "lq_clear_device_flags", "lq_selftest_bounded_wait",
+           "lq_static_stage_bytes", "lq_status_string", "lq_version"]
 
 
 class LqError(RuntimeError):
@@ -55,6 +56,12 @@ def lib() -> C.CDLL:
             getattr(L, name).argtypes = [C.c_void_p]
         L.lq_decode_launches.restype = C.c_int
         L.lq_decode_launches.argtypes = [C.c_void_p]
+        L.lq_static_stage_bytes.restype = C.c_uint64
+        L.lq_static_stage_bytes.argtypes = []
+        L.lq_clear_device_flags.restype = C.c_int
+        L.lq_clear_device_flags.argtypes = []
+        L.lq_selftest_bounded_wait.restype = C.c_int
+        L.lq_selftest_bounded_wait.argtypes = [C.c_void_p]
         for name in ("lq_decode_step", "lq_decode_step_profiled", "lq_decode_step_host", "lq_decode_step_host_pipelined",
                      "lq_decode_step_host_static", "lq_check_device", "lq_window_flush", "lq_quantize_state",
                      "lq_dequantize_state", "lq_ref_decode_step_f32", "lq_ref_decode_step_bf16"):
@@ -276,6 +283,21 @@ def check_device() -> int:
     flags = C.c_int(0)
     _check(lib().lq_check_device(C.byref(flags)), "lq_check_device")
     return int(flags.value)
+
+
+def clear_device_flags() -> None:
+    """lq_clear_device_flags: the error flags stay set until this is called."""
+    _check(lib().lq_clear_device_flags(), "lq_clear_device_flags")
+
+
+def selftest_bounded_wait(stream=None) -> None:
+    """lq_selftest_bounded_wait: one warp lets a bounded wait run out; sets bit 3 of the error flags."""
+    _check(lib().lq_selftest_bounded_wait(_stream(stream)), "lq_selftest_bounded_wait")
+
+
+def static_stage_bytes() -> int:
+    """LQ_STATIC_STAGE_BYTES as the loaded library was built with."""
+    return int(lib().lq_static_stage_bytes())
 
 
 def version() -> int:

@@ -28,8 +28,10 @@ def test_every_declared_symbol_is_exported(L):
 
 def test_version_and_status_strings(L):
     assert lq.version() >= 1
-    texts = [L.lq_status_string(i).decode() for i in range(6)]
-    assert texts[0] == "ok" and len(set(texts)) == 6
+    texts = [L.lq_status_string(i).decode() for i in range(7)]
+    assert texts[0] == "ok" and len(set(texts)) == 7 and "unknown" not in texts
+    assert L.lq_status_string(7).decode() == "unknown status"
+    assert lq.static_stage_bytes() == lq.STATIC_STAGE_BYTES      # the binding's constant is the library's
 
 
 def test_argument_errors_are_reported_before_any_launch(L):
@@ -62,6 +64,15 @@ def test_argument_errors_are_reported_before_any_launch(L):
     st_bad = lq._State(*fake)
     assert L.lq_quantize_state(C.byref(s), C.c_void_p(0x100000), C.byref(st_bad), null) == 3
     assert L.lq_quantize_state(C.byref(s), C.c_void_p(0x100004), C.byref(st_ok), null) == 3
+    # the host-buffer entry points check the state as well before they enqueue anything (fake host / stage pointers)
+    hp = C.c_void_p(0x200000)
+    assert L.lq_decode_step_host(C.byref(s), null, hp, hp, hp, hp, hp, hp, hp, null) == 1
+    assert L.lq_decode_step_host(C.byref(s), C.byref(st), hp, hp, hp, hp, hp, hp, hp, null) == 1
+    assert L.lq_decode_step_host(C.byref(s), C.byref(st_bad), hp, hp, hp, hp, hp, hp, hp, null) == 3
+    assert L.lq_decode_step_host_static(C.byref(s), C.byref(st), hp, hp, hp, hp, hp, hp, null) == 1
+    assert L.lq_decode_step_host_static(C.byref(s), C.byref(st_bad), hp, hp, hp, hp, hp, hp, null) == 3
+    big = lq.Shape(64, 32, 16).c()                                # (the pipelined path proper starts at 16 sequences)
+    assert L.lq_decode_step_host_pipelined(C.byref(big), C.byref(st_bad), hp, hp, hp, hp, hp, hp, hp, null) == 3
     assert lq.decode_stage_bytes(sh) > 0 and lq.decode_launches(sh) >= 1
     assert lq.head_bytes(sh) == 19456 and lq.record_floats(sh) == 256
     assert lq.record_floats(lq.Shape(2, 4, 2, gate=lq.GATE_DIAG)) == 384

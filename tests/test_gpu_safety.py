@@ -118,3 +118,24 @@ def test_checkpoint_in_mid_window_resumes_bit_for_bit(gate, rec16):
         assert torch.equal(a.cpu().view(torch.uint8), b.view(torch.uint8)), name
     assert all(b.intact() for b in g.values())
     assert lq.check_device() == 0
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable():
+    """Waits in the kernels are bounded.  The library's self test lets one run out on purpose (a barrier nothing
+    completes, 64 polls): the kernel must come back, the give-up must show in the error flags, the flags must stay
+    set until cleared, and the device must go on working afterwards."""
+    assert lq.check_device() == 0
+    lq.selftest_bounded_wait()
+    assert lq.check_device() == 8
+    assert lq.check_device() == 8                      # sticky
+    lq.clear_device_flags()
+    assert lq.check_device() == 0
+    wl = synth.Workload("after", 2, 2, 2, W=4, r=2, seed=990)
+    _, sh = gu.shapes(wl)
+    st = lq.State(sh)
+    lq.quantize_state(sh, gu.dev(synth.dense_states(wl, 1)), st)
+    o = torch.empty((2, 2, 128), dtype=torch.float32, device="cuda")
+    td = gu.tok_dev(synth.token_inputs(wl, 0))
+    lq.decode_step(sh, st, td["q"], td["k"], td["v"], td["beta"], td["alpha"], o)
+    torch.cuda.synchronize()
+    assert lq.check_device() == 0 and bool(torch.isfinite(o).all())

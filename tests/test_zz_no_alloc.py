@@ -43,8 +43,13 @@ def test_static_staging_matches_caller_staging_on_two_calls(gate):
         tok = _pinned(synth.token_inputs(wl, call))
         o_a.fill_(-1.0); o_b.fill_(-2.0)
         lq.decode_step_host(sh, st_a, tok["q"], tok["k"], tok["v"], tok["beta"], tok["alpha"], o_a, stage)
+        torch.cuda.synchronize()
+        free_before, used_before = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated()
         lq.decode_step_host_static(sh, st_b, tok["q"], tok["k"], tok["v"], tok["beta"], tok["alpha"], o_b)
         torch.cuda.synchronize()
+        if call == 1:        # (the first call may load the module and look the array's address up; the second must not
+            #                   take or return a byte of device memory, through the driver or through torch)
+            assert torch.cuda.mem_get_info()[0] == free_before and torch.cuda.memory_allocated() == used_before
         assert np.allclose(o_b.numpy(), o_a.numpy(), rtol=1e-3, atol=1e-5), call
         assert np.array_equal(o_b.numpy(), o_a.numpy()), call        # same kernels, same bits
         assert call == 1 or not np.any(o_b.numpy()[3])               # cleared rows of the skipped sequence
