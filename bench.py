@@ -50,7 +50,8 @@ def metric_name(wl) -> str:
 
 # DRAM bytes per launch from the ncu captures summarised under profiles/ (dram__bytes_read.sum +
 # dram__bytes_write.sum of one full-batch launch of the gdn_b256 workload, W = 16), or None when not captured.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"decode_kernel": 235.0e6, "boundary_kernel": 18.4e6}
+NCU_CAPTURE_N_ITER = 1                                # (the captures were taken with the default number of rounds)
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"decode_kernel": 235.0e6, "boundary_kernel": 18.5e6}
 # The same two counters from a launch list taken with --cache-control none (the caches are left as the kernel ahead
 # left them, as in a real step): what the L2 serves - the records written by the last tokens, the token vectors, and
 # for the boundary kernel the heads the decode kernel asked the L2 to keep - no longer comes from DRAM.
@@ -76,16 +77,35 @@ def algorithmic_bytes_per_head_step(W: int, r: int, diag: bool, group: int, laun
     return state + buf_read + inputs + rec + 512 + flush / W
 
 
-def config_dict(wl, world: int, warm_tokens: int) -> dict:
+L2_BYTES = 126e6
+
+
+def l2_note(wl) -> str:
+    """Whether the window representation of the whole batch (what a step streams) exceeds the L2."""
     heads = wl.batch * wl.heads_v
+    rec = record_bytes(wl.gate == synth.GATE_DIAG, wl.rec16)
+    mb = heads * (state_bytes(wl.r) + wl.W * rec) / 1e6
+    if mb * 1e6 > 2 * L2_BYTES:
+        return "working set %.0f MB per step exceeds the 126 MB L2; no flush needed" % mb
+    return ("working set %.0f MB per step is below twice the 126 MB L2: this point is (partly) L2-resident and says "
+            "nothing about HBM" % mb)
+
+
+def config_dict(wl, world: int) -> dict:
+    """The workload, the same for both arms (what differs between runs - warm-up length, steps - is not here)."""
     return {"workload": wl.name, "batch": wl.batch, "heads_v": wl.heads_v, "heads_qk": wl.heads_qk,
             "d_k": wl.d_k, "d_v": wl.d_v, "W": wl.W, "r": wl.r, "n_iter": wl.n_iter,
             "gate": "scalar (GDN)" if wl.gate == synth.GATE_SCALAR else "diagonal (KDA)",
             "state_dtype": "int8 + fp32 scales + fp16 compensators", "record_buffer_dtype": "f16" if wl.rec16 else "f32",
-            "inputs_dtype": "bf16", "warmup_tokens": warm_tokens, "window_offsets": "uniform over [0,W)",
-            "l2": "working set %.0f MB per step exceeds the 126 MB L2; no flush needed" %
-                  (heads * (state_bytes(wl.r) + wl.W * (1028 if wl.gate == synth.GATE_SCALAR else 1536)) / 1e6),
+            "inputs_dtype": "bf16", "window_offsets": "uniform over [0,W)", "l2": l2_note(wl),
             "parallelism": "dp%d (independent batches, no collective)" % world}
+
+
+def captured_traffic(wl, table):
+    """The ncu DRAM bytes per launch of `table`, if this run's workload is the one they were captured on."""
+    same = (wl.name == "gdn_b256" and wl.batch == 256 and wl.W == 16 and wl.r == 4 and wl.n_iter == NCU_CAPTURE_N_ITER and
+            wl.gate == synth.GATE_SCALAR and not wl.rec16 and not wl.state_bf16 and wl.smooth == 1 and wl.delta == 1)
+    return dict(table) if same else {k: None for k in table}
 
 
 def shard_workload(wl, rank: int):
@@ -224,7 +244,7 @@ def run_reference(args, wl):
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": s_per_step * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "tokens_heads_per_s": hs,
-            "config": config_dict(wl, args.gpus, 0),
+            "config": config_dict(wl, args.gpus),
             "cpu_baseline": {"value": value, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
@@ -365,13 +385,15 @@ def run_cuda(args, wl):
                 synth.token_inputs(wl, WARM_TOKENS + t).items()} for t in range(wl.W)]
         o_h = torch.empty((wl.batch, wl.heads_v, wl.d_v), dtype=torch.float32).pin_memory()
         stage = torch.empty((lq.decode_stage_bytes(sh),), dtype=torch.uint8, device="cuda")
-        n_e2e = min(args.steps, 2000)
+        # at least 256 calls, after a warm-up of two windows: consecutive calls chain onto each other (the inputs of
+        # a call are fetched next to the previous call's boundary kernels), and a handful of calls is not that regime
+        n_e2e = max(min(args.steps, 2000), 256)
 
         def step_host(t):
             d = pin[t % wl.W]
             lq.decode_step_host_pipelined(sh, st, d["q"], d["k"], d["v"], d["beta"], d["alpha"], o_h, stage, stream)
 
-        for t in range(5):
+        for t in range(2 * wl.W + max(args.warmup, 3)):
             step_host(t)
         barrier()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -435,21 +457,23 @@ def run_cuda(args, wl):
                           "of the timed region; the decode kernel carries 93 % of the bytes)",
                 "algorithmic_bytes_per_head_step": bytes_hs, "algorithmic_bytes_per_step": heads * bytes_hs,
                 "frac_of_nominal_8TBps": achieved / 8000.0}
+    cold, warm = captured_traffic(wl, NCU_TRAFFIC_BYTES_PER_LAUNCH), captured_traffic(wl, NCU_TRAFFIC_WARM_BYTES_PER_LAUNCH)
     if kern:
         dk, bk = kern["decode_ms"], kern["boundary_ms"]
         roofline["kernels"] = {
             "decode_kernel": {"ms": dk, "algorithmic_bytes": decode_bytes, "achieved": decode_bytes / dk / 1e6,
                               "frac": decode_bytes / dk / 1e6 / peak, "bound": "hbm",
-                              "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH["decode_kernel"]},
+                              "traffic": cold["decode_kernel"]},
             "boundary_kernel": {"ms": bk, "algorithmic_bytes": boundary_bytes, "achieved": boundary_bytes / bk / 1e6,
                                 "frac": boundary_bytes / bk / 1e6 / peak,
                                 "bound": "fp32 issue and dependency latency, not hbm",
-                                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH["boundary_kernel"]},
+                                "traffic": cold["boundary_kernel"]},
             "how": "CUDA events on the launching stream around each kernel, mean of %d steps in a second loop" %
                    kern["steps"]}
-        t_d, t_b = NCU_TRAFFIC_BYTES_PER_LAUNCH["decode_kernel"], NCU_TRAFFIC_BYTES_PER_LAUNCH["boundary_kernel"]
-        roofline["traffic"] = (t_d + t_b) if (t_d and t_b) else None
-        roofline["traffic_warm_caches"] = sum(NCU_TRAFFIC_WARM_BYTES_PER_LAUNCH.values())
+    # ncu's DRAM bytes of one step: only for the workload the capture was taken on (profiles/), else null
+    t_d, t_b = cold["decode_kernel"], cold["boundary_kernel"]
+    roofline["traffic"] = (t_d + t_b) if (t_d and t_b) else None
+    roofline["traffic_warm_caches"] = sum(warm.values()) if all(warm.values()) else None
 
     # speed baselines in the same run: dense fp32 / bf16 state, read and written every token
     base = {}
@@ -488,7 +512,7 @@ def run_cuda(args, wl):
     line = {"metric": metric_name(wl), "value": hs * state_bytes(wl.r) / 1e9, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": config_dict(wl, world, args.warm_tokens),
+            "config": config_dict(wl, world), "warmup_tokens": args.warm_tokens,
             "tokens_heads_per_s": hs, "pct_hbm_peak_measured": 100 * achieved / peak,
             "pct_hbm_peak_nominal_8TBps": 100 * achieved / 8000.0,
             "cuda_graph_ms_per_step": graph_ms, "gpu_launches": launches * args.steps,
