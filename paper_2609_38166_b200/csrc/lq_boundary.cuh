@@ -16,7 +16,7 @@ struct BoundarySmem {
   float *cu;     // [r][128]  compensator values widened to fp32
   float *vec;    // [128]     row-sum results (row mean-abs)
   float *colv;   // [128]     1 / c
-  float *part;   // [8][2][128] per-warp column partial sums of two vectors (column maxima: [8][128])
+  float *part;   // [8][4][128] per-warp column partial sums of four vectors (column maxima: [8][128])
   float *gam;    // [128]     Gamma_{1:n}
   float *gram;   // [16][16]  Gram matrix of the vectors being orthonormalised (lower triangle), later K^T K
   float *chol;   // [16][16]  its Cholesky factor L (strictly lower triangle), then [16] 1 / L_hh, [16] alive flags
@@ -31,13 +31,13 @@ struct BoundarySmem {
   uint8_t *zt;   // [128][128] codes Z^T, 16-byte chunk q of row v stored at chunk q ^ ((v >> 3) & 7)
   __half *raw;   // fp16 records only: [W] rows as stored (kt | u | (alpha)), widened into kd, bu by the decay scan
   __host__ __device__ static constexpr int fixed_floats(int r) {
-    return 2 * r * D + 19 * D + 2 * MAX_R * MAX_R + 2 * MAX_R;
+    return 2 * r * D + 35 * D + 2 * MAX_R * MAX_R + 2 * MAX_R;
   }
   __host__ __device__ static constexpr int stage_floats(int W, int r, bool diag, bool rec16) {
     return 2 * W * D + (diag ? W * D : MAX_W) + 2 * D + r * D + D * D / 4 + (rec16 ? W * record_floats(diag) / 2 : 0);
   }
   __device__ __forceinline__ BoundarySmem(float *base, int W, int r, bool diag, bool rec16, int buf) {
-    ck = base; cu = ck + r * D; vec = cu + r * D; colv = vec + D; part = colv + D; gam = part + 16 * D;
+    ck = base; cu = ck + r * D; vec = cu + r * D; colv = vec + D; part = colv + D; gam = part + 32 * D;
     gram = gam + D; chol = gram + MAX_R * MAX_R;
     kd = base + fixed_floats(r) + buf * stage_floats(W, r, diag, rec16);
     bu = kd + W * D; ba = bu + W * D; cs = ba + (diag ? W * D : MAX_W); ss = cs + D;
@@ -266,21 +266,54 @@ __device__ __forceinline__ void orthonormalize(const Params &p, const BoundarySm
   __syncthreads();
   gram_lower(X, nv, sm.gram, t, true);
   __syncthreads();
+  LQ_BTICK(7);
   if (t.tid == 0) cholesky_lower(sm.gram, nv, sm.chol);
   __syncthreads();
+  LQ_BTICK(8);
   if (t.tid < D) {
     const float *L = sm.chol, *inv = L + MAX_R * MAX_R, *alive = inv + MAX_R;
     const int i = t.tid;
-    for (int h = 0; h < nv; h++) {
-      float x = X[h * D + i];
-      for (int j = 0; j < h; j++) x = fmaf(-L[h * MAX_R + j], X[j * D + i], x);
-      X[h * D + i] = x * inv[h];
-    }
-    if (FINAL) {
+    if (nv <= 4) {                                            // everything loaded at once, then registers only
+      float x[4], l[4][4], iv[4], al[4];
+#pragma unroll
+      for (int h = 0; h < 4; h++) {
+        const bool in = h < nv;
+        x[h] = in ? X[h * D + i] : 0.0f;
+        iv[h] = in ? inv[h] : 0.0f;
+        al[h] = in ? alive[h] : 0.0f;
+#pragma unroll
+        for (int j = 0; j < h; j++) l[h][j] = in ? L[h * MAX_R + j] : 0.0f;
+      }
+#pragma unroll
+      for (int h = 0; h < 4; h++) {
+#pragma unroll
+        for (int j = 0; j < h; j++) x[h] = fmaf(-l[h][j], x[j], x[h]);
+        x[h] = x[h] * iv[h];
+      }
+#pragma unroll
+      for (int h = 0; h < 4; h++) {
+        if (h < nv) {
+          float out = x[h];
+          if (FINAL) {
+            const uint16_t bits = al[h] != 0.0f ? to_f16_bits_sat(out) : static_cast<uint16_t>(0);
+            p.comp_k(bh)[h * D + i] = bits;
+            out = f16_bits(bits);
+          }
+          X[h * D + i] = out;
+        }
+      }
+    } else {
       for (int h = 0; h < nv; h++) {
-        const uint16_t bits = alive[h] != 0.0f ? to_f16_bits_sat(X[h * D + i]) : static_cast<uint16_t>(0);
-        p.comp_k(bh)[h * D + i] = bits;
-        X[h * D + i] = f16_bits(bits);
+        float x = X[h * D + i];
+        for (int j = 0; j < h; j++) x = fmaf(-L[h * MAX_R + j], X[j * D + i], x);
+        X[h * D + i] = x * inv[h];
+      }
+      if (FINAL) {
+        for (int h = 0; h < nv; h++) {
+          const uint16_t bits = alive[h] != 0.0f ? to_f16_bits_sat(X[h * D + i]) : static_cast<uint16_t>(0);
+          p.comp_k(bh)[h * D + i] = bits;
+          X[h * D + i] = f16_bits(bits);
+        }
       }
     }
   }
@@ -308,37 +341,33 @@ __device__ __forceinline__ void rows_times_vectors(const float (&M)[8][8], const
   }
 }
 
-// Out[h] = M^T x_h for the nv vectors x_h in Xm (rows of 128 floats in shared memory), two at a time.
+// Out[h] = M^T x_h for the nv vectors x_h in Xm (rows of 128 floats in shared memory), four to a round of barriers.
 // Column sums in the fixed order: this thread's eight rows, its neighbour in the warp (lane ^ 16), then the
 // eight warps as a balanced tree.  Begins after a barrier of the caller (Xm complete); ends with a barrier.
 __device__ __forceinline__ void columns_times_vectors(const float (&M)[8][8], const BoundarySmem &sm, const Tile &t,
                                                       int nv, const float *Xm, float *Out) {
   const bool up = t.lane & 16;
-  for (int h0 = 0; h0 < nv; h0 += 2) {
-    const bool two = h0 + 1 < nv;
-    float x0[8], x1[8], pc0[8], pc1[8];
-    load8(Xm + h0 * D + 8 * t.ty, x0);
-    load8(Xm + (two ? h0 + 1 : h0) * D + 8 * t.ty, x1);
-    col_blocks(M, x0, pc0);
-    col_blocks(M, x1, pc1);
-    float r0[4], r1[4];
+  for (int h0 = 0; h0 < nv; h0 += 4) {
+    const int nh = nv - h0 < 4 ? nv - h0 : 4;
+    if (h0 > 0) __syncthreads();                              // the previous round's partial sums have been read
+    for (int hh = 0; hh < nh; hh++) {                         // first half: own rows, then the neighbour's
+      float x[8], pc[8], rr[4];
+      load8(Xm + (h0 + hh) * D + 8 * t.ty, x);
+      col_blocks(M, x, pc);
 #pragma unroll
-    for (int e = 0; e < 4; e++) {
-      const float keep0 = up ? pc0[e + 4] : pc0[e], send0 = up ? pc0[e] : pc0[e + 4];
-      const float keep1 = up ? pc1[e + 4] : pc1[e], send1 = up ? pc1[e] : pc1[e + 4];
-      r0[e] = keep0 + __shfl_xor_sync(FULL, send0, 16);
-      r1[e] = keep1 + __shfl_xor_sync(FULL, send1, 16);
+      for (int e = 0; e < 4; e++) {
+        const float keep = up ? pc[e + 4] : pc[e], send = up ? pc[e] : pc[e + 4];
+        rr[e] = keep + __shfl_xor_sync(FULL, send, 16);
+      }
+      *reinterpret_cast<float4 *>(sm.part + (t.warp * 4 + hh) * D + 8 * t.tx + (up ? 4 : 0)) =
+          make_float4(rr[0], rr[1], rr[2], rr[3]);
     }
-    if (h0 > 0) __syncthreads();                              // the previous pair's partial sums have been read
-    float *part = sm.part + t.warp * 2 * D + 8 * t.tx + (up ? 4 : 0);
-    *reinterpret_cast<float4 *>(part) = make_float4(r0[0], r0[1], r0[2], r0[3]);
-    *reinterpret_cast<float4 *>(part + D) = make_float4(r1[0], r1[1], r1[2], r1[3]);
     __syncthreads();
-    {
-      const int v = t.tid >> 7, col = t.tid & (D - 1);
+    for (int idx = t.tid; idx < nh * D; idx += 256) {         // second half: the eight warps
+      const int v = idx >> 7, col = idx & (D - 1);
       const float *c = sm.part + v * D + col;
-      const float sum = ((c[0] + c[2 * D]) + (c[4 * D] + c[6 * D])) + ((c[8 * D] + c[10 * D]) + (c[12 * D] + c[14 * D]));
-      if (v == 0 || two) Out[(h0 + v) * D + col] = sum;
+      Out[(h0 + v) * D + col] =
+          ((c[0] + c[4 * D]) + (c[8 * D] + c[12 * D])) + ((c[16 * D] + c[20 * D]) + (c[24 * D] + c[28 * D]));
     }
   }
   __syncthreads();
@@ -386,12 +415,35 @@ __device__ __forceinline__ void quantize_tile(const Params &p, const BoundarySme
     if (t.tid < D) {
       const float *alive = sm.chol + MAX_R * MAX_R + MAX_R;
       const int j = t.tid;
-      for (int h = 0; h < r; h++) {                           // (reads back the stored values u_a it wrote)
-        float x = Wm[h * D + j];
-        for (int a = 0; a < h; a++) x = fmaf(-Wm[a * D + j], sm.gram[h * MAX_R + a], x);
-        const uint16_t bits = alive[h] != 0.0f ? to_f16_bits_sat(x) : static_cast<uint16_t>(0);
-        p.comp_u(bh)[h * D + j] = bits;
-        Wm[h * D + j] = f16_bits(bits);
+      if (r <= 4) {                                           // everything loaded at once, then registers only
+        float x[4], g[4][4], al[4], uf[4];
+#pragma unroll
+        for (int h = 0; h < 4; h++) {
+          const bool in = h < r;
+          x[h] = in ? Wm[h * D + j] : 0.0f;
+          al[h] = in ? alive[h] : 0.0f;
+#pragma unroll
+          for (int a = 0; a < h; a++) g[h][a] = in ? sm.gram[h * MAX_R + a] : 0.0f;
+        }
+#pragma unroll
+        for (int h = 0; h < 4; h++) {
+#pragma unroll
+          for (int a = 0; a < h; a++) x[h] = fmaf(-uf[a], g[h][a], x[h]);
+          const uint16_t bits = al[h] != 0.0f ? to_f16_bits_sat(x[h]) : static_cast<uint16_t>(0);
+          uf[h] = f16_bits(bits);
+          if (h < r) {
+            p.comp_u(bh)[h * D + j] = bits;
+            Wm[h * D + j] = uf[h];
+          }
+        }
+      } else {
+        for (int h = 0; h < r; h++) {                         // (reads back the stored values u_a it wrote)
+          float x = Wm[h * D + j];
+          for (int a = 0; a < h; a++) x = fmaf(-Wm[a * D + j], sm.gram[h * MAX_R + a], x);
+          const uint16_t bits = alive[h] != 0.0f ? to_f16_bits_sat(x) : static_cast<uint16_t>(0);
+          p.comp_u(bh)[h * D + j] = bits;
+          Wm[h * D + j] = f16_bits(bits);
+        }
       }
     }
     __syncthreads();
