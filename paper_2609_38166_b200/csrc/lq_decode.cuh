@@ -40,12 +40,19 @@ namespace lq {
 // kernel's waits; bit 3: the wait of lq_selftest_bounded_wait).  Never cleared by kernels: lq_clear_device_flags.
 __device__ int g_device_error = 0;
 
+// Rows of the record buffer that a scalar-gate decode slot holds at a time (a multiple of four: the walk takes the
+// records four at a time from the newest back, so a group of four never straddles two segments).
+constexpr int REC_SEG = 32;
+
 // ---- shared-memory slot of one CTA ----
 struct DecodeSlot {
   // byte offsets inside the slot; every region starts on a 16-byte boundary
   int head, rec, bas, digits, y, pk, pq, mbar, bytes;
   __host__ __device__ DecodeSlot(int W, int r, bool diag, bool rec16 = false) {
-    const int rows = W > 1 ? W - 1 : 1;   // a window holds at most W-1 records when a token arrives
+    // a window holds at most W-1 records when a token arrives; with the scalar gate, where only the dot warp reads
+    // them, they are staged REC_SEG rows at a time (newest first), which keeps the slot small for long windows
+    int rows = W > 1 ? W - 1 : 1;
+    if (!diag && rows > REC_SEG) rows = REC_SEG;
     int o = 0;
     head = o; o += head_bytes(r);          // the head block: codes | col_scale | row_smooth | comp_k | comp_u
     rec = o; o += (rec16 ? 2 : 4) * record_floats(diag) * rows;   // buffered record rows (fp32 or fp16)
@@ -263,16 +270,21 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
       else bulk_g2s_hint(slot_a + L.head, p.head(bh), head_bytes(r), barA, stream);
     }
   };
-  auto request_records = [&](unsigned bh, int n) {
+  // first record of the segment that ends before record `hi` (everything from record 0 with the diagonal gate)
+  auto seg_base = [&](int hi) { return (!DIAG && hi > REC_SEG) ? hi - REC_SEG : 0; };
+  // records [seg_base(hi), hi) of head bh, n of which are buffered in all, into the slot
+  auto request_segment = [&](unsigned bh, int n, int hi) {
     if (lane == 0) {
-      const uint32_t rb = static_cast<uint32_t>(sizeof(rec_t)) * RF * n;
+      const int lo = seg_base(hi);
+      const uint32_t rb = static_cast<uint32_t>(sizeof(rec_t)) * RF * (hi - lo);
       mbar_expect_tx(barR, rb);              // with no records the phase completes at once
-      if (n > 0) {
-        if (n == W - 1) bulk_g2s_hint(slot_a + L.rec, p.record<rec_t>(bh, 0, DIAG), rb, barR, keep);
-        else bulk_g2s_hint(slot_a + L.rec, p.record<rec_t>(bh, 0, DIAG), rb, barR, stream);
+      if (hi > lo) {
+        if (n == W - 1) bulk_g2s_hint(slot_a + L.rec, p.record<rec_t>(bh, lo, DIAG), rb, barR, keep);
+        else bulk_g2s_hint(slot_a + L.rec, p.record<rec_t>(bh, lo, DIAG), rb, barR, stream);
       }
     }
   };
+  auto request_records = [&](unsigned bh, int n) { request_segment(bh, n, n); };   // the newest segment
   // Bounded wait for one of the two.  A copy that never lands must not hang the GPU: when the limit runs out the
   // error flag is set and the warp goes on (its results are garbage, the flag says so); the other warp, which
   // meets this one at the named barriers, is not left waiting.
@@ -446,7 +458,14 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
       LQ_TICK(4);
       if (!DIAG) wait_for(barR, parR);
       float rk_rec[4] = {0.0f, 0.0f, 0.0f, 0.0f}, rq_rec[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+      int base = seg_base(n);                        // the slot holds records base .. (row = record - base)
       for (int jt = n - 1; jt >= 0; jt -= 4) {       // records jt, jt-1, jt-2, jt-3
+        if (!DIAG && jt < base) {                    // the segment is walked: fetch the one before it
+          __syncwarp();
+          request_segment(bh, n, base);
+          base = seg_base(base);
+          wait_for(barR, parR);
+        }
         float s4[4];
         int jo[2];
 #pragma unroll
@@ -454,7 +473,7 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
           // the decays of the two records of this pair; the half that owns the older one steps over the newer
           const int jn = jt - 2 * u, jold = jn - 1;  // newer, older
           float2 an[4], ao[4], gmine[4];
-          if (DIAG) {
+          if (DIAG) {                                // (base = 0 with the diagonal gate)
             load8p(rec + (jn > 0 ? jn : 0) * RF + REC_A + 8 * c, an);
             load8p(rec + (jold > 0 ? jold : 0) * RF + REC_A + 8 * c, ao);
           } else {
@@ -469,9 +488,9 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
             g2[cc] = __fmul2_rn(go, ao[cc]);                          // past both records
           }
           jo[u] = jn - half;
-          const int j = jo[u] >= 0 ? jo[u] : 0;
+          const int j = jo[u] >= 0 ? jo[u] : 0;      // (record 0 is in the slot whenever an index runs below it)
           float2 x2[4], yk2[4], yq2[4];
-          load8p(rec + j * RF + REC_KT + 8 * c, x2);
+          load8p(rec + (j - base) * RF + REC_KT + 8 * c, x2);
 #pragma unroll
           for (int cc = 0; cc < 4; cc++) { yk2[cc] = __fmul2_rn(gmine[cc], k2[cc]); yq2[cc] = __fmul2_rn(gmine[cc], q2[cc]); }
           s4[2 * u] = block8(x2, yk2);
@@ -492,7 +511,7 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
             const int u = i4 >> 1;
             const bool mine = (i4 & 1) == half;
             const float pkj = mine ? s4[2 * u] : oth[2 * u], pqj = mine ? s4[2 * u + 1] : oth[2 * u + 1];
-            const float4 u4 = load4(rec + j * RF + REC_U + 4 * lane);
+            const float4 u4 = load4(rec + (j - base) * RF + REC_U + 4 * lane);
             rk_rec[0] = fmaf(u4.x, pkj, rk_rec[0]); rq_rec[0] = fmaf(u4.x, pqj, rq_rec[0]);
             rk_rec[1] = fmaf(u4.y, pkj, rk_rec[1]); rq_rec[1] = fmaf(u4.y, pqj, rq_rec[1]);
             rk_rec[2] = fmaf(u4.z, pkj, rk_rec[2]); rq_rec[2] = fmaf(u4.z, pqj, rq_rec[2]);
