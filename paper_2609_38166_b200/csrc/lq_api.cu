@@ -20,7 +20,8 @@ namespace lq {
 // MODE 0: flush (window representation -> dense -> new window representation)
 // MODE 1: quantize dense fp32 states         MODE 2: dequantize to dense fp32 states
 // ---------------------------------------------------------------------------------------------
-template <int GATE, int MODE, bool R16>
+// RM: the largest r the instance handles (4, 8 or MAX_R; the fit keeps its small matrices in registers, RM wide).
+template <int GATE, int MODE, bool R16, int RM>
 __global__ void __launch_bounds__(256, 2) boundary_kernel(const Params p, const int stage_bufs) {
   extern __shared__ float4 lq_smem4[];
   float *smem = reinterpret_cast<float *>(lq_smem4);
@@ -92,7 +93,7 @@ __global__ void __launch_bounds__(256, 2) boundary_kernel(const Params p, const 
 #pragma unroll
         for (int a = 0; a < 8; a++) store8(S + (8 * t.ty + a) * D + 8 * t.tx, M[a]);
       } else {
-        quantize_tile(p, sm, t, bh, MODE == 0 ? n : 0, M);
+        quantize_tile<RM>(p, sm, t, bh, MODE == 0 ? n : 0, M);
       }
       __syncthreads();                       // this head's use of shared memory is over
       LQ_BTICK(9);
@@ -365,11 +366,25 @@ static lq_status launch_boundary(const lq_shape *s, const Params &p, cudaStream_
   const long nh = (long)s->batch * s->heads_v;
   // persistent: the CTAs that are resident at once (two per SM), each striding over the heads
   const int grid = static_cast<int>(nh < 2L * sm_count() ? nh : 2L * sm_count());
+  // the flush (the hot one) is compiled for r <= 4, r <= 8 and any r; the others once
+  constexpr int M_ = MODE;
+  if (MODE == 0 && s->r <= 4) {
+    if (r16) return diag ? launch_dependent(boundary_kernel<LQ_GATE_DIAG, M_, true, 4>, grid, 256, smem, stream, p, bufs)
+                         : launch_dependent(boundary_kernel<LQ_GATE_SCALAR, M_, true, 4>, grid, 256, smem, stream, p, bufs);
+    return diag ? launch_dependent(boundary_kernel<LQ_GATE_DIAG, M_, false, 4>, grid, 256, smem, stream, p, bufs)
+                : launch_dependent(boundary_kernel<LQ_GATE_SCALAR, M_, false, 4>, grid, 256, smem, stream, p, bufs);
+  }
+  if (MODE == 0 && s->r <= 8) {
+    if (r16) return diag ? launch_dependent(boundary_kernel<LQ_GATE_DIAG, M_, true, 8>, grid, 256, smem, stream, p, bufs)
+                         : launch_dependent(boundary_kernel<LQ_GATE_SCALAR, M_, true, 8>, grid, 256, smem, stream, p, bufs);
+    return diag ? launch_dependent(boundary_kernel<LQ_GATE_DIAG, M_, false, 8>, grid, 256, smem, stream, p, bufs)
+                : launch_dependent(boundary_kernel<LQ_GATE_SCALAR, M_, false, 8>, grid, 256, smem, stream, p, bufs);
+  }
   if (r16)
-    return diag ? launch_dependent(boundary_kernel<LQ_GATE_DIAG, MODE == 1 ? 0 : MODE, true>, grid, 256, smem, stream, p, bufs)
-                : launch_dependent(boundary_kernel<LQ_GATE_SCALAR, MODE == 1 ? 0 : MODE, true>, grid, 256, smem, stream, p, bufs);
-  return diag ? launch_dependent(boundary_kernel<LQ_GATE_DIAG, MODE, false>, grid, 256, smem, stream, p, bufs)
-              : launch_dependent(boundary_kernel<LQ_GATE_SCALAR, MODE, false>, grid, 256, smem, stream, p, bufs);
+    return diag ? launch_dependent(boundary_kernel<LQ_GATE_DIAG, MODE == 1 ? 0 : MODE, true, MAX_R>, grid, 256, smem, stream, p, bufs)
+                : launch_dependent(boundary_kernel<LQ_GATE_SCALAR, MODE == 1 ? 0 : MODE, true, MAX_R>, grid, 256, smem, stream, p, bufs);
+  return diag ? launch_dependent(boundary_kernel<LQ_GATE_DIAG, MODE, false, MAX_R>, grid, 256, smem, stream, p, bufs)
+              : launch_dependent(boundary_kernel<LQ_GATE_SCALAR, MODE, false, MAX_R>, grid, 256, smem, stream, p, bufs);
 }
 
 // The step as one cooperative kernel (lq_fused.cuh): one decode CTA and one boundary CTA per SM.

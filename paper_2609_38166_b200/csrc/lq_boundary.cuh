@@ -206,114 +206,124 @@ __device__ __forceinline__ void gram_lower(const float *X, int nv, float *G, con
   }
 }
 
-// Cholesky factor of the Gram matrix, by one thread: L (strictly lower part), inv[h] = 1 / L_hh, alive[h].
+// Cholesky factor of the Gram matrix of up to four vectors, by one thread, in registers (all loads first):
+// L (strictly lower part), inv[h] = 1 / L_hh, alive[h], to shared memory.  Same arithmetic as the warp's version below.
+__device__ __forceinline__ void cholesky_lower_4(const float *G, int nv, float *L) {
+  float *inv = L + MAX_R * MAX_R, *alive = inv + MAX_R;
+  float g[4][4], l[4][4], iv[4];
+#pragma unroll
+  for (int h = 0; h < 4; h++)
+#pragma unroll
+    for (int j = 0; j <= h; j++) g[h][j] = h < nv ? G[h * MAX_R + j] : 0.0f;
+#pragma unroll
+  for (int h = 0; h < 4; h++) {
+#pragma unroll
+    for (int j = 0; j < h; j++) {
+      float sacc = g[h][j];
+#pragma unroll
+      for (int m = 0; m < j; m++) sacc = fmaf(-l[h][m], l[j][m], sacc);
+      l[h][j] = sacc * iv[j];
+    }
+    float d = g[h][h];
+#pragma unroll
+    for (int m = 0; m < h; m++) d = fmaf(-l[h][m], l[h][m], d);
+    const bool ok = g[h][h] >= 1e-30f && d > 1e-6f * g[h][h];
+    iv[h] = ok ? 1.0f / sqrtf(d) : 0.0f;
+    if (h < nv) {
+#pragma unroll
+      for (int j = 0; j < h; j++) L[h * MAX_R + j] = l[h][j];
+      inv[h] = iv[h];
+      alive[h] = ok ? 1.0f : 0.0f;
+    }
+  }
+}
+
+// Cholesky factor of the Gram matrix, by one warp: lane h owns row h of L.  Column by column: lane j finishes
+// L_jj from its own row, the lanes below it their entry of column j (the entries of row j they need come by
+// shuffle from lane j); the arithmetic of an entry is  s = G_hj; s = fma(-L_hm, L_jm, s) for m < j; L_hj = s / L_jj.
+// Writes L (strictly lower part), inv[h] = 1 / L_hh and alive[h] to shared memory.
 // A vector whose squared length is below 1e-30, or of which the vectors before it leave no more than 1e-6 of its
 // squared length, is dropped: inv = 0, which makes its orthonormalised vector and all its L entries zero.
-// Up to four vectors are handled in registers (all loads first, then arithmetic only); more go through shared memory.
-__device__ __forceinline__ void cholesky_lower(const float *G, int nv, float *L) {
+// RM: the largest number of vectors this instance is compiled for (nv <= RM <= MAX_R).
+template <int RM>
+__device__ __forceinline__ void cholesky_lower_warp(const float *G, int nv, float *L, int lane) {
   float *inv = L + MAX_R * MAX_R, *alive = inv + MAX_R;
-  if (nv <= 4) {
-    float g[4][4], l[4][4], iv[4];
+  const int h = lane;
+  float g[RM], l[RM];
 #pragma unroll
-    for (int h = 0; h < 4; h++)
-#pragma unroll
-      for (int j = 0; j <= h; j++) g[h][j] = h < nv ? G[h * MAX_R + j] : 0.0f;
-#pragma unroll
-    for (int h = 0; h < 4; h++) {
-#pragma unroll
-      for (int j = 0; j < h; j++) {
-        float sacc = g[h][j];
-#pragma unroll
-        for (int m = 0; m < j; m++) sacc = fmaf(-l[h][m], l[j][m], sacc);
-        l[h][j] = sacc * iv[j];
-      }
-      float d = g[h][h];
-#pragma unroll
-      for (int m = 0; m < h; m++) d = fmaf(-l[h][m], l[h][m], d);
-      const bool ok = g[h][h] >= 1e-30f && d > 1e-6f * g[h][h];
-      iv[h] = ok ? 1.0f / sqrtf(d) : 0.0f;
-      if (h < nv) {
-#pragma unroll
-        for (int j = 0; j < h; j++) L[h * MAX_R + j] = l[h][j];
-        inv[h] = iv[h];
-        alive[h] = ok ? 1.0f : 0.0f;
-      }
-    }
-    return;
+  for (int j = 0; j < RM; j++) {
+    g[j] = (h < nv && j <= h) ? G[h * MAX_R + j] : 0.0f;
+    l[j] = 0.0f;
   }
-  for (int h = 0; h < nv; h++) {
-    for (int j = 0; j < h; j++) {
-      float sacc = G[h * MAX_R + j];
-      for (int m = 0; m < j; m++) sacc = fmaf(-L[h * MAX_R + m], L[j * MAX_R + m], sacc);
-      L[h * MAX_R + j] = sacc * inv[j];
+  float inv_h = 0.0f;
+  bool ok_h = false;
+#pragma unroll
+  for (int j = 0; j < RM; j++) {
+    if (j < nv) {                                            // (the same for every lane)
+      float d = g[j];                                        // meaningful in lane j: G_jj minus the squares of row j
+#pragma unroll
+      for (int m = 0; m < j; m++) d = fmaf(-l[m], l[m], d);
+      const bool ok = g[j] >= 1e-30f && d > 1e-6f * g[j];
+      const float iv = ok ? 1.0f / sqrtf(d) : 0.0f;
+      const float inv_j = __shfl_sync(FULL, iv, j);
+      if (lane == j) { inv_h = iv; ok_h = ok; }
+      float sacc = g[j];                                     // meaningful in lanes h > j: G_hj
+#pragma unroll
+      for (int m = 0; m < j; m++) sacc = fmaf(-l[m], __shfl_sync(FULL, l[m], j), sacc);
+      if (h > j) l[j] = sacc * inv_j;
     }
-    const float ghh = G[h * MAX_R + h];
-    float d = ghh;
-    for (int m = 0; m < h; m++) d = fmaf(-L[h * MAX_R + m], L[h * MAX_R + m], d);
-    const bool ok = ghh >= 1e-30f && d > 1e-6f * ghh;
-    inv[h] = ok ? 1.0f / sqrtf(d) : 0.0f;
-    alive[h] = ok ? 1.0f : 0.0f;
+  }
+  if (h < nv) {
+#pragma unroll
+    for (int j = 0; j < RM; j++)
+      if (j < h) L[h * MAX_R + j] = l[j];
+    inv[h] = inv_h;
+    alive[h] = ok_h ? 1.0f : 0.0f;
   }
 }
 
 // Orthonormalise the nv vectors X (rows of 128 floats in shared memory) in place, in order:
-// q_h = (x_h - sum_{j<h} L_hj q_j) / L_hh, one thread per element index (it reads back the q_j it wrote).
+// q_h = (x_h - sum_{j<h} L_hj q_j) / L_hh, one thread per element index, its nv values in registers.
 // With FINAL the results are then rounded to fp16 (what is stored as compensator keys), written to comp_k of
 // head bh and kept in X as the stored values.  Begins and ends with a barrier.
-template <bool FINAL>
+template <bool FINAL, int RM>
 __device__ __forceinline__ void orthonormalize(const Params &p, const BoundarySmem &sm, const Tile &t, float *X,
                                                int nv, size_t bh) {
   __syncthreads();
   gram_lower(X, nv, sm.gram, t, true);
   __syncthreads();
   LQ_BTICK(7);
-  if (t.tid == 0) cholesky_lower(sm.gram, nv, sm.chol);
+  if (RM <= 4) {                                             // four dependent 1/sqrt: one thread is the shortest chain
+    if (t.tid == 0) cholesky_lower_4(sm.gram, nv, sm.chol);
+  } else if (t.warp == 0) {
+    cholesky_lower_warp<RM>(sm.gram, nv, sm.chol, t.lane);
+  }
   __syncthreads();
   LQ_BTICK(8);
   if (t.tid < D) {
     const float *L = sm.chol, *inv = L + MAX_R * MAX_R, *alive = inv + MAX_R;
     const int i = t.tid;
-    if (nv <= 4) {                                            // everything loaded at once, then registers only
-      float x[4], l[4][4], iv[4], al[4];
+    float x[RM];
 #pragma unroll
-      for (int h = 0; h < 4; h++) {
-        const bool in = h < nv;
-        x[h] = in ? X[h * D + i] : 0.0f;
-        iv[h] = in ? inv[h] : 0.0f;
-        al[h] = in ? alive[h] : 0.0f;
+    for (int h = 0; h < RM; h++) x[h] = h < nv ? X[h * D + i] : 0.0f;
 #pragma unroll
-        for (int j = 0; j < h; j++) l[h][j] = in ? L[h * MAX_R + j] : 0.0f;
+    for (int h = 0; h < RM; h++) {
+      if (h < nv) {
+#pragma unroll
+        for (int j = 0; j < h; j++) x[h] = fmaf(-L[h * MAX_R + j], x[j], x[h]);
+        x[h] = x[h] * inv[h];
       }
+    }
 #pragma unroll
-      for (int h = 0; h < 4; h++) {
-#pragma unroll
-        for (int j = 0; j < h; j++) x[h] = fmaf(-l[h][j], x[j], x[h]);
-        x[h] = x[h] * iv[h];
-      }
-#pragma unroll
-      for (int h = 0; h < 4; h++) {
-        if (h < nv) {
-          float out = x[h];
-          if (FINAL) {
-            const uint16_t bits = al[h] != 0.0f ? to_f16_bits_sat(out) : static_cast<uint16_t>(0);
-            p.comp_k(bh)[h * D + i] = bits;
-            out = f16_bits(bits);
-          }
-          X[h * D + i] = out;
-        }
-      }
-    } else {
-      for (int h = 0; h < nv; h++) {
-        float x = X[h * D + i];
-        for (int j = 0; j < h; j++) x = fmaf(-L[h * MAX_R + j], X[j * D + i], x);
-        X[h * D + i] = x * inv[h];
-      }
-      if (FINAL) {
-        for (int h = 0; h < nv; h++) {
-          const uint16_t bits = alive[h] != 0.0f ? to_f16_bits_sat(X[h * D + i]) : static_cast<uint16_t>(0);
+    for (int h = 0; h < RM; h++) {
+      if (h < nv) {
+        float out = x[h];
+        if (FINAL) {
+          const uint16_t bits = alive[h] != 0.0f ? to_f16_bits_sat(out) : static_cast<uint16_t>(0);
           p.comp_k(bh)[h * D + i] = bits;
-          X[h * D + i] = f16_bits(bits);
+          out = f16_bits(bits);
         }
+        X[h * D + i] = out;
       }
     }
   }
@@ -381,6 +391,8 @@ __device__ __forceinline__ void columns_times_vectors(const float (&M)[8][8], co
 // (h+1)-th newest of the n records in sm.bu, from a Walsh vector where there is no such record.  The keys are
 // rounded to fp16; value side h is M^T k_h - sum_{a<h} u_a (k_a^T k_h) with the stored values (the least-squares
 // answer for what components 0..h-1 leave), rounded to fp16 in turn; then M -= K U^T with the stored values.
+// RM: the largest r this instance is compiled for (the small matrices of the fit live in registers, RM wide).
+template <int RM>
 __device__ __forceinline__ void quantize_tile(const Params &p, const BoundarySmem &sm, const Tile &t, size_t bh,
                                               int n, float (&M)[8][8]) {
   const int r = p.r;
@@ -402,12 +414,12 @@ __device__ __forceinline__ void quantize_tile(const Params &p, const BoundarySme
       }
       LQ_BTICK(10);
       if (it + 1 < p.n_iter) {
-        orthonormalize<false>(p, sm, t, Tm, r, bh);
+        orthonormalize<false, RM>(p, sm, t, Tm, r, bh);
         columns_times_vectors(M, sm, t, r, Tm, Wm);
-        orthonormalize<false>(p, sm, t, Wm, r, bh);
+        orthonormalize<false, RM>(p, sm, t, Wm, r, bh);
       }
     }
-    orthonormalize<true>(p, sm, t, Tm, r, bh);                // Tm now holds the keys as stored
+    orthonormalize<true, RM>(p, sm, t, Tm, r, bh);                // Tm now holds the keys as stored
     LQ_BTICK(11);
     gram_lower(Tm, r, sm.gram, t, false);                     // k_a^T k_h, a < h, in gram[h][a]
     columns_times_vectors(M, sm, t, r, Tm, Wm);               // M^T k_h (its barriers also publish gram)
@@ -415,34 +427,24 @@ __device__ __forceinline__ void quantize_tile(const Params &p, const BoundarySme
     if (t.tid < D) {
       const float *alive = sm.chol + MAX_R * MAX_R + MAX_R;
       const int j = t.tid;
-      if (r <= 4) {                                           // everything loaded at once, then registers only
-        float x[4], g[4][4], al[4], uf[4];
+      float x[RM], uf[RM];                                    // this column's sums, then its stored values u_a
+      uint16_t ub[RM];
 #pragma unroll
-        for (int h = 0; h < 4; h++) {
-          const bool in = h < r;
-          x[h] = in ? Wm[h * D + j] : 0.0f;
-          al[h] = in ? alive[h] : 0.0f;
+      for (int h = 0; h < RM; h++) x[h] = h < r ? Wm[h * D + j] : 0.0f;
 #pragma unroll
-          for (int a = 0; a < h; a++) g[h][a] = in ? sm.gram[h * MAX_R + a] : 0.0f;
+      for (int h = 0; h < RM; h++) {
+        if (h < r) {
+#pragma unroll
+          for (int a = 0; a < h; a++) x[h] = fmaf(-uf[a], sm.gram[h * MAX_R + a], x[h]);
+          ub[h] = alive[h] != 0.0f ? to_f16_bits_sat(x[h]) : static_cast<uint16_t>(0);
+          uf[h] = f16_bits(ub[h]);
         }
+      }
 #pragma unroll
-        for (int h = 0; h < 4; h++) {
-#pragma unroll
-          for (int a = 0; a < h; a++) x[h] = fmaf(-uf[a], g[h][a], x[h]);
-          const uint16_t bits = al[h] != 0.0f ? to_f16_bits_sat(x[h]) : static_cast<uint16_t>(0);
-          uf[h] = f16_bits(bits);
-          if (h < r) {
-            p.comp_u(bh)[h * D + j] = bits;
-            Wm[h * D + j] = uf[h];
-          }
-        }
-      } else {
-        for (int h = 0; h < r; h++) {                         // (reads back the stored values u_a it wrote)
-          float x = Wm[h * D + j];
-          for (int a = 0; a < h; a++) x = fmaf(-Wm[a * D + j], sm.gram[h * MAX_R + a], x);
-          const uint16_t bits = alive[h] != 0.0f ? to_f16_bits_sat(x) : static_cast<uint16_t>(0);
-          p.comp_u(bh)[h * D + j] = bits;
-          Wm[h * D + j] = f16_bits(bits);
+      for (int h = 0; h < RM; h++) {
+        if (h < r) {
+          p.comp_u(bh)[h * D + j] = ub[h];
+          Wm[h * D + j] = uf[h];
         }
       }
     }

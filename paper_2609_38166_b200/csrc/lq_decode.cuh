@@ -42,7 +42,7 @@ __device__ int g_device_error = 0;
 
 // Rows of the record buffer that a scalar-gate decode slot holds at a time (a multiple of four: the walk takes the
 // records four at a time from the newest back, so a group of four never straddles two segments).
-constexpr int REC_SEG = 32;
+constexpr int REC_SEG = 32;                // (16 was tried: no faster at W = 32 or 64)
 
 // ---- shared-memory slot of one CTA ----
 struct DecodeSlot {

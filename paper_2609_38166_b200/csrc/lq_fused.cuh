@@ -44,7 +44,7 @@ __device__ __forceinline__ void fused_boundary_head(const Params &p, float *smem
   if (!DIAG && t.tid < n) sm.ba[t.tid] = __ldcg(p.decays + bh * (size_t)p.W + t.tid);
   __syncthreads();
   reconstruct_tile<GATE, R16>(p, sm, t, bh, n, M);
-  quantize_tile(p, sm, t, bh, n, M);
+  quantize_tile<MAX_R>(p, sm, t, bh, n, M);
   __syncthreads();                           // this head's use of shared memory is over
   if (t.tid == 0) arrive_and_set(p.win_pos, b, p.heads_v, 0);
 }
