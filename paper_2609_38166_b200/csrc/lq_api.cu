@@ -469,12 +469,22 @@ static lq_status decode_step_impl(const lq_shape *shape, const lq_state *state, 
     if (frc != LQ_ERR_UNSUPPORTED) return frc;       // does not fit this device or shape: the two kernels below
   }
   const size_t smem = DecodeSlot(shape->W, shape->r, diag, r16).bytes;
-  if (r16)
-    rc = diag ? launch_persistent(decode_kernel<LQ_GATE_DIAG, true>, nh, 64, smem, st, p)
-              : launch_persistent(decode_kernel<LQ_GATE_SCALAR, true>, nh, 64, smem, st, p);
-  else
-    rc = diag ? launch_persistent(decode_kernel<LQ_GATE_DIAG, false>, nh, 64, smem, st, p)
-              : launch_persistent(decode_kernel<LQ_GATE_SCALAR, false>, nh, 64, smem, st, p);
+  const bool longw = shape->W - 1 > REC_SEG;               // windows whose records come in more than one segment
+  if (longw) {
+    if (r16)
+      rc = diag ? launch_persistent(decode_kernel<LQ_GATE_DIAG, true, true>, nh, 64, smem, st, p)
+                : launch_persistent(decode_kernel<LQ_GATE_SCALAR, true, true>, nh, 64, smem, st, p);
+    else
+      rc = diag ? launch_persistent(decode_kernel<LQ_GATE_DIAG, false, true>, nh, 64, smem, st, p)
+                : launch_persistent(decode_kernel<LQ_GATE_SCALAR, false, true>, nh, 64, smem, st, p);
+  } else {
+    if (r16)
+      rc = diag ? launch_persistent(decode_kernel<LQ_GATE_DIAG, true, false>, nh, 64, smem, st, p)
+                : launch_persistent(decode_kernel<LQ_GATE_SCALAR, true, false>, nh, 64, smem, st, p);
+    else
+      rc = diag ? launch_persistent(decode_kernel<LQ_GATE_DIAG, false, false>, nh, 64, smem, st, p)
+                : launch_persistent(decode_kernel<LQ_GATE_SCALAR, false, false>, nh, 64, smem, st, p);
+  }
   if (rc != LQ_OK) return rc;
   if (between && cudaEventRecord(between, st) != cudaSuccess) {
     cudaGetLastError();

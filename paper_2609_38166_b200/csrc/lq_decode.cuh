@@ -40,8 +40,8 @@ namespace lq {
 // kernel's waits; bit 3: the wait of lq_selftest_bounded_wait).  Never cleared by kernels: lq_clear_device_flags.
 __device__ int g_device_error = 0;
 
-// Rows of the record buffer that a scalar-gate decode slot holds at a time (a multiple of four: the walk takes the
-// records four at a time from the newest back, so a group of four never straddles two segments).
+// Rows of the record buffer that a decode slot holds at a time (a multiple of four: the walk takes the records four
+// at a time from the newest back, so a group of four never straddles two segments).
 constexpr int REC_SEG = 32;                // (16 was tried: no faster at W = 32 or 64)
 
 // ---- shared-memory slot of one CTA ----
@@ -49,10 +49,10 @@ struct DecodeSlot {
   // byte offsets inside the slot; every region starts on a 16-byte boundary
   int head, rec, bas, digits, y, pk, pq, mbar, bytes;
   __host__ __device__ DecodeSlot(int W, int r, bool diag, bool rec16 = false) {
-    // a window holds at most W-1 records when a token arrives; with the scalar gate, where only the dot warp reads
-    // them, they are staged REC_SEG rows at a time (newest first), which keeps the slot small for long windows
+    // a window holds at most W-1 records when a token arrives; they are staged REC_SEG rows at a time (newest
+    // first), which keeps the slot small for long windows
     int rows = W > 1 ? W - 1 : 1;
-    if (!diag && rows > REC_SEG) rows = REC_SEG;
+    if (rows > REC_SEG) rows = REC_SEG;
     int o = 0;
     head = o; o += head_bytes(r);          // the head block: codes | col_scale | row_smooth | comp_k | comp_u
     rec = o; o += (rec16 ? 2 : 4) * record_floats(diag) * rows;   // buffered record rows (fp32 or fp16)
@@ -221,7 +221,9 @@ __device__ __forceinline__ void decode_slot_init(const Params &p, unsigned char 
 // PASS: 0 in the ordinary kernel; in the fused one 0 = the heads whose window fills with this token, 1 = the
 // others (two instances of the code: only the first carries the fences that publish a head to other CTAs, and a
 // fence anywhere in the loop costs every trip).  parA, parR: the phases of the two copy barriers, carried over.
-template <int GATE, bool R16, bool FUSED, int PASS>
+// LONGW: the window may hold more records than the slot stages at a time (W - 1 > REC_SEG); in the instances for
+// shorter windows everything to do with a second segment drops out at compile time.
+template <int GATE, bool R16, bool FUSED, int PASS, bool LONGW = true>
 __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot, const int lane, const int role,
                                             const int bar0, const unsigned first, const unsigned G,
                                             uint16_t *nbuf, uint32_t &parA, uint32_t &parR) {
@@ -270,8 +272,8 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
       else bulk_g2s_hint(slot_a + L.head, p.head(bh), head_bytes(r), barA, stream);
     }
   };
-  // first record of the segment that ends before record `hi` (everything from record 0 with the diagonal gate)
-  auto seg_base = [&](int hi) { return (!DIAG && hi > REC_SEG) ? hi - REC_SEG : 0; };
+  // first record of the segment that ends before record `hi`
+  auto seg_base = [&](int hi) { return (LONGW && hi > REC_SEG) ? hi - REC_SEG : 0; };
   // records [seg_base(hi), hi) of head bh, n of which are buffered in all, into the slot
   auto request_segment = [&](unsigned bh, int n, int hi) {
     if (lane == 0) {
@@ -412,23 +414,7 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
       }
       if (DIAG) wait_for(barR, parR);        // diagonal gate: Gamma_{1:l} is built from the records' decays
       // Compensator keys against Gamma_{1:l} k and Gamma_{1:l} q (the projections go to pk[h], pq[h]).
-      // g2 may have run past record 0 above: Gamma_{1:l} is taken from the exact chain.
-      if (r > 0) {
-        float2 gam[4];
-        if (DIAG) {
-#pragma unroll
-          for (int cc = 0; cc < 4; cc++) gam[cc] = a2[cc];
-#pragma unroll 4
-          for (int j = n - 1; j >= 0; j--) {
-            float2 aj[4];
-            load8p(rec + j * RF + REC_A + 8 * c, aj);
-#pragma unroll
-            for (int cc = 0; cc < 4; cc++) gam[cc] = __fmul2_rn(gam[cc], aj[cc]);
-          }
-        } else {
-#pragma unroll
-          for (int cc = 0; cc < 4; cc++) gam[cc] = pair(gsc);
-        }
+      auto project_compensators = [&](const float2 (&gam)[4]) {
         float2 gk2[4], gq2[4];
 #pragma unroll
         for (int cc = 0; cc < 4; cc++) { gk2[cc] = __fmul2_rn(gam[cc], k2[cc]); gq2[cc] = __fmul2_rn(gam[cc], q2[cc]); }
@@ -452,16 +438,41 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
           for (int u = 0; u < 2; u++)
             if (c == 0 && ho[u] < r) { pk[ho[u]] = s4[2 * u]; pq[ho[u]] = s4[2 * u + 1]; }
         }
+      };
+      // A head of the diagonal gate with more records than the slot holds at a time: Gamma_{1:l} is complete only
+      // after the walk over all segments, so its compensators are projected after the walk (and the head block is
+      // released that much later).  Otherwise first the projections, from a chain of their own over the decays.
+      const bool long_head = LONGW && DIAG && n > REC_SEG;
+      if (!long_head) {
+        if (r > 0) {
+          float2 gam[4];
+          if (DIAG) {
+#pragma unroll
+            for (int cc = 0; cc < 4; cc++) gam[cc] = a2[cc];
+#pragma unroll 4
+            for (int j = n - 1; j >= 0; j--) {
+              float2 aj[4];
+              load8p(rec + j * RF + REC_A + 8 * c, aj);
+#pragma unroll
+              for (int cc = 0; cc < 4; cc++) gam[cc] = __fmul2_rn(gam[cc], aj[cc]);
+            }
+          } else {
+#pragma unroll
+            for (int cc = 0; cc < 4; cc++) gam[cc] = pair(gsc);
+          }
+          project_compensators(gam);
+        }
+        __syncwarp();
+        named_arrive(bar0 + 3);                     // the compensator projections are in pk, pq; this warp is done with the head block
       }
-      __syncwarp();
-      named_arrive(bar0 + 3);                       // the compensator projections are in pk, pq; this warp is done with the head block
       LQ_TICK(4);
       if (!DIAG) wait_for(barR, parR);
       float rk_rec[4] = {0.0f, 0.0f, 0.0f, 0.0f}, rq_rec[4] = {0.0f, 0.0f, 0.0f, 0.0f};
       int base = seg_base(n);                        // the slot holds records base .. (row = record - base)
       for (int jt = n - 1; jt >= 0; jt -= 4) {       // records jt, jt-1, jt-2, jt-3
-        if (!DIAG && jt < base) {                    // the segment is walked: fetch the one before it
+        if (LONGW && jt < base) {                    // the segment is walked: fetch the one before it
           __syncwarp();
+          if (DIAG) named_wait(bar0 + 4);            // (the stream warp has taken this segment's decays as well)
           request_segment(bh, n, base);
           base = seg_base(base);
           wait_for(barR, parR);
@@ -473,9 +484,9 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
           // the decays of the two records of this pair; the half that owns the older one steps over the newer
           const int jn = jt - 2 * u, jold = jn - 1;  // newer, older
           float2 an[4], ao[4], gmine[4];
-          if (DIAG) {                                // (base = 0 with the diagonal gate)
-            load8p(rec + (jn > 0 ? jn : 0) * RF + REC_A + 8 * c, an);
-            load8p(rec + (jold > 0 ? jold : 0) * RF + REC_A + 8 * c, ao);
+          if (DIAG) {
+            load8p(rec + ((jn > 0 ? jn : 0) - base) * RF + REC_A + 8 * c, an);
+            load8p(rec + ((jold > 0 ? jold : 0) - base) * RF + REC_A + 8 * c, ao);
           } else {
             const float2 x = pair(bas[jn > 0 ? jn : 0]), z = pair(bas[jold > 0 ? jold : 0]);
 #pragma unroll
@@ -485,7 +496,9 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
           for (int cc = 0; cc < 4; cc++) {
             const float2 gn = g2[cc], go = __fmul2_rn(gn, an[cc]);   // Gamma_{jn+1:l}, Gamma_{jold+1:l}
             gmine[cc] = half ? go : gn;
-            g2[cc] = __fmul2_rn(go, ao[cc]);                          // past both records
+            // past both records; the chain stops at record 0, so that it ends as Gamma_{1:l} exactly
+            // (selects: a branch for the last trip of a long head was slower)
+            g2[cc] = (!LONGW || jold >= 0) ? __fmul2_rn(go, ao[cc]) : (jn >= 0 ? go : gn);
           }
           jo[u] = jn - half;
           const int j = jo[u] >= 0 ? jo[u] : 0;      // (record 0 is in the slot whenever an index runs below it)
@@ -520,6 +533,11 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
         }
       }
       LQ_TICK(3);
+      if (long_head) {                              // g2 is Gamma_{1:l} now
+        if (r > 0) project_compensators(g2);
+        __syncwarp();
+        named_arrive(bar0 + 3);
+      }
       if (DIAG) named_wait(bar0 + 4);               // diagonal gate: the stream warp read the records' decays too
       if (next_active) request_records(bh_next, n_next);
       named_wait(bar0 + 2);                         // the stream warp has taken its sums out of y
@@ -550,16 +568,21 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
 #pragma unroll
       for (int e = 0; e < 8; e++) gam[e] = a8[e];
       if (DIAG) {
-        wait_for(barR, parR);
+        for (int hi = n;;) {                        // segment after segment, in step with the dot warp
+          const int lo = seg_base(hi);
+          wait_for(barR, parR);
 #pragma unroll 2
-        for (int j = n - 1; j >= 0; j--) {
-          float aj[8];
-          load8(rec + j * RF + REC_A + 8 * c, aj);
+          for (int j = hi - 1; j >= lo; j--) {
+            float aj[8];
+            load8(rec + (j - lo) * RF + REC_A + 8 * c, aj);
 #pragma unroll
-          for (int e = 0; e < 8; e++) gam[e] = gam[e] * aj[e];
+            for (int e = 0; e < 8; e++) gam[e] = gam[e] * aj[e];
+          }
+          __syncwarp();
+          named_arrive(bar0 + 4);                   // this warp is done with the segment
+          if (lo == 0) break;
+          hi = lo;
         }
-        __syncwarp();
-        named_arrive(bar0 + 4);                     // this warp is done with the records
       } else {
 #pragma unroll
         for (int e = 0; e < 8; e++) gam[e] = gsc;
@@ -708,14 +731,14 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
 }
 
 // Persistent kernel of two-warp CTAs: CTA `blockIdx.x` takes heads blockIdx.x, blockIdx.x + gridDim.x, ...
-template <int GATE, bool R16>
+template <int GATE, bool R16, bool LONGW>
 __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
   extern __shared__ __align__(128) unsigned char lq_slot[];
   grid_dependency_wait();                    // no global memory is touched above this line
   const int lane = threadIdx.x & 31, role = threadIdx.x >> 5;
   uint32_t parA = 0, parR = 0;
   decode_slot_init<GATE, R16, false>(p, lq_slot, lane, role, 0, blockIdx.x, gridDim.x, nullptr);
-  decode_slot<GATE, R16, false, 0>(p, lq_slot, lane, role, 0, blockIdx.x, gridDim.x, nullptr, parA, parR);
+  decode_slot<GATE, R16, false, 0, LONGW>(p, lq_slot, lane, role, 0, blockIdx.x, gridDim.x, nullptr, parA, parR);
 }
 
 }  // namespace lq
