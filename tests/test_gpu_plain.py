@@ -80,9 +80,9 @@ class Tally:
                "code_mismatch_fraction": self.diff / max(self.entries, 1), "worst_code_difference": self.worst,
                "code_mismatch_fraction_in_flipped_heads": self.flipped_diff / max(self.flipped_entries, 1)}
         print("plain-definition parity:", json.dumps(row))
-        out = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "gpurun_out")
-        if os.path.isdir(out):
-            with open(os.path.join(out, "plain_parity.jsonl"), "a") as f:
+        report = os.environ.get("LQ_PARITY_REPORT")          # optional: a file to append the rows to
+        if report:
+            with open(report, "a") as f:
                 f.write(json.dumps(row) + "\n")
         assert self.same > 0, "no head with identical compensators: nothing was measured"
         assert self.diff <= 1e-4 * self.entries, row
