@@ -121,6 +121,15 @@ def test_staggered_batch_chain(oracle, gate, W, r):
 
 
 @pytest.mark.parametrize("gate", GATES)
+@pytest.mark.parametrize("r,n_iter", [(4, 2), (8, 3), (16, 2), (3, 4)])
+def test_chain_with_several_rounds_of_power_iteration(oracle, gate, r, n_iter):
+    # more than one round: the boundary kernel then also runs W = S^T T and its orthonormalisation between the passes;
+    # r = 8 and 16 take the instances of the kernel whose Cholesky factor is computed by a warp
+    wl = synth.Workload("iters", 5, 4, 2, W=8, r=r, n_iter=n_iter, gate=gate, seed=470 + r + n_iter)
+    _run_chain(oracle, wl, 2 * wl.W + 3, init="dense", stagger=True, check_every=4)
+
+
+@pytest.mark.parametrize("gate", GATES)
 def test_chain_without_the_delta_rule(oracle, gate):
     """b_t = 0 (Mamba2 / GLA style instances): u = v; decode, boundaries and both baseline kernels against the oracle."""
     wl = synth.Workload("nd", 5, 4, 2, W=4, r=2, gate=gate, seed=470, delta=0)
