@@ -325,13 +325,40 @@ def run_cuda(args, wl):
 
     for t in range(max(args.warmup, 3)):
         step(t)
+
+    # The timed steps are launched the way a serving loop launches a decode step: W consecutive steps captured once
+    # in a CUDA graph and replayed (every sequence passes exactly one window boundary per replay); steps beyond a
+    # multiple of W are plain launches.  --no-graph times plain launches only.
+    graph = None
+    if not args.no_graph and args.steps >= wl.W:
+        try:
+            gs = torch.cuda.Stream()
+            with torch.cuda.stream(gs):
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=gs):
+                    for t in range(wl.W):
+                        d = toks[t]
+                        lq.decode_step(sh, st, d["q"], d["k"], d["v"], d["beta"], d["alpha"], o, gs)
+            torch.cuda.synchronize()
+            graph.replay()                               # uploads the graph to the device (untimed)
+            torch.cuda.synchronize()
+        except Exception as exc:                         # reported, never hidden
+            log(f"CUDA-graph capture failed, timing plain launches: {exc!r}")
+            graph = None
+
+    def run_steps(k, use_graph=True):
+        reps = k // wl.W if (graph is not None and use_graph) else 0
+        for _ in range(reps):
+            graph.replay()
+        for t in range(reps * wl.W, k):
+            step(t)
+
     sampler = ClockSampler(local)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     sampler.start()
     ev0.record(stream)
-    for t in range(args.steps):
-        step(t)
+    run_steps(args.steps)
     ev1.record(stream)
     barrier()
     sampler.stop()
@@ -350,31 +377,17 @@ def run_cuda(args, wl):
         clock_source = "identical loop run right after the timed region (timed region shorter than the sampling period)"
     ms = max_over_ranks(ms, dist if world > 1 else None, "cuda")
 
-    # the same step captured in a CUDA graph (one graph = W steps), for the launch-overhead-free figure
-    graph_ms = None
-    try:
-        if args.only_timed:
-            raise RuntimeError("skipped (--only-timed)")
-        gstream = torch.cuda.Stream()
-        with torch.cuda.stream(gstream):
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g, stream=gstream):
-                for t in range(wl.W):
-                    d = toks[t]
-                    lq.decode_step(sh, st, d["q"], d["k"], d["v"], d["beta"], d["alpha"], o, gstream)
-            reps = max(args.steps // wl.W, 1)
-            for _ in range(3):
-                g.replay()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            torch.cuda.synchronize()
-            e0.record(gstream)
-            for _ in range(reps):
-                g.replay()
-            e1.record(gstream)
-            torch.cuda.synchronize()
-            graph_ms = e0.elapsed_time(e1) / (reps * wl.W)
-    except Exception as exc:                             # reported, never hidden
-        log(f"CUDA-graph timing failed: {exc!r}")
+    # the same K steps as plain launches (two kernel launches per step from the host), for comparison
+    plain_ms = None
+    if graph is not None and not args.only_timed:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(stream)
+        run_steps(args.steps, use_graph=False)
+        e1.record(stream)
+        barrier()
+        plain_ms = max_over_ranks(e0.elapsed_time(e1), dist if world > 1 else None, "cuda") / args.steps
+    graph_ms = ms / args.steps if graph is not None else None
 
     # end to end through the host-buffer entry point: inputs in pinned host memory, output read back
     e2e = None
@@ -515,7 +528,10 @@ def run_cuda(args, wl):
             "config": config_dict(wl, world), "warmup_tokens": args.warm_tokens,
             "tokens_heads_per_s": hs, "pct_hbm_peak_measured": 100 * achieved / peak,
             "pct_hbm_peak_nominal_8TBps": 100 * achieved / 8000.0,
-            "cuda_graph_ms_per_step": graph_ms, "gpu_launches": launches * args.steps,
+            "launch_mode": ("CUDA graph of W = %d steps replayed %d times + %d plain steps" %
+                            (wl.W, args.steps // wl.W, args.steps % wl.W)) if graph is not None else "plain launches",
+            "cuda_graph_ms_per_step": graph_ms, "plain_launch_ms_per_step": plain_ms,
+            "gpu_launches": launches * args.steps,
             "clocks": sampler.summary(clock_source), "roofline": roofline, "baselines": base,
             "e2e": e2e, "cpu_baseline": cpu}
     print(json.dumps(line), flush=True)
@@ -807,6 +823,7 @@ def main():
     ap.add_argument("--batch", type=int, default=256)
     ap.add_argument("--warm-tokens", type=int, default=WARM_TOKENS,
                     help="tokens of the fp32 recurrence that pre-fill the states (512 in the headline workload)")
+    ap.add_argument("--no-graph", action="store_true", help="time plain launches instead of CUDA-graph replays")
     ap.add_argument("--only-timed", action="store_true",
                     help="skip the CUDA-graph, end-to-end, baseline-kernel and CPU legs (for profiler runs)")
     ap.add_argument("--r", type=int, default=4, help="Compensator Tokens per state")
