@@ -55,7 +55,7 @@ NCU_TRAFFIC_BYTES_PER_LAUNCH = {"decode_kernel": 235.0e6, "boundary_kernel": 18.
 # The same two counters from a launch list taken with --cache-control none (the caches are left as the kernel ahead
 # left them, as in a real step): what the L2 serves - the records written by the last tokens, the token vectors, and
 # for the boundary kernel the heads the decode kernel asked the L2 to keep - no longer comes from DRAM.
-NCU_TRAFFIC_WARM_BYTES_PER_LAUNCH = {"decode_kernel": 198.9e6, "boundary_kernel": 1.3e6}
+NCU_TRAFFIC_WARM_BYTES_PER_LAUNCH = {"decode_kernel": 194.5e6, "boundary_kernel": 1.4e6}
 
 
 def record_bytes(diag: bool, rec16: int) -> int:
