@@ -49,6 +49,10 @@ __global__ void __launch_bounds__(256, 2) boundary_kernel(const Params p, const 
       const uint32_t m = __ballot_sync(FULL, want);
       todo_n[t.lane] = n_mine > p.W ? p.W : n_mine;
       if (t.lane == 0) todo_mask = m;
+      // The arrival on win_pos (arrive_and_set: the last head of a sequence to arrive stores 0) only says "this head
+      // has read the old value", which it just did; nobody inside this kernel waits for the 0.  Made here, 32 heads
+      // at once, the atomic's round trip hides behind the wait for the first staging buffer.
+      if (MODE == 0 && want) arrive_and_set(p.win_pos, static_cast<int>(cand / p.heads_v), p.heads_v, 0);
     }
     __syncthreads();
     LQ_BTICK(0);
@@ -97,10 +101,7 @@ __global__ void __launch_bounds__(256, 2) boundary_kernel(const Params p, const 
       }
       __syncthreads();                       // this head's use of shared memory is over
       LQ_BTICK(9);
-      if (MODE != 2 && t.tid == 0) {
-        if (MODE == 0) arrive_and_set(p.win_pos, b, p.heads_v, 0);
-        else p.win_pos[b] = 0;               // nobody reads win_pos in this mode
-      }
+      if (MODE == 1 && t.tid == 0) p.win_pos[b] = 0;      // (nobody reads win_pos in this mode)
       if (staged) buf ^= 1;
     }
     __syncthreads();                         // todo_mask / todo_n are rewritten by the next round
