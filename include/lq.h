@@ -246,6 +246,37 @@ lq_status lq_quantize_state(const lq_shape *shape, const float *S, const lq_stat
 lq_status lq_dequantize_state(const lq_shape *shape, const lq_state *state, float *S, lq_stream stream);
 
 /*
+ * The window representation as separate arrays in the paper's notation and orientation (Sec. 3.1: S is d_k x d_v;
+ * Appendix B.3 for Z and B; Sec. 3.4 for c; Sec. 3.3 for the compensators; Eq. 3 for the records), for callers
+ * that hold or want the state that way instead of in the packed head blocks above.  All arrays dense, row-major,
+ * device memory, 16-byte aligned:
+ *   codes      int8 [B,Hv,d_k,d_v]   Z (NOT transposed)
+ *   col_scale  fp32 [B,Hv,d_v]       step of the code per value channel, B_j / 127
+ *   row_smooth fp32 [B,Hv,d_k]       c
+ *   comp_k     fp16 [B,Hv,r,d_k]     comp_u  fp16 [B,Hv,r,d_v]      (null when r = 0)
+ *   buf_k      fp32 [B,Hv,W,d_k]     write keys beta*k of the buffered records
+ *   buf_u      fp32 [B,Hv,W,d_v]     corrections u
+ *   buf_a      fp32 [B,Hv,W] (scalar gate) or [B,Hv,W,d_k] (diagonal gate): the records' decays
+ *   win_pos    int32 [B]
+ * lq_import_state fills `dst` from the arrays, lq_export_state the arrays from `src`; both copy all W record
+ * slots whatever win_pos says.  With shape.rec16 the records are narrowed to fp16 on import (nearest even,
+ * saturating) and widened on export.  Not available with shape.state_bf16 (LQ_ERR_UNSUPPORTED).
+ */
+typedef struct {
+  int8_t *codes;
+  float *col_scale;
+  float *row_smooth;
+  uint16_t *comp_k;
+  uint16_t *comp_u;
+  float *buf_k;
+  float *buf_u;
+  float *buf_a;
+  int32_t *win_pos;
+} lq_state_arrays;
+lq_status lq_import_state(const lq_shape *shape, const lq_state_arrays *src, const lq_state *dst, lq_stream stream);
+lq_status lq_export_state(const lq_shape *shape, const lq_state *src, const lq_state_arrays *dst, lq_stream stream);
+
+/*
  * Speed and accuracy baselines: the same token on an unquantized dense state (Eq. 1 with the GDN / KDA
  * coefficients of Table 4), read and written in full every token.  S is [B,Hv,d_k,d_v], fp32 or bf16
  * (rounded to nearest even after every token, the "BF16 per-step" setting); o is computed from the

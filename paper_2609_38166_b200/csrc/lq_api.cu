@@ -188,6 +188,71 @@ __global__ void __launch_bounds__(256, (BF16 || GATE == LQ_GATE_SCALAR) ? 3 : 2)
 }
 
 // ---------------------------------------------------------------------------------------------
+// The window representation as separate arrays in the paper's orientation <-> the packed layout of lq_state
+// (lq_import_state / lq_export_state): pure data movement, one CTA per head.
+// ---------------------------------------------------------------------------------------------
+template <bool IMPORT>
+__global__ void __launch_bounds__(256) convert_state_kernel(const Params p, const lq_state_arrays a, const int diag) {
+  __shared__ __align__(16) int8_t tile[D][D + 16];            // the code matrix on its way through the transposition
+  const size_t bh = blockIdx.x;
+  const int tid = threadIdx.x, W = p.W, r = p.r;
+  const int b = static_cast<int>(bh / p.heads_v), hv = static_cast<int>(bh % p.heads_v);
+  int8_t *Z = a.codes + bh * (size_t)(D * D);                 // [d_k][d_v]
+  int8_t *ZT = p.codes(bh);                                   // [d_v][d_k]
+  const int8_t *src = IMPORT ? Z : ZT;
+  int8_t *dst = IMPORT ? ZT : Z;
+  for (int e = tid; e < D * D / 16; e += 256) {
+    const int row = e >> 3, c16 = e & 7;
+    *reinterpret_cast<uint4 *>(&tile[row][16 * c16]) = *reinterpret_cast<const uint4 *>(src + row * D + 16 * c16);
+  }
+  __syncthreads();
+  for (int e = tid; e < D * D / 16; e += 256) {
+    const int row = e >> 3, c16 = e & 7;
+    uint32_t w[4];
+#pragma unroll
+    for (int q = 0; q < 4; q++) {
+      uint32_t x = 0;
+#pragma unroll
+      for (int j = 0; j < 4; j++) x |= static_cast<uint32_t>(static_cast<uint8_t>(tile[16 * c16 + 4 * q + j][row])) << (8 * j);
+      w[q] = x;
+    }
+    *reinterpret_cast<uint4 *>(dst + row * D + 16 * c16) = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+  auto move = [&](auto *packed, auto *plain) {
+    if (IMPORT) *packed = *plain;
+    else *plain = *packed;
+  };
+  if (tid < D) {
+    move(p.col_scale(bh) + tid, a.col_scale + bh * D + tid);
+    move(p.row_smooth(bh) + tid, a.row_smooth + bh * D + tid);
+  }
+  for (int e = tid; e < r * D; e += 256) {
+    move(p.comp_k(bh) + e, a.comp_k + bh * (size_t)(r * D) + e);
+    move(p.comp_u(bh) + e, a.comp_u + bh * (size_t)(r * D) + e);
+  }
+  const int RF = record_floats(diag != 0);
+  auto move_record = [&](int j, int off, float *plain) {       // one element of record j, fp32 or fp16 in the packed rows
+    if (p.rec16) {
+      __half *row = p.record<__half>(bh, j, diag != 0);
+      if (IMPORT) row[off] = __ushort_as_half(to_f16_bits_sat(*plain));
+      else *plain = __half2float(row[off]);
+    } else {
+      float *row = p.record<float>(bh, j, diag != 0);
+      if (IMPORT) row[off] = *plain;
+      else *plain = row[off];
+    }
+  };
+  for (int e = tid; e < W * D; e += 256) {
+    const int j = e / D, i = e % D;
+    move_record(j, REC_KT + i, a.buf_k + (bh * W + j) * (size_t)D + i);
+    move_record(j, REC_U + i, a.buf_u + (bh * W + j) * (size_t)D + i);
+    if (diag) move_record(j, REC_A + i, a.buf_a + (bh * W + j) * (size_t)D + i);
+  }
+  if (!diag && tid < W) move(p.decays + bh * (size_t)W + tid, a.buf_a + bh * (size_t)W + tid);
+  if (hv == 0 && tid == 0) move(p.win_pos + b, a.win_pos + b);
+}
+
+// ---------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------
 static bool aligned16(const void *ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15u) == 0; }
@@ -928,6 +993,34 @@ lq_status lq_ref_decode_step_bf16(const lq_shape *shape, uint16_t *S, const uint
   return ref_step(shape, nullptr, S, q, k, v, beta, alpha, o, stream);
 }
 
+static lq_status convert_state(const lq_shape *shape, const lq_state_arrays *arr, const lq_state *state, lq_stream stream,
+                               bool import) {
+  lq_status rc = check_shape(shape);
+  if (rc != LQ_OK) return rc;
+  if (shape->state_bf16) return LQ_ERR_UNSUPPORTED;
+  if ((rc = check_state(shape, state, true)) != LQ_OK) return rc;
+  if (!arr) return LQ_ERR_NULL;
+  if ((rc = check_ptrs({arr->codes, arr->col_scale, arr->row_smooth, arr->buf_k, arr->buf_u, arr->buf_a})) != LQ_OK) return rc;
+  if (shape->r > 0 && (rc = check_ptrs({arr->comp_k, arr->comp_u})) != LQ_OK) return rc;
+  if ((rc = check_scalar_ptrs({arr->win_pos}, 4)) != LQ_OK) return rc;
+  Params p = make_params(shape, state);
+  const int nh = shape->batch * shape->heads_v;
+  const int diag = shape->gate == LQ_GATE_DIAG ? 1 : 0;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (nh <= 0) return LQ_OK;
+  if (import) convert_state_kernel<true><<<nh, 256, 0, st>>>(p, *arr, diag);
+  else convert_state_kernel<false><<<nh, 256, 0, st>>>(p, *arr, diag);
+  return cudaGetLastError() == cudaSuccess ? LQ_OK : LQ_ERR_CUDA;
+}
+
+lq_status lq_import_state(const lq_shape *shape, const lq_state_arrays *src, const lq_state *dst, lq_stream stream) {
+  return convert_state(shape, src, dst, stream, true);
+}
+
+lq_status lq_export_state(const lq_shape *shape, const lq_state *src, const lq_state_arrays *dst, lq_stream stream) {
+  return convert_state(shape, dst, src, stream, false);
+}
+
 lq_status lq_check_device(int *flags) {
   if (!flags) return LQ_ERR_NULL;
   int v = 0;
@@ -996,6 +1089,6 @@ const char *lq_status_string(lq_status status) {
   return "unknown status";
 }
 
-int lq_version(void) { return 5; }
+int lq_version(void) { return 6; }
 
 }  // extern "C"

@@ -23,7 +23,7 @@ EXPORTS = ["lq_decode_step", "lq_decode_step_profiled", "lq_decode_step_host", "
            "lq_window_flush",
            "lq_quantize_state", "lq_dequantize_state", "lq_ref_decode_step_f32", "lq_ref_decode_step_bf16",
            "lq_decode_launches", "lq_check_device", "lq_clear_device_flags", "lq_selftest_bounded_wait",
-           "lq_static_stage_bytes", "lq_status_string", "lq_version"]
+           "lq_static_stage_bytes", "lq_import_state", "lq_export_state", "lq_status_string", "lq_version"]
 
 
 class LqError(RuntimeError):
@@ -62,6 +62,8 @@ def lib() -> C.CDLL:
         L.lq_clear_device_flags.argtypes = []
         L.lq_selftest_bounded_wait.restype = C.c_int
         L.lq_selftest_bounded_wait.argtypes = [C.c_void_p]
+        for name in ("lq_import_state", "lq_export_state"):
+            getattr(L, name).restype = C.c_int
         for name in ("lq_decode_step", "lq_decode_step_profiled", "lq_decode_step_host", "lq_decode_step_host_pipelined",
                      "lq_decode_step_host_static", "lq_check_device", "lq_window_flush", "lq_quantize_state",
                      "lq_dequantize_state", "lq_ref_decode_step_f32", "lq_ref_decode_step_bf16"):
@@ -283,6 +285,47 @@ def check_device() -> int:
     flags = C.c_int(0)
     _check(lib().lq_check_device(C.byref(flags)), "lq_check_device")
     return int(flags.value)
+
+
+class _StateArrays(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in
+                ("codes", "col_scale", "row_smooth", "comp_k", "comp_u", "buf_k", "buf_u", "buf_a", "win_pos")]
+
+
+class StateArrays:
+    """The window representation as separate device tensors in the paper's orientation (``lq_state_arrays``):
+    codes int8 [B,Hv,d_k,d_v], col_scale / row_smooth fp32, comp_k / comp_u fp16, buf_k / buf_u / buf_a fp32,
+    win_pos int32 [B]."""
+
+    def __init__(self, sh: Shape, device="cuda"):
+        B, H, K, V, W, r = sh.batch, sh.heads_v, sh.d_k, sh.d_v, sh.W, sh.r
+        z = lambda shape, dt: torch.zeros(shape, dtype=dt, device=device)
+        self.codes = z((B, H, K, V), torch.int8)
+        self.col_scale = z((B, H, V), torch.float32)
+        self.row_smooth = z((B, H, K), torch.float32)
+        self.comp_k = z((B, H, r, K), torch.float16)
+        self.comp_u = z((B, H, r, V), torch.float16)
+        self.buf_k = z((B, H, W, K), torch.float32)
+        self.buf_u = z((B, H, W, V), torch.float32)
+        self.buf_a = z((B, H, W, K) if sh.gate == GATE_DIAG else (B, H, W), torch.float32)
+        self.win_pos = z((B,), torch.int32)
+
+    def c(self) -> _StateArrays:
+        ptr = lambda t: t.data_ptr() if t.numel() else None
+        return _StateArrays(ptr(self.codes), ptr(self.col_scale), ptr(self.row_smooth), ptr(self.comp_k), ptr(self.comp_u),
+                            ptr(self.buf_k), ptr(self.buf_u), ptr(self.buf_a), ptr(self.win_pos))
+
+
+def import_state(sh: Shape, arrays: StateArrays, st: State, stream=None) -> None:
+    """lq_import_state: fill the packed state from the separate arrays."""
+    s, a, cs = sh.c(), arrays.c(), st.c()
+    _check(lib().lq_import_state(C.byref(s), C.byref(a), C.byref(cs), _stream(stream)), "lq_import_state")
+
+
+def export_state(sh: Shape, st: State, arrays: StateArrays, stream=None) -> None:
+    """lq_export_state: write the packed state out as separate arrays."""
+    s, a, cs = sh.c(), arrays.c(), st.c()
+    _check(lib().lq_export_state(C.byref(s), C.byref(cs), C.byref(a), _stream(stream)), "lq_export_state")
 
 
 def clear_device_flags() -> None:

@@ -71,6 +71,13 @@ def test_argument_errors_are_reported_before_any_launch(L):
     assert L.lq_decode_step_host(C.byref(s), C.byref(st_bad), hp, hp, hp, hp, hp, hp, hp, null) == 3
     assert L.lq_decode_step_host_static(C.byref(s), C.byref(st), hp, hp, hp, hp, hp, hp, null) == 1
     assert L.lq_decode_step_host_static(C.byref(s), C.byref(st_bad), hp, hp, hp, hp, hp, hp, null) == 3
+    # import / export of the separate-array form: null struct, null arrays, a state with a misaligned pointer
+    arr = lq._StateArrays(*([None] * 9))
+    assert L.lq_import_state(C.byref(s), null, C.byref(st_ok), null) == 1
+    assert L.lq_import_state(C.byref(s), C.byref(arr), C.byref(st_ok), null) == 1
+    assert L.lq_export_state(C.byref(s), C.byref(st_bad), C.byref(arr), null) == 3
+    w16 = lq.Shape(2, 4, 2, r=0, smooth=0, state_bf16=1).c()
+    assert L.lq_import_state(C.byref(w16), C.byref(arr), C.byref(st_ok), null) == 4
     big = lq.Shape(64, 32, 16).c()                                # (the pipelined path proper starts at 16 sequences)
     assert L.lq_decode_step_host_pipelined(C.byref(big), C.byref(st_bad), hp, hp, hp, hp, hp, hp, hp, null) == 3
     assert lq.decode_stage_bytes(sh) > 0 and lq.decode_launches(sh) >= 1

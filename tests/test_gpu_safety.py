@@ -139,3 +139,40 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable():
     lq.decode_step(sh, st, td["q"], td["k"], td["v"], td["beta"], td["alpha"], o)
     torch.cuda.synchronize()
     assert lq.check_device() == 0 and bool(torch.isfinite(o).all())
+
+
+@pytest.mark.parametrize("gate", [synth.GATE_SCALAR, synth.GATE_DIAG])
+@pytest.mark.parametrize("rec16", [0, 1])
+def test_import_and_export_of_the_separate_array_form(oracle, gate, rec16):
+    """A state built by the oracle (the paper's orientation: Z not transposed, one array per piece) is imported into
+    the packed layout; decoding from it must give the oracle's outputs bit for bit, and exporting the result must
+    give back the oracle's arrays."""
+    from oracle.lq_oracle import State as OState
+    wl = synth.Workload("imp", 3, 4, 2, W=8, r=4, gate=gate, rec16=rec16, seed=1200 + gate + 2 * rec16)
+    osh, sh = gu.shapes(wl)
+    ost = OState(osh)
+    oracle.quantize_state(osh, synth.dense_states(wl, 4), ost)
+    for step in range(5):                                        # five records in the buffer
+        oracle.decode_step(osh, ost, **synth.token_inputs(wl, step))
+    arr = lq.StateArrays(sh)
+    for name in ("codes", "col_scale", "row_smooth", "buf_k", "buf_u", "buf_a", "win_pos"):
+        getattr(arr, name).copy_(gu.dev(getattr(ost, name)))
+    arr.comp_k.copy_(gu.dev(ost.comp_k).view(torch.float16)); arr.comp_u.copy_(gu.dev(ost.comp_u).view(torch.float16))
+    st = lq.State(sh)
+    lq.import_state(sh, arr, st)
+    o = torch.empty((wl.batch, wl.heads_v, 128), dtype=torch.float32, device="cuda")
+    for step in range(5, 5 + wl.W + 2):                          # through a boundary
+        tok = synth.token_inputs(wl, step)
+        td = gu.tok_dev(tok)
+        want = oracle.decode_step(osh, ost, **tok)
+        lq.decode_step(sh, st, td["q"], td["k"], td["v"], td["beta"], td["alpha"], o)
+        assert np.array_equal(gu.host(o), want), step
+    out = lq.StateArrays(sh)
+    lq.export_state(sh, st, out)
+    torch.cuda.synchronize()
+    n = int(ost.win_pos[0])
+    assert np.array_equal(gu.host(out.codes), ost.codes) and np.array_equal(gu.host(out.win_pos), ost.win_pos)
+    assert np.array_equal(gu.host(out.col_scale), ost.col_scale) and np.array_equal(gu.host(out.row_smooth), ost.row_smooth)
+    assert np.array_equal(gu.host(out.comp_k), ost.comp_k) and np.array_equal(gu.host(out.comp_u), ost.comp_u)
+    for name in ("buf_k", "buf_u", "buf_a"):                     # the live records
+        assert np.array_equal(gu.host(getattr(out, name))[:, :, :n], getattr(ost, name)[:, :, :n]), name
