@@ -392,8 +392,9 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
     }
     LQ_TICK(1);
 
-    // ---- wait for the head block; the records are waited for where they are first needed ----
-    wait_for(barA, parA);
+    // ---- the stream warp waits for the head block; the dot warp first takes the records, which it asked for
+    // earlier and which need nothing from the head block, and waits for the block when it gets to the compensators ----
+    if (role == 0 && !DIAG) wait_for(barA, parA);  // (diagonal gate: after its own walk of the records' decays)
     LQ_TICK(2);
 
     if (role == 1) {
@@ -412,7 +413,7 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
         g2[cc] = a2[cc];
         kt2[cc] = __fmul2_rn(pair(beta), k2[cc]);
       }
-      if (DIAG) wait_for(barR, parR);        // diagonal gate: Gamma_{1:l} is built from the records' decays
+      wait_for(barR, parR);                  // the newest segment of the records
       // Compensator keys against Gamma_{1:l} k and Gamma_{1:l} q (the projections go to pk[h], pq[h]).
       auto project_compensators = [&](const float2 (&gam)[4]) {
         float2 gk2[4], gq2[4];
@@ -439,34 +440,6 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
             if (c == 0 && ho[u] < r) { pk[ho[u]] = s4[2 * u]; pq[ho[u]] = s4[2 * u + 1]; }
         }
       };
-      // A head of the diagonal gate with more records than the slot holds at a time: Gamma_{1:l} is complete only
-      // after the walk over all segments, so its compensators are projected after the walk (and the head block is
-      // released that much later).  Otherwise first the projections, from a chain of their own over the decays.
-      const bool long_head = LONGW && DIAG && n > REC_SEG;
-      if (!long_head) {
-        if (r > 0) {
-          float2 gam[4];
-          if (DIAG) {
-#pragma unroll
-            for (int cc = 0; cc < 4; cc++) gam[cc] = a2[cc];
-#pragma unroll 4
-            for (int j = n - 1; j >= 0; j--) {
-              float2 aj[4];
-              load8p(rec + j * RF + REC_A + 8 * c, aj);
-#pragma unroll
-              for (int cc = 0; cc < 4; cc++) gam[cc] = __fmul2_rn(gam[cc], aj[cc]);
-            }
-          } else {
-#pragma unroll
-            for (int cc = 0; cc < 4; cc++) gam[cc] = pair(gsc);
-          }
-          project_compensators(gam);
-        }
-        __syncwarp();
-        named_arrive(bar0 + 3);                     // the compensator projections are in pk, pq; this warp is done with the head block
-      }
-      LQ_TICK(4);
-      if (!DIAG) wait_for(barR, parR);
       float rk_rec[4] = {0.0f, 0.0f, 0.0f, 0.0f}, rq_rec[4] = {0.0f, 0.0f, 0.0f, 0.0f};
       int base = seg_base(n);                        // the slot holds records base .. (row = record - base)
       for (int jt = n - 1; jt >= 0; jt -= 4) {       // records jt, jt-1, jt-2, jt-3
@@ -498,7 +471,7 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
             gmine[cc] = half ? go : gn;
             // past both records; the chain stops at record 0, so that it ends as Gamma_{1:l} exactly
             // (selects: a branch for the last trip of a long head was slower)
-            g2[cc] = (!LONGW || jold >= 0) ? __fmul2_rn(go, ao[cc]) : (jn >= 0 ? go : gn);
+            g2[cc] = (!DIAG || jold >= 0) ? __fmul2_rn(go, ao[cc]) : (jn >= 0 ? go : gn);
           }
           jo[u] = jn - half;
           const int j = jo[u] >= 0 ? jo[u] : 0;      // (record 0 is in the slot whenever an index runs below it)
@@ -533,11 +506,22 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
         }
       }
       LQ_TICK(3);
-      if (long_head) {                              // g2 is Gamma_{1:l} now
-        if (r > 0) project_compensators(g2);
-        __syncwarp();
-        named_arrive(bar0 + 3);
+      // Now the head block: the compensators are projected with Gamma_{1:l}, which for the diagonal gate is where
+      // the walk's chain of decays has arrived (g2), for the scalar gate the product taken before the wait.
+      wait_for(barA, parA);
+      if (r > 0) {
+        if (DIAG) {
+          project_compensators(g2);
+        } else {
+          float2 gam[4];
+#pragma unroll
+          for (int cc = 0; cc < 4; cc++) gam[cc] = pair(gsc);
+          project_compensators(gam);
+        }
       }
+      __syncwarp();
+      named_arrive(bar0 + 3);                       // the compensator projections are in pk, pq; this warp is done with the head block
+      LQ_TICK(4);
       if (DIAG) named_wait(bar0 + 4);               // diagonal gate: the stream warp read the records' decays too
       if (next_active) request_records(bh_next, n_next);
       named_wait(bar0 + 2);                         // the stream warp has taken its sums out of y
@@ -583,6 +567,7 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
           if (lo == 0) break;
           hi = lo;
         }
+        wait_for(barA, parA);
       } else {
 #pragma unroll
         for (int e = 0; e < 8; e++) gam[e] = gsc;
