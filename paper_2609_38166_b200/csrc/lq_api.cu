@@ -30,9 +30,12 @@ __global__ void __launch_bounds__(256, 2) boundary_kernel(const Params p, const 
   const size_t nh = (size_t)p.batch * p.heads_v;
   __shared__ uint32_t todo_mask;
   __shared__ int todo_n[32];
+  LQ_STAMP(1, 0);
   grid_dependency_wait();                    // everything the kernel before this one wrote is visible from here on
+  LQ_STAMP(1, 1);
 #ifdef LQ_TIMING
   if (threadIdx.x == 0) { for (int i = 0; i < 16; i++) lq_bacc[i] = 0; lq_btick = clock64(); }
+  bool first_flush_ = true;
 #endif
   // The CTA owns heads blockIdx.x + k * gridDim.x.  Warp 0 looks at 32 of them at a time (one load each, all in
   // flight together) and publishes which ones have work and how many records each holds; then the CTA takes
@@ -90,6 +93,9 @@ __global__ void __launch_bounds__(256, 2) boundary_kernel(const Params p, const 
         }
         __syncthreads();
         LQ_BTICK(1);
+#ifdef LQ_TIMING
+        if (first_flush_) LQ_STAMP(1, 2);
+#endif
         reconstruct_tile<GATE, R16>(p, sm, t, bh, n, M);
       }
       if (MODE == 2) {
@@ -101,12 +107,17 @@ __global__ void __launch_bounds__(256, 2) boundary_kernel(const Params p, const 
       }
       __syncthreads();                       // this head's use of shared memory is over
       LQ_BTICK(9);
+#ifdef LQ_TIMING
+      if (first_flush_) LQ_STAMP(1, 3);
+      first_flush_ = false;
+#endif
       if (MODE == 1 && t.tid == 0) p.win_pos[b] = 0;      // (nobody reads win_pos in this mode)
       if (staged) buf ^= 1;
     }
     __syncthreads();                         // todo_mask / todo_n are rewritten by the next round
   }
 #ifdef LQ_TIMING
+  LQ_STAMP(1, 4);
   if (threadIdx.x == 0) {
     for (int i = 0; i < 16; i++) atomicAdd(&g_phase_cycles[32 + i], (unsigned long long)lq_bacc[i]);
   }
@@ -396,7 +407,7 @@ static lq_status launch_dependent(K kernel, int grid, int block, size_t smem, cu
   return LQ_OK;
 }
 
-// grid = min(work items, CTAs that fit on the device at once), for kernels that stride over their work
+// grid <= min(work items, CTAs that fit on the device at once), for kernels that stride over their work
 template <typename K>
 static lq_status launch_persistent(K kernel, long items, int block, size_t smem, cudaStream_t stream, const Params &p) {
   if (items <= 0) return LQ_OK;
@@ -404,7 +415,12 @@ static lq_status launch_persistent(K kernel, long items, int block, size_t smem,
   const int per_sm = ctas_per_sm(reinterpret_cast<const void *>(kernel), block, smem);
   if (per_sm < 1) return LQ_ERR_CUDA;
   const long resident = (long)per_sm * sm_count();
-  return launch_dependent(kernel, static_cast<int>(items < resident ? items : resident), block, smem, stream, p);
+  // every CTA takes ceil(items / resident) items at most; the smallest grid with that property leaves no last
+  // round in which a fraction of the CTAs works while the others have left (8192 heads: 820 CTAs of 10 heads
+  // instead of 888 of which 200 take a tenth)
+  const long rounds = (items + resident - 1) / resident;
+  const long grid = (items + rounds - 1) / rounds;
+  return launch_dependent(kernel, static_cast<int>(grid), block, smem, stream, p);
 }
 
 // per-window BF16: persistent CTAs that stride over the heads
@@ -508,6 +524,10 @@ static lq_status decode_step_impl(const lq_shape *shape, const lq_state *state, 
   if ((rc = check_scalar_ptrs({beta}, 2)) != LQ_OK) return rc;
   if ((rc = shape->gate == LQ_GATE_DIAG ? check_ptrs({alpha}) : check_scalar_ptrs({alpha}, 2)) != LQ_OK) return rc;
   Params p = make_params(shape, state);
+#ifdef LQ_TIMING
+  static int generation = 0;
+  p.gen = generation++;
+#endif
   p.q = q; p.k = k; p.v = v; p.beta = beta; p.alpha = alpha; p.o = o;
   const bool diag = shape->gate == LQ_GATE_DIAG;
   const long nh = (long)shape->batch * shape->heads_v;
@@ -1066,6 +1086,10 @@ lq_status lq_selftest_bounded_wait(lq_stream stream) {
 }
 
 #ifdef LQ_TIMING
+// development aid: copies the time stamps of the last four steps to host memory (4 x 2 x 6 x 1024 values)
+int lq_debug_timeline(unsigned long long *out) {
+  return cudaMemcpyFromSymbol(out, g_timeline, sizeof(unsigned long long) * 4 * 2 * 6 * 1024) != cudaSuccess;
+}
 // development aid: copies the phase counters to host memory and clears them
 int lq_debug_phase_cycles(unsigned long long *out) {
   unsigned long long zero[64] = {0};

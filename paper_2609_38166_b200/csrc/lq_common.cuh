@@ -44,6 +44,9 @@ struct Params {
   float *o;
   float *S;          // dense fp32 states (quantize / dequantize / fp32 baseline)
   uint16_t *S16;     // dense bf16 states (bf16 baseline)
+#ifdef LQ_TIMING
+  int gen;           // development aid: which of the four generations of time stamps this launch writes
+#endif
 
   __device__ __forceinline__ uint8_t *head(size_t bh) const { return heads + bh * (size_t)head_bytes(r); }
   __device__ __forceinline__ int8_t *codes(size_t bh) const { return reinterpret_cast<int8_t *>(head(bh) + HB_CODES); }
@@ -167,9 +170,20 @@ __shared__ long long lq_btick;
       lq_btick = now_;                                          \
     }                                                           \
   } while (0)
+// time stamps (ns, the GPU's global timer) of thread 0 of every CTA: [generation][kernel][stamp][CTA]
+__device__ unsigned long long g_timeline[4][2][6][1024];
+#define LQ_STAMP(kernel, slot)                                                                   \
+  do {                                                                                           \
+    if (threadIdx.x == 0 && blockIdx.x < 1024) {                                                 \
+      unsigned long long t_;                                                                     \
+      asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_));                                      \
+      g_timeline[p.gen & 3][kernel][slot][blockIdx.x] = t_;                                      \
+    }                                                                                            \
+  } while (0)
 #else
 #define LQ_TICK(slot) do { } while (0)
 #define LQ_BTICK(slot) do { } while (0)
+#define LQ_STAMP(kernel, slot) do { } while (0)
 #endif
 
 // =====================================================================================

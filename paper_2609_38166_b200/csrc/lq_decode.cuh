@@ -396,6 +396,7 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
     // earlier and which need nothing from the head block, and waits for the block when it gets to the compensators ----
     if (role == 0 && !DIAG) wait_for(barA, parA);  // (diagonal gate: after its own walk of the records' decays)
     LQ_TICK(2);
+    if (idx == 0) LQ_STAMP(0, 2);
 
     if (role == 1) {
       // =========================== DOT WARP ===========================
@@ -719,7 +720,9 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
 template <int GATE, bool R16, bool LONGW>
 __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
   extern __shared__ __align__(128) unsigned char lq_slot[];
+  LQ_STAMP(0, 0);
   grid_dependency_wait();                    // no global memory is touched above this line
+  LQ_STAMP(0, 1);
   const int lane = threadIdx.x & 31, role = threadIdx.x >> 5;
   uint32_t parA = 0, parR = 0;
   decode_slot_init<GATE, R16, false>(p, lq_slot, lane, role, 0, blockIdx.x, gridDim.x, nullptr);
