@@ -253,6 +253,9 @@ def run_reference(args, wl):
 # --------------------------------------------------------------------------------------------------
 # CUDA arm
 # --------------------------------------------------------------------------------------------------
+BOUNDARY_QUEUE = True     # --no-queue: states without lq_state.work (the boundary kernel starts after the decode kernel)
+
+
 def to_dev(tok, torch):
     return {k: torch.from_numpy(v.view(np.int16)).cuda(non_blocking=False) for k, v in tok.items()}
 
@@ -263,7 +266,7 @@ def prepare_state(wl, lq, torch, log, WARM_TOKENS=WARM_TOKENS):
     sh = lq.Shape(wl.batch, wl.heads_v, wl.heads_qk, wl.d_k, wl.d_v, wl.W, wl.r, wl.n_iter, wl.gate, wl.smooth, wl.delta,
                   wl.rec16, wl.state_bf16)
     B, W = wl.batch, wl.W
-    st = lq.State(sh)
+    st = lq.State(sh, queue=BOUNDARY_QUEUE)
     S = torch.zeros((B, wl.heads_v, wl.d_k, wl.d_v), dtype=torch.float32, device="cuda")
     o = torch.empty((B, wl.heads_v, wl.d_v), dtype=torch.float32, device="cuda")
     per = max(B // W, 1)
@@ -824,6 +827,8 @@ def main():
     ap.add_argument("--warm-tokens", type=int, default=WARM_TOKENS,
                     help="tokens of the fp32 recurrence that pre-fill the states (512 in the headline workload)")
     ap.add_argument("--no-graph", action="store_true", help="time plain launches instead of CUDA-graph replays")
+    ap.add_argument("--no-queue", action="store_true",
+                    help="states without the queue words: the boundary kernel starts when the decode kernel has ended")
     ap.add_argument("--only-timed", action="store_true",
                     help="skip the CUDA-graph, end-to-end, baseline-kernel and CPU legs (for profiler runs)")
     ap.add_argument("--r", type=int, default=4, help="Compensator Tokens per state")
@@ -847,6 +852,8 @@ def main():
     ap.add_argument("--rec16", type=int, default=0, choices=[0, 1],
                     help="1: fp16 record buffer (the paper's storage) instead of the fp32 buffer of the headline")
     args = ap.parse_args()
+    global BOUNDARY_QUEUE
+    BOUNDARY_QUEUE = not args.no_queue
     if args.sweep:
         run_sweep(args)
         return

@@ -114,12 +114,21 @@ typedef struct {
  * decays: scalar gate only, fp32 [B,Hv,W]: the decay of each buffered record (ignored for the diagonal gate).
  * win_pos: int32 [B], records buffered per sequence, 0..W-1 between calls.  Bits 16 and up are used as a
  *     scratch counter while a call runs and are zero again when it has finished.
+ * work: optional (may be null): int32 [LQ_WORK_WORDS], all zero when the state is created and zero again after
+ *     every call.  With it, the decode kernel of lq_decode_step hands out the heads of its last, partial round
+ *     (B*Hv heads over the CTAs that are resident at once) to the CTAs that get there first, instead of giving
+ *     every CTA the same number of heads: on a GPU whose memory system does not serve all SMs alike, equal shares
+ *     do not take equal time.  Results are the same bit for bit either way.  Sub-batches of one state that are
+ *     addressed by pointer offset may share one `work` as long as their calls do not run at the same time (calls
+ *     in one stream never do).
  */
+#define LQ_WORK_WORDS 8
 typedef struct {
   uint8_t *heads;
   void *records;   /* float rows, or (shape.rec16) fp16 rows of the same element counts */
   float *decays;
   int32_t *win_pos;
+  int32_t *work;
 } lq_state;
 
 /* Size in bytes of one head block, and the number of fp32 values in one record row (0 for an invalid shape). */

@@ -33,6 +33,8 @@ __global__ void __launch_bounds__(256, 2) boundary_kernel(const Params p, const 
   LQ_STAMP(1, 0);
   grid_dependency_wait();                    // everything the kernel before this one wrote is visible from here on
   LQ_STAMP(1, 1);
+  // the decode kernel ahead of a flush counts the tickets of its pool of heads in the state's scratch words
+  if (MODE == 0 && p.work != nullptr && blockIdx.x == 0 && threadIdx.x == 0) p.work[0] = 0;
 #ifdef LQ_TIMING
   if (threadIdx.x == 0) { for (int i = 0; i < 16; i++) lq_bacc[i] = 0; lq_btick = clock64(); }
   bool first_flush_ = true;
@@ -301,6 +303,7 @@ static lq_status check_state(const lq_shape *s, const lq_state *st, bool need_bu
   lq_status rc = check_ptrs({st->heads});
   if (rc != LQ_OK) return rc;
   if ((rc = check_scalar_ptrs({st->win_pos}, 4)) != LQ_OK) return rc;
+  if (st->work && (reinterpret_cast<uintptr_t>(st->work) & 3u)) return LQ_ERR_ALIGN;
   if (need_buffers) {
     if ((rc = check_ptrs({st->records})) != LQ_OK) return rc;
     if (s->gate == LQ_GATE_SCALAR && (rc = check_scalar_ptrs({st->decays}, 4)) != LQ_OK) return rc;
@@ -314,6 +317,7 @@ static Params make_params(const lq_shape *s, const lq_state *st) {
   p.n_iter = s->n_iter; p.smooth = s->smooth; p.delta = s->delta; p.rec16 = s->rec16; p.force = 0;
   if (st) {
     p.heads = st->heads; p.records = st->records; p.decays = st->decays; p.win_pos = st->win_pos;
+    p.work = st->work;
   }
   return p;
 }
@@ -415,11 +419,12 @@ static lq_status launch_persistent(K kernel, long items, int block, size_t smem,
   const int per_sm = ctas_per_sm(reinterpret_cast<const void *>(kernel), block, smem);
   if (per_sm < 1) return LQ_ERR_CUDA;
   const long resident = (long)per_sm * sm_count();
-  // every CTA takes ceil(items / resident) items at most; the smallest grid with that property leaves no last
+  // Every CTA takes ceil(items / resident) items at most; the smallest grid with that property leaves no last
   // round in which a fraction of the CTAs works while the others have left (8192 heads: 820 CTAs of 10 heads
-  // instead of 888 of which 200 take a tenth)
+  // instead of 888 of which 200 take a tenth).  With scratch words in the state the items of a partial last round
+  // go to the CTAs that get there first (decode_slot), and every CTA that fits is launched.
   const long rounds = (items + resident - 1) / resident;
-  const long grid = (items + rounds - 1) / rounds;
+  const long grid = p.work != nullptr ? (items < resident ? items : resident) : (items + rounds - 1) / rounds;
   return launch_dependent(kernel, static_cast<int>(grid), block, smem, stream, p);
 }
 
@@ -1113,6 +1118,6 @@ const char *lq_status_string(lq_status status) {
   return "unknown status";
 }
 
-int lq_version(void) { return 6; }
+int lq_version(void) { return 7; }
 
 }  // extern "C"

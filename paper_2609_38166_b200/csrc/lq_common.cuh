@@ -40,6 +40,7 @@ struct Params {
   void *records;     // [B*Hv][W] record rows of record_floats(gate) elements, fp32 or (rec16) fp16
   float *decays;     // scalar gate: [B*Hv][W]
   int32_t *win_pos;
+  int32_t *work;     // lq_state.work (scratch words, zero between calls), or null
   const uint16_t *q, *k, *v, *beta, *alpha;
   float *o;
   float *S;          // dense fp32 states (quantize / dequantize / fp32 baseline)

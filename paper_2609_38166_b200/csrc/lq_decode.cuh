@@ -332,8 +332,46 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
 #ifdef LQ_TIMING
   tick_ = clock64();
 #endif
+  // Equal shares do not take equal time: pairs that share an SM with fewer others, or sit nearer the memory they
+  // read, are through with ten heads when others have done eight.  With scratch words in the state (lq_state.work)
+  // every pair therefore takes S = floor(nh / G) heads in turn, and the nh - S G heads that are left (heads S G + t)
+  // go to the pairs that reach their last head but one first: there the dot warp draws a ticket t (word 0 of the
+  // scratch words counts them; the boundary kernel behind this one puts it back to zero), hands it to the stream
+  // warp with the record terms (barrier 1), and at the end of the trip both warps load that head's scalars.
+  const bool draw = !FUSED && p.work != nullptr && nh >= 2 * G && nh % G != 0;
+  const int S = draw ? static_cast<int>(nh / G) : 0;
+  const unsigned pool = draw ? nh - static_cast<unsigned>(S) * G : 0;
+  unsigned *qidx = reinterpret_cast<unsigned *>(pk + r);      // (a spare word of the projection area)
+  unsigned ticket = 0xFFFFFFFFu;             // (dot warp, lane 0) what was drawn
   int idx = 0;                               // position of the head in this slot's list
-  for (; hd.bh < nh; hd = hd1, hd1.step(G, G_b, G_hv, Hv), idx++) {
+  // end of a trip; in the trip in which the ticket was drawn: the head it stands for becomes the pair's last one
+  auto finish_trip = [&]() {
+    unsigned extra = nh;
+    if (draw && idx == S - 2) {
+      const unsigned tk = role == 1 ? __shfl_sync(FULL, ticket, 0) : *reinterpret_cast<volatile unsigned *>(qidx);
+      if (tk < pool) {
+        extra = static_cast<unsigned>(S) * G + tk;
+        if (lane == (S & 31)) {
+          sc_n = p.win_pos[extra / Hv];
+          sc_beta = p.beta[extra];
+          if (!DIAG) sc_alpha = p.alpha[extra];
+        }
+      }
+    }
+    hd = hd1;
+    idx++;
+    hd1.step(G, G_b, G_hv, Hv);
+    if (draw && idx + 1 >= S) {              // what follows the last head taken in turn: the drawn head, then nothing
+      if (idx + 1 == S && extra < nh) {
+        const unsigned b_ = extra / Hv;
+        hd1 = HeadIdx{extra, b_, extra - b_ * Hv};
+      } else {
+        hd1 = HeadIdx{nh, 0u, 0u};
+      }
+    }
+  };
+  for (; hd.bh < nh; finish_trip()) {
+    if (draw && idx == S - 2 && role == 1 && lane == 0) ticket = static_cast<unsigned>(atomicAdd(p.work, 1));
     const size_t bh = hd.bh;
     const int n = __shfl_sync(FULL, sc_n, idx & 31) & 0xFFFF;
     const float beta = __uint_as_float(__shfl_sync(FULL, sc_beta, idx & 31) << 16);
@@ -351,6 +389,15 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
         load_token<GATE>(p, hd1, group, lane, role, nxt);
         if (role == 0) request_head(bh_next, n_next);
         else request_records(bh_next, n_next);
+      }
+      if (draw && idx == S - 2) {            // the ticket changes hands outside the usual place
+        if (role == 1) {
+          if (lane == 0) *qidx = ticket;
+          __syncwarp();
+          named_arrive(bar0 + 1);
+        } else {
+          named_wait(bar0 + 1);
+        }
       }
       continue;
     }
@@ -528,8 +575,9 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
       named_wait(bar0 + 2);                         // the stream warp has taken its sums out of y
       *reinterpret_cast<float4 *>(y + 4 * lane) = make_float4(rk_rec[0], rk_rec[1], rk_rec[2], rk_rec[3]);
       *reinterpret_cast<float4 *>(y + D + 4 * lane) = make_float4(rq_rec[0], rq_rec[1], rq_rec[2], rq_rec[3]);
+      if (draw && idx == S - 2 && lane == 0) *qidx = ticket;
       __syncwarp();
-      named_arrive(bar0 + 1);                       // the record terms are in shared memory
+      named_arrive(bar0 + 1);                       // the record terms are in shared memory (and the ticket)
       LQ_TICK(5);
       // append the key side of the record (and its decay)
       {
@@ -727,6 +775,14 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
   uint32_t parA = 0, parR = 0;
   decode_slot_init<GATE, R16, false>(p, lq_slot, lane, role, 0, blockIdx.x, gridDim.x, nullptr);
   decode_slot<GATE, R16, false, 0, LONGW>(p, lq_slot, lane, role, 0, blockIdx.x, gridDim.x, nullptr, parA, parR);
+  LQ_STAMP(0, 3);
+#ifdef LQ_TIMING
+  if (threadIdx.x == 0 && blockIdx.x < 1024) {
+    unsigned smid_;
+    asm volatile("mov.u32 %0, %smid;" : "=r"(smid_));
+    g_timeline[p.gen & 3][0][4][blockIdx.x] = smid_;
+  }
+#endif
 }
 
 }  // namespace lq

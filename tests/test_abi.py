@@ -38,7 +38,7 @@ def test_argument_errors_are_reported_before_any_launch(L):
     sh = lq.Shape(2, 4, 2)
     s = sh.c()
     null = C.c_void_p(None)
-    st = lq._State(*([None] * 4))
+    st = lq._State(*([None] * 5))
     # null shape / null state / null pointers inside the state
     assert L.lq_decode_step(null, C.byref(st), null, null, null, null, null, null, null) == 1
     assert L.lq_decode_step(C.byref(s), null, null, null, null, null, null, null, null) == 1
