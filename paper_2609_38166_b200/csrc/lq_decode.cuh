@@ -296,12 +296,26 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
     __syncwarp();
   };
 
+  // Equal shares do not take equal time: pairs that share an SM with fewer others, or sit nearer the memory they
+  // read, are through with ten heads when others have done eight.  With scratch words in the state (lq_state.work)
+  // every pair therefore takes only its first S heads in turn (DRAWN_ROUNDS rounds fewer than would fall to it), and
+  // the heads that are left (S G + t, t < pool) go to whoever gets there first: from its last turn but one on, the dot
+  // warp draws a ticket t in every trip, for the head two trips on (word 0 of the scratch words counts the tickets;
+  // the boundary kernel behind this one puts it back to zero), hands it to the stream warp with the record terms
+  // (barrier 1), and at the end of the trip both warps ask for that head's scalars, which they look at for the first
+  // time half a trip later (ext_*) and move to the lane registers of the other heads' at the end of the next trip.
+  // A pair stops when a ticket is beyond the pool.
+  const int rounds_all = static_cast<int>(nh / G);             // rounds in which every pair has a head
+  const int DRAWN_ROUNDS = rounds_all >= 6 ? 2 : 1;            // (with few rounds, more of them in turn)
+  const bool draw = !FUSED && p.work != nullptr && rounds_all >= 3;
+  const int S = draw ? rounds_all - DRAWN_ROUNDS : 0;
+  const unsigned pool = draw ? nh - static_cast<unsigned>(S) * G : 0;
   // Per-head scalars of this CTA's heads, 32 heads at a time: lane l holds those of the CTA's (32*batch+l)-th head
   int sc_n = 0;
   uint32_t sc_beta = 0, sc_alpha = 0;
   auto load_scalars = [&](unsigned first_bh) {
     const unsigned bh = first_bh + lane * G;  // (once per 32 heads: a division is fine here)
-    if (bh < nh) {
+    if (bh < (draw ? static_cast<unsigned>(S) * G : nh)) {     // (the heads taken in turn)
       sc_n = FUSED ? nbuf[(first_bh - first) / G + lane]
                    : p.win_pos[bh / Hv];    // bits 16.. are the arrival counter of this launch: masked at use
       sc_beta = p.beta[bh];
@@ -332,46 +346,42 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
 #ifdef LQ_TIMING
   tick_ = clock64();
 #endif
-  // Equal shares do not take equal time: pairs that share an SM with fewer others, or sit nearer the memory they
-  // read, are through with ten heads when others have done eight.  With scratch words in the state (lq_state.work)
-  // every pair therefore takes S = floor(nh / G) heads in turn, and the nh - S G heads that are left (heads S G + t)
-  // go to the pairs that reach their last head but one first: there the dot warp draws a ticket t (word 0 of the
-  // scratch words counts them; the boundary kernel behind this one puts it back to zero), hands it to the stream
-  // warp with the record terms (barrier 1), and at the end of the trip both warps load that head's scalars.
-  const bool draw = !FUSED && p.work != nullptr && nh >= 2 * G && nh % G != 0;
-  const int S = draw ? static_cast<int>(nh / G) : 0;
-  const unsigned pool = draw ? nh - static_cast<unsigned>(S) * G : 0;
   unsigned *qidx = reinterpret_cast<unsigned *>(pk + r);      // (a spare word of the projection area)
-  unsigned ticket = 0xFFFFFFFFu;             // (dot warp, lane 0) what was drawn
+  unsigned ticket = 0xFFFFFFFFu;             // (dot warp, lane 0) what was drawn in this trip
+  bool drawing = draw;                       // no ticket has been beyond the pool yet
+  int ext_n = 0;                             // scalars of the head drawn a trip ago, on their way
+  uint32_t ext_beta = 0, ext_alpha = 0;
   int idx = 0;                               // position of the head in this slot's list
-  // end of a trip; in the trip in which the ticket was drawn: the head it stands for becomes the pair's last one
+  // end of a trip
   auto finish_trip = [&]() {
-    unsigned extra = nh;
-    if (draw && idx == S - 2) {
+    // the next head, if it was drawn: its scalars, asked for a trip ago, go where the others' are
+    if (draw && idx + 1 >= S && lane == ((idx + 1) & 31)) { sc_n = ext_n; sc_beta = ext_beta; sc_alpha = ext_alpha; }
+    unsigned extra = nh;                     // the head after the next one, if it is a drawn one
+    if (drawing && idx + 2 >= S) {
       const unsigned tk = role == 1 ? __shfl_sync(FULL, ticket, 0) : *reinterpret_cast<volatile unsigned *>(qidx);
       if (tk < pool) {
         extra = static_cast<unsigned>(S) * G + tk;
-        if (lane == (S & 31)) {
-          sc_n = p.win_pos[extra / Hv];
-          sc_beta = p.beta[extra];
-          if (!DIAG) sc_alpha = p.alpha[extra];
-        }
+        ext_n = p.win_pos[extra / Hv];
+        ext_beta = p.beta[extra];
+        if (!DIAG) ext_alpha = p.alpha[extra];
+      } else {
+        drawing = false;
       }
     }
     hd = hd1;
     idx++;
-    hd1.step(G, G_b, G_hv, Hv);
-    if (draw && idx + 1 >= S) {              // what follows the last head taken in turn: the drawn head, then nothing
-      if (idx + 1 == S && extra < nh) {
-        const unsigned b_ = extra / Hv;
-        hd1 = HeadIdx{extra, b_, extra - b_ * Hv};
-      } else {
-        hd1 = HeadIdx{nh, 0u, 0u};
-      }
+    if (!draw || idx + 1 < S) {
+      hd1.step(G, G_b, G_hv, Hv);
+    } else if (extra < nh) {
+      const unsigned b_ = extra / Hv;
+      hd1 = HeadIdx{extra, b_, extra - b_ * Hv};
+    } else {
+      hd1 = HeadIdx{nh, 0u, 0u};
     }
   };
   for (; hd.bh < nh; finish_trip()) {
-    if (draw && idx == S - 2 && role == 1 && lane == 0) ticket = static_cast<unsigned>(atomicAdd(p.work, 1));
+    const bool draws = drawing && idx + 2 >= S;                 // a ticket is drawn in this trip
+    if (draws && role == 1 && lane == 0) ticket = static_cast<unsigned>(atomicAdd(p.work, 1));
     const size_t bh = hd.bh;
     const int n = __shfl_sync(FULL, sc_n, idx & 31) & 0xFFFF;
     const float beta = __uint_as_float(__shfl_sync(FULL, sc_beta, idx & 31) << 16);
@@ -379,18 +389,25 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
     // the next head's scalars: from the next batch when this head is the last of its batch
     const unsigned bh_next = hd1.bh;
     if ((idx & 31) == 31) load_scalars(bh_next);
-    const int n_next = bh_next < nh ? (__shfl_sync(FULL, sc_n, (idx + 1) & 31) & 0xFFFF) : W;
-    const bool active = wanted(n), next_active = wanted(n_next);
+    // The next head's window position.  Of a drawn head it is still on its way (ext_n, asked for at the end of the
+    // trip before): it is looked at only where the head's data is requested, half a trip from here; until then the
+    // head counts as one that gets a token (its token is loaded, which does no harm if it gets none).
+    const bool next_drawn = draw && idx + 1 >= S;
+    const int n_next_turn = bh_next < nh ? (__shfl_sync(FULL, sc_n, (idx + 1) & 31) & 0xFFFF) : W;
+    auto n_next_now = [&]() { return next_drawn ? (bh_next < nh ? (ext_n & 0xFFFF) : W) : n_next_turn; };
+    const bool next_token = next_drawn ? bh_next < nh : wanted(n_next_turn);
+    const bool active = wanted(n);
     const int b = static_cast<int>(hd.b);
     LQ_TICK(0);
 
     if (!active) {                           // nothing was requested for this head; keep the pipeline going
-      if (next_active) {
+      const int n_next = n_next_now();
+      if (wanted(n_next)) {
         load_token<GATE>(p, hd1, group, lane, role, nxt);
         if (role == 0) request_head(bh_next, n_next);
         else request_records(bh_next, n_next);
       }
-      if (draw && idx == S - 2) {            // the ticket changes hands outside the usual place
+      if (draws) {                           // the ticket changes hands outside the usual place
         if (role == 1) {
           if (lane == 0) *qidx = ticket;
           __syncwarp();
@@ -416,7 +433,7 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
       bas[lane] = nxt.ba_lo;
       bas[lane + 32] = nxt.ba_hi;
     }
-    if (next_active) load_token<GATE>(p, hd1, group, lane, role, nxt);       // used one trip from now
+    if (next_token) load_token<GATE>(p, hd1, group, lane, role, nxt);        // used one trip from now
     // scalar gate: Gamma_{1:l}, the chain of decays from the newest record back (Appendix B.2), needs nothing
     // from the slot, so the stream warp takes it before it waits
     float gsc = alpha_s;
@@ -571,11 +588,14 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
       named_arrive(bar0 + 3);                       // the compensator projections are in pk, pq; this warp is done with the head block
       LQ_TICK(4);
       if (DIAG) named_wait(bar0 + 4);               // diagonal gate: the stream warp read the records' decays too
-      if (next_active) request_records(bh_next, n_next);
+      {
+        const int n_next = n_next_now();
+        if (wanted(n_next)) request_records(bh_next, n_next);
+      }
       named_wait(bar0 + 2);                         // the stream warp has taken its sums out of y
       *reinterpret_cast<float4 *>(y + 4 * lane) = make_float4(rk_rec[0], rk_rec[1], rk_rec[2], rk_rec[3]);
       *reinterpret_cast<float4 *>(y + D + 4 * lane) = make_float4(rq_rec[0], rq_rec[1], rq_rec[2], rq_rec[3]);
-      if (draw && idx == S - 2 && lane == 0) *qidx = ticket;
+      if (draws && lane == 0) *qidx = ticket;
       __syncwarp();
       named_arrive(bar0 + 1);                       // the record terms are in shared memory (and the ticket)
       LQ_TICK(5);
@@ -731,7 +751,10 @@ __device__ __forceinline__ void decode_slot(const Params &p, unsigned char *slot
           for (int e = 0; e < 4; e++) { rk[e] = fmaf(uc[e], pkh, rk[e]); rq[e] = fmaf(uc[e], pqh, rq[e]); }
         }
         __syncwarp();                        // nobody reads the head block any more (the dot warp finished with
-        if (next_active) request_head(bh_next, n_next);   // it before barrier 3): the next head's may land
+        {
+          const int n_next = n_next_now();
+          if (wanted(n_next)) request_head(bh_next, n_next);   // it before barrier 3): the next head's may land
+        }
         named_wait(bar0 + 1);                       // the record terms are complete
         {
           const float4 tk = *reinterpret_cast<const float4 *>(y + 4 * lane);
