@@ -51,11 +51,11 @@ def metric_name(wl) -> str:
 # DRAM bytes per launch from the ncu captures summarised under profiles/ (dram__bytes_read.sum +
 # dram__bytes_write.sum of one full-batch launch of the gdn_b256 workload, W = 16), or None when not captured.
 NCU_CAPTURE_N_ITER = 1                                # (the captures were taken with the default number of rounds)
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"decode_kernel": 235.0e6, "boundary_kernel": 18.5e6}
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"decode_kernel": 232.9e6, "boundary_kernel": 18.5e6}
 # The same two counters from a launch list taken with --cache-control none (the caches are left as the kernel ahead
 # left them, as in a real step): what the L2 serves - the records written by the last tokens, the token vectors, and
 # for the boundary kernel the heads the decode kernel asked the L2 to keep - no longer comes from DRAM.
-NCU_TRAFFIC_WARM_BYTES_PER_LAUNCH = {"decode_kernel": 194.5e6, "boundary_kernel": 1.4e6}
+NCU_TRAFFIC_WARM_BYTES_PER_LAUNCH = {"decode_kernel": 195.1e6, "boundary_kernel": 2.2e6}
 
 
 def record_bytes(diag: bool, rec16: int) -> int:
