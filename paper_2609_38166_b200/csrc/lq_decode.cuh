@@ -108,6 +108,10 @@ __device__ __forceinline__ void bulk_g2s_hint(uint32_t dst, const void *src, uin
       "l"(src), "r"(bytes), "r"(bar), "l"(policy)
       : "memory");
 }
+// Ask the L2 for a piece of global memory (no data comes back, nothing waits for it).
+__device__ __forceinline__ void bulk_prefetch_l2(const void *src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(src), "r"(bytes) : "memory");
+}
 // Bounded wait for phase `parity`; false if the limit of LIMIT polls ran out (the caller then reports and bails out).
 template <int LIMIT = (1 << 20)>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
@@ -792,7 +796,12 @@ template <int GATE, bool R16, bool LONGW>
 __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
   extern __shared__ __align__(128) unsigned char lq_slot[];
   LQ_STAMP(0, 0);
-  grid_dependency_wait();                    // no global memory is touched above this line
+  // Resident while the kernel ahead drains: the CTA asks the L2 for its first head block meanwhile (a prefetch returns
+  // no data, so it does not matter that the kernel ahead may still be writing that block: the L2 is where its writes
+  // go).  The first head of a CTA is the only one whose copy nothing hides.
+  if (threadIdx.x == 0 && blockIdx.x < static_cast<unsigned>(p.batch) * p.heads_v)
+    bulk_prefetch_l2(p.head(blockIdx.x), head_bytes(p.r));
+  grid_dependency_wait();                    // no data in global memory is read or written above this line
   LQ_STAMP(0, 1);
   const int lane = threadIdx.x & 31, role = threadIdx.x >> 5;
   uint32_t parA = 0, parR = 0;
