@@ -253,7 +253,7 @@ def run_reference(args, wl):
 # --------------------------------------------------------------------------------------------------
 # CUDA arm
 # --------------------------------------------------------------------------------------------------
-BOUNDARY_QUEUE = True     # --no-queue: states without lq_state.work (the boundary kernel starts after the decode kernel)
+SCRATCH_WORDS = True      # --no-scratch-words: states without lq_state.work (every decode CTA takes an equal share of heads)
 
 
 def to_dev(tok, torch):
@@ -266,7 +266,7 @@ def prepare_state(wl, lq, torch, log, WARM_TOKENS=WARM_TOKENS):
     sh = lq.Shape(wl.batch, wl.heads_v, wl.heads_qk, wl.d_k, wl.d_v, wl.W, wl.r, wl.n_iter, wl.gate, wl.smooth, wl.delta,
                   wl.rec16, wl.state_bf16)
     B, W = wl.batch, wl.W
-    st = lq.State(sh, queue=BOUNDARY_QUEUE)
+    st = lq.State(sh, work=SCRATCH_WORDS)
     S = torch.zeros((B, wl.heads_v, wl.d_k, wl.d_v), dtype=torch.float32, device="cuda")
     o = torch.empty((B, wl.heads_v, wl.d_v), dtype=torch.float32, device="cuda")
     per = max(B // W, 1)
@@ -827,8 +827,8 @@ def main():
     ap.add_argument("--warm-tokens", type=int, default=WARM_TOKENS,
                     help="tokens of the fp32 recurrence that pre-fill the states (512 in the headline workload)")
     ap.add_argument("--no-graph", action="store_true", help="time plain launches instead of CUDA-graph replays")
-    ap.add_argument("--no-queue", action="store_true",
-                    help="states without the queue words: the boundary kernel starts when the decode kernel has ended")
+    ap.add_argument("--no-scratch-words", action="store_true",
+                    help="states without lq_state.work: every CTA of the decode kernel takes an equal share of the heads")
     ap.add_argument("--only-timed", action="store_true",
                     help="skip the CUDA-graph, end-to-end, baseline-kernel and CPU legs (for profiler runs)")
     ap.add_argument("--r", type=int, default=4, help="Compensator Tokens per state")
@@ -852,8 +852,8 @@ def main():
     ap.add_argument("--rec16", type=int, default=0, choices=[0, 1],
                     help="1: fp16 record buffer (the paper's storage) instead of the fp32 buffer of the headline")
     args = ap.parse_args()
-    global BOUNDARY_QUEUE
-    BOUNDARY_QUEUE = not args.no_queue
+    global SCRATCH_WORDS
+    SCRATCH_WORDS = not args.no_scratch_words
     if args.sweep:
         run_sweep(args)
         return

@@ -109,14 +109,14 @@ class State:
     ``decays`` (scalar gate) and ``win_pos``.  The named pieces (codes, col_scale, row_smooth, comp_k,
     comp_u, buf_k, buf_u, buf_a) are strided views into those tensors."""
 
-    def __init__(self, sh: Shape, device="cuda", storage=None, queue=True):
+    def __init__(self, sh: Shape, device="cuda", storage=None, work=True):
         """``storage``: optionally the four tensors (heads, records, decays, win_pos) to use instead of fresh
         ones - contiguous, of the shapes and dtypes below (callers that place the state in memory of their own).
-        ``queue``: give the state the ``work`` words (LQ_WORK_WORDS) with which the decode kernel hands out the heads
+        ``work``: give the state the ``work`` words (LQ_WORK_WORDS) with which the decode kernel hands out the heads
         of its last round to the CTAs that get there first; without them every CTA takes the same number."""
         B, H, K, V, W, r = sh.batch, sh.heads_v, sh.d_k, sh.d_v, sh.W, sh.r
         self.shape = sh
-        self.work = torch.zeros((8,), dtype=torch.int32, device=device) if queue else None
+        self.work = torch.zeros((8,), dtype=torch.int32, device=device) if work else None
         hb, rf = head_bytes(sh), record_floats(sh)
         assert hb > 0 and rf > 0, "shape not supported by the library"
         rec_dtype = torch.float16 if sh.rec16 else torch.float32

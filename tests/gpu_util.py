@@ -37,8 +37,8 @@ def tok_dev(tok: dict) -> dict:
     return {k: dev(v) for k, v in tok.items()}
 
 
-def state_to_dev(ost: OState, lsh, queue: bool = True) -> "lq.State":
-    st = lq.State(lsh, queue=queue)
+def state_to_dev(ost: OState, lsh, work: bool = True) -> "lq.State":
+    st = lq.State(lsh, work=work)
     if lsh.state_bf16:
         st.state16.copy_(dev(np.ascontiguousarray(ost.S0.transpose(0, 1, 3, 2))).to(torch.bfloat16))   # exact: bfloat16 values
         st.buf_k.copy_(dev(ost.buf_k)); st.buf_u.copy_(dev(ost.buf_u)); st.buf_a.copy_(dev(ost.buf_a))

@@ -64,6 +64,9 @@ def test_argument_errors_are_reported_before_any_launch(L):
     st_bad = lq._State(*fake)
     assert L.lq_quantize_state(C.byref(s), C.c_void_p(0x100000), C.byref(st_bad), null) == 3
     assert L.lq_quantize_state(C.byref(s), C.c_void_p(0x100004), C.byref(st_ok), null) == 3
+    # the optional scratch words: null is fine (checked above), a pointer that is not 4-byte aligned is not
+    st_w = lq._State(*[0x1000 * (i + 1) for i in range(4)], 0x5002)
+    assert L.lq_quantize_state(C.byref(s), C.c_void_p(0x100000), C.byref(st_w), null) == 3
     # the host-buffer entry points check the state as well before they enqueue anything (fake host / stage pointers)
     hp = C.c_void_p(0x200000)
     assert L.lq_decode_step_host(C.byref(s), null, hp, hp, hp, hp, hp, hp, hp, null) == 1

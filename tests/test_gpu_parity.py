@@ -82,18 +82,18 @@ def test_reference_kernels(oracle, gate):
     assert np.array_equal(gu.host(S16d), S16)
 
 
-def _run_chain(oracle, wl, steps, init="zero", stagger=False, check_every=1, queue=True):
+def _run_chain(oracle, wl, steps, init="zero", stagger=False, check_every=1, work=True):
     osh, lsh = gu.shapes(wl)
     ost = OState(osh)
     S0 = np.zeros((wl.batch, wl.heads_v, 128, 128), np.float32) if init == "zero" else synth.dense_states(wl, 9)
     oracle.quantize_state(osh, S0, ost)
-    st = lq.State(lsh, queue=queue)
+    st = lq.State(lsh, work=work)
     lq.quantize_state(lsh, gu.dev(S0), st)
     if stagger:       # window positions spread over [0, W): pre-fill with harmless records of zero update
         pos = (np.arange(wl.batch) * wl.W // max(wl.batch, 1)).astype(np.int32) % wl.W
         ost.win_pos[:] = pos
         ost.buf_a[...] = 1.0
-        st = gu.state_to_dev(ost, lsh, queue=queue)
+        st = gu.state_to_dev(ost, lsh, work=work)
     o = torch.empty((wl.batch, wl.heads_v, 128), dtype=torch.float32, device="cuda")
     for step in range(steps):
         tok = synth.token_inputs(wl, step)
@@ -209,16 +209,17 @@ def test_fused_step_kernel_gives_the_same_bits(oracle, gate, monkeypatch):
 
 
 @pytest.mark.parametrize("gate", GATES)
-@pytest.mark.parametrize("queue", [False, True])
-def test_heads_of_the_last_round_are_drawn(oracle, gate, queue):
-    """More than two heads per resident CTA, with a remainder: with the scratch words in the state (lq_state.work)
-    the decode kernel hands the heads of the partial last round to the CTAs that get there first, without them every
-    CTA takes the heads that fall to it in turn.  Same chain, same oracle, bit for bit; the words are zero after
-    every call."""
-    wl = synth.Workload("pool", 62, 32, 16, W=4, r=2, gate=gate, seed=496)
-    _, st = _run_chain(oracle, wl, 6, init="dense", stagger=True, check_every=2, queue=queue)
-    assert (st.work is not None) == queue
-    if queue:
+@pytest.mark.parametrize("work", [False, True])
+def test_heads_of_the_last_round_are_drawn(oracle, gate, work):
+    """More than three heads per resident CTA: with the scratch words in the state (lq_state.work) the decode kernel
+    hands the heads of its last rounds to the CTAs that get there first (here every CTA takes two heads in turn and
+    the other third of the heads is drawn; the full-size tests have seven in turn and two rounds drawn), without them
+    every CTA takes the heads that fall to it in turn.  Same chain, same oracle, bit for bit; the words are zero
+    after every call."""
+    wl = synth.Workload("pool", 90, 32, 16, W=4, r=2, gate=gate, seed=496)
+    _, st = _run_chain(oracle, wl, 6, init="dense", stagger=True, check_every=2, work=work)
+    assert (st.work is not None) == work
+    if work:
         assert int(st.work.abs().sum().item()) == 0
     assert lq.check_device() == 0
 
