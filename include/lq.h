@@ -120,7 +120,8 @@ typedef struct {
  *     every CTA the same number of heads: on a GPU whose memory system does not serve all SMs alike, equal shares
  *     do not take equal time.  Results are the same bit for bit either way.  Sub-batches of one state that are
  *     addressed by pointer offset may share one `work` as long as their calls do not run at the same time (calls
- *     in one stream never do).
+ *     in one stream never do).  After a call that returned LQ_ERR_CUDA the words are to be zeroed again (and the
+ *     state restored from a checkpoint: a step that was enqueued in part leaves neither valid).
  */
 #define LQ_WORK_WORDS 8
 typedef struct {
