@@ -801,11 +801,11 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
   // go).  The first head of a CTA is the only one whose copy nothing hides.
   if (threadIdx.x == 0 && blockIdx.x < static_cast<unsigned>(p.batch) * p.heads_v)
     bulk_prefetch_l2(p.head(blockIdx.x), head_bytes(p.r));
-  grid_dependency_wait();                    // no data in global memory is read or written above this line
-  LQ_STAMP(0, 1);
   const int lane = threadIdx.x & 31, role = threadIdx.x >> 5;
   uint32_t parA = 0, parR = 0;
-  decode_slot_init<GATE, R16, false>(p, lq_slot, lane, role, 0, blockIdx.x, gridDim.x, nullptr);
+  decode_slot_init<GATE, R16, false>(p, lq_slot, lane, role, 0, blockIdx.x, gridDim.x, nullptr);      // (shared memory only)
+  grid_dependency_wait();                    // no data in global memory is read or written above this line
+  LQ_STAMP(0, 1);
   decode_slot<GATE, R16, false, 0, LONGW>(p, lq_slot, lane, role, 0, blockIdx.x, gridDim.x, nullptr, parA, parR);
   LQ_STAMP(0, 3);
 #ifdef LQ_TIMING
