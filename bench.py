@@ -759,6 +759,55 @@ def run_ladder(args):
 
 
 # --------------------------------------------------------------------------------------------------
+# --timeline: where a step's time goes.  Runs the headline workload on the library variant with per-CTA time
+# stamps (python -m paper_2609_38166_b200.build --stamps; thread 0 of every CTA reads the GPU's global timer when it
+# becomes resident, when its wait for the kernel ahead ends, when its first head's data is there and when it leaves)
+# and prints, for three consecutive steps, the spread of those moments over the CTAs of both kernels.  Not a
+# measurement of throughput: the stamps cost a little, and nothing here is timed from the host.
+# --------------------------------------------------------------------------------------------------
+def run_timeline(args):
+    import ctypes
+    import torch
+    from paper_2609_38166_b200 import build, lq
+
+    torch.cuda.set_device(0)
+    log = lambda m: print(f"[timeline] {m}", file=sys.stderr, flush=True)
+    lq._LIB_PATH = build.build(stamps=True)
+    L = lq.lib()
+    wl = synth.config("gdn_b256").with_(W=args.W, batch=args.batch, r=args.r, rec16=args.rec16)
+    if args.gate == "kda":
+        wl = wl.with_(gate=synth.GATE_DIAG, heads_qk=wl.heads_v)
+    sh, st, o = prepare_state(wl, lq, torch, log, min(args.warm_tokens, 64))
+    toks = [to_dev(synth.token_inputs(wl, 64 + t), torch) for t in range(wl.W)]
+    for t in range(4 * wl.W + 4):                       # (the stamps of the last four steps are kept)
+        d = toks[t % wl.W]
+        lq.decode_step(sh, st, d["q"], d["k"], d["v"], d["beta"], d["alpha"], o)
+    torch.cuda.synchronize()
+    buf = np.zeros((4, 2, 6, 1024), dtype=np.uint64)
+    if L.lq_debug_timeline(buf.ctypes.data_as(ctypes.c_void_p)) != 0:
+        raise RuntimeError("lq_debug_timeline failed")
+    tl = buf.astype(np.int64)
+    gd, gb = int((tl[0, 0, 1] != 0).sum()), int((tl[0, 1, 1] != 0).sum())
+    pct = lambda a, t0: [round(float(np.percentile((a - t0) / 1e3, q)), 2) for q in (0, 10, 50, 90, 100)]
+    steps = []
+    order = sorted(range(4), key=lambda g_: tl[g_, 0, 1, :gd].min())       # the four generations, oldest first
+    for g, g_next in zip(order[:3], order[1:]):
+        t0 = tl[g, 0, 1, :gd].min()
+        steps.append({
+            "decode_resident": pct(tl[g, 0, 0, :gd], t0), "decode_first_head_there": pct(tl[g, 0, 2, :gd], t0),
+            "decode_leaves": pct(tl[g, 0, 3, :gd], t0),
+            "boundary_resident": pct(tl[g, 1, 0, :gb], t0), "boundary_wait_over": pct(tl[g, 1, 1, :gb], t0),
+            "boundary_first_head_staged": pct(tl[g, 1, 2, :gb], t0), "boundary_first_head_done": pct(tl[g, 1, 3, :gb], t0),
+            "boundary_leaves": pct(tl[g, 1, 4, :gb], t0),
+            "next_decode_wait_over": round(float(tl[g_next, 0, 1, :gd].min() - t0) / 1e3, 2)})
+    print(json.dumps({"timeline": True, "workload": wl.name, "gate": args.gate, "batch": wl.batch, "W": wl.W, "r": wl.r,
+                      "unit": "us after the decode kernel's wait for the kernel ahead is over; "
+                              "[min, 10 %, median, 90 %, max] over the CTAs",
+                      "decode_ctas": gd, "boundary_ctas": gb, "steps": steps,
+                      "device_error_flags": lq.check_device()}))
+
+
+# --------------------------------------------------------------------------------------------------
 # Long-chain drift: GDN, 64 x 16 heads, heavy-tailed values, 4096 consecutive tokens, W = 16.  Error of o of
 # the 8-bit per-window path (and of the bf16-state baseline) against the fp32 recurrence fed the same tokens,
 # per block of 256 steps.  All on the GPU through the library; the code parity of the same chain against the
@@ -843,6 +892,8 @@ def main():
                     help="long-chain drift of the 8-bit path and of the bf16-state baseline against the fp32 recurrence, "
                          "per 256 steps (GDN 64 x 16 heads, Student-t values)")
     ap.add_argument("--drift-steps", type=int, default=4096)
+    ap.add_argument("--timeline", action="store_true",
+                    help="per-CTA time stamps of both kernels over three steps (library variant built with --stamps)")
     ap.add_argument("--sweep-batches", default="32,128,256,512,1024")
     ap.add_argument("--sweep-W", default="8,16,32,64")
     ap.add_argument("--sweep-r", default="4,8")
@@ -862,6 +913,9 @@ def main():
         return
     if args.drift:
         run_drift(args)
+        return
+    if args.timeline:
+        run_timeline(args)
         return
     wl = synth.config("gdn_b256").with_(W=args.W, batch=args.batch, r=args.r)
     if args.gate == "kda":

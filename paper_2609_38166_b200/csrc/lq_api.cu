@@ -31,6 +31,13 @@ __global__ void __launch_bounds__(256, 2) boundary_kernel(const Params p, const 
   __shared__ uint32_t todo_mask;
   __shared__ int todo_n[32];
   LQ_STAMP(1, 0);
+#ifdef LQ_TIMING
+  if (threadIdx.x == 0 && blockIdx.x < 1024) {
+    unsigned smid_;
+    asm volatile("mov.u32 %0, %smid;" : "=r"(smid_));
+    g_timeline[p.gen & 3][1][5][blockIdx.x] = smid_;
+  }
+#endif
   grid_dependency_wait();                    // everything the kernel before this one wrote is visible from here on
   LQ_STAMP(1, 1);
   // the decode kernel ahead of a flush counts the tickets of its pool of heads in the state's scratch words

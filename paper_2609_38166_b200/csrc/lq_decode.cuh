@@ -814,6 +814,11 @@ __global__ void __launch_bounds__(64, 6) decode_kernel(const Params p) {
     asm volatile("mov.u32 %0, %smid;" : "=r"(smid_));
     g_timeline[p.gen & 3][0][4][blockIdx.x] = smid_;
   }
+  if (threadIdx.x == 32 && blockIdx.x < 1024) {          // the dot warp's last instruction
+    unsigned long long t_;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_));
+    g_timeline[p.gen & 3][0][5][blockIdx.x] = t_;
+  }
 #endif
 }
 
